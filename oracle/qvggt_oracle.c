@@ -1,0 +1,285 @@
+/*
+ * CPU ORACLE -- TEST INFRASTRUCTURE ONLY.
+ *
+ * Plain, slow, scalar restatement of the W4A4 linear layer of Dual-Smoothed Fine-Grained
+ * Quantization (Sec. 3.2 of the QuantVGGT paper), written step by step from the paper's
+ * formulas.  It shares no code with the CUDA path and must never be called from it; only the
+ * tests, the smoke check and the CPU-baseline leg of the benchmark use it.
+ *
+ * Build: gcc -O2 -ffp-contract=off -fopenmp (no fast-math; OpenMP only across independent rows).
+ * "fl(.)" below is one IEEE-754 binary32 round-to-nearest-even operation; no FMA is ever formed.
+ *
+ * Pins (see tests/test_oracle_pins.py): Sylvester closed form (-1)^popcount(i&j), H H^T = K I,
+ * brute-force dense +-1 products on integer inputs, fp64 rotation/smoothing invariance,
+ * |y - scale*q| <= scale/2, hand-built rounding ties, brute-force integer GEMMs, fp64 epilogue.
+ * Unpinned by the paper (this build's conventions): the fp32 butterfly stage order, the
+ * group-wise (per 128 channels) variant for G < K, and the end-to-end layer error vs. the
+ * unquantized layer ("parity unpinned": information only).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+static inline float orc_bf16_to_f32(uint16_t b)
+{
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+/* binary32 -> bf16 bits, round to nearest even; NaN stays NaN. */
+static inline uint16_t orc_f32_to_bf16(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)((u >> 16) | 0x0040u);
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+/*
+ * Un-normalized Sylvester-Hadamard transform of one row, in place (pre-global rotation; the
+ * Kronecker recursion H_{2^n} = H_2 (x) H_{2^{n-1}} of Sec. 3.2 unrolled into radix-2 stages).
+ * Stage order is ascending stride h = 1, 2, 4, ..., K/2; each butterfly is
+ * (a, b) -> (fl(a+b), fl(a-b)).  The result equals u * H_K with H_K[i][j] = (-1)^popcount(i&j),
+ * H_K H_K^T = K I.
+ */
+void orc_fwht_f32(float *u, int K)
+{
+    for (int h = 1; h < K; h <<= 1)
+        for (int i = 0; i < K; ++i)
+            if (!(i & h)) {
+                float a = u[i], b = u[i + h];
+                u[i] = a + b;
+                u[i + h] = a - b;
+            }
+}
+
+void orc_fwht_f64(double *u, int K)
+{
+    for (int h = 1; h < K; h <<= 1)
+        for (int i = 0; i < K; ++i)
+            if (!(i & h)) {
+                double a = u[i], b = u[i + h];
+                u[i] = a + b;
+                u[i + h] = a - b;
+            }
+}
+
+/* K^{-1/2}: an exact power of two when log2 K is even (K = 1024, 4096). */
+static float orc_norm(int K)
+{
+    return (float)(1.0 / sqrt((double)K));
+}
+
+/*
+ * Per-rotated-channel multipliers.  With the random Hadamard H = K^{-1/2} H_K diag(v) and the
+ * smoothing identity  X W^T = (X H diag(c)^-1)(diag(c) H^T W^T)  (Eq. "smooth_factor"):
+ *   amul[k] = fl( (v_k K^{-1/2}) / c_k )   applied to rotated activations,
+ *   wmul[k] = fl( (v_k K^{-1/2}) * c_k )   applied to rotated weight rows.
+ * v may be NULL (all +1).
+ */
+void orc_multipliers(const float *c, const int8_t *v, int K, float *amul, float *wmul)
+{
+    float nrm = orc_norm(K);
+    for (int k = 0; k < K; ++k) {
+        float s = (v && v[k] < 0) ? -nrm : nrm;
+        amul[k] = s / c[k];
+        wmul[k] = s * c[k];
+    }
+}
+
+/*
+ * Rotate -> smooth -> symmetric 4-bit quantize, row by row (Eq. "quantization" with N = 4:
+ * Delta = max|y| / 7, q = clamp(round(y / Delta), -8, 7)).
+ *   X      bf16 bits [M, K], row stride ldx elements
+ *   mul    fp32 [K] (amul for activations, wmul for weight rows)
+ *   group  scale granularity along K: 0 = one scale per row (the paper's token-wise /
+ *          out-channel-wise setting); g > 0 = one scale per g consecutive rotated channels
+ *   codes  int8 [M, K], values in [-8, 7] (in fact [-7, 7])
+ *   scales fp32 [M, K/group]
+ * Reading of the unspecified points: round() is round-half-to-even; y/Delta is evaluated as the
+ * exact product y * fl(7/amax) rounded once to an integer; an all-zero group gets amax = 1e-8.
+ */
+void orc_rotate_smooth_quantize(const uint16_t *X, int64_t ldx, int64_t M, int K, const float *mul,
+                                int group, int8_t *codes, float *scales)
+{
+    int G = group > 0 ? K / group : 1;
+    int glen = group > 0 ? group : K;
+#pragma omp parallel
+    {
+        float *u = (float *)malloc(sizeof(float) * (size_t)K);
+#pragma omp for schedule(static)
+        for (int64_t m = 0; m < M; ++m) {
+            const uint16_t *x = X + m * ldx;
+            for (int k = 0; k < K; ++k) u[k] = orc_bf16_to_f32(x[k]);
+            orc_fwht_f32(u, K);
+            for (int k = 0; k < K; ++k) u[k] = u[k] * mul[k];
+            for (int g = 0; g < G; ++g) {
+                const float *y = u + g * glen;
+                float amax = 0.0f;
+                for (int k = 0; k < glen; ++k) {
+                    float a = fabsf(y[k]);
+                    if (a > amax) amax = a;
+                }
+                if (amax < 1e-8f) amax = 1e-8f;
+                float scale = amax / 7.0f;
+                float inv = 7.0f / amax;
+                scales[m * G + g] = scale;
+                int8_t *q = codes + m * K + g * glen;
+                for (int k = 0; k < glen; ++k) {
+                    double r = nearbyint((double)y[k] * (double)inv); /* exact product, one rounding */
+                    if (r < -8.0) r = -8.0;
+                    if (r > 7.0) r = 7.0;
+                    q[k] = (int8_t)r;
+                }
+            }
+        }
+        free(u);
+    }
+}
+
+/* Canonical packed layout: byte i of a row = code 2i in bits 0-3, code 2i+1 in bits 4-7 (two's complement). */
+void orc_pack_int4(const int8_t *codes, int64_t rows, int K, uint8_t *packed)
+{
+    for (int64_t r = 0; r < rows; ++r)
+        for (int i = 0; i < K / 2; ++i) {
+            uint8_t lo = (uint8_t)codes[r * K + 2 * i] & 0xF;
+            uint8_t hi = (uint8_t)codes[r * K + 2 * i + 1] & 0xF;
+            packed[r * (K / 2) + i] = (uint8_t)(lo | (hi << 4));
+        }
+}
+
+void orc_unpack_int4(const uint8_t *packed, int64_t rows, int K, int8_t *codes)
+{
+    for (int64_t r = 0; r < rows; ++r)
+        for (int i = 0; i < K / 2; ++i) {
+            uint8_t b = packed[r * (K / 2) + i];
+            int lo = b & 0xF, hi = b >> 4;
+            codes[r * K + 2 * i] = (int8_t)(lo >= 8 ? lo - 16 : lo);
+            codes[r * K + 2 * i + 1] = (int8_t)(hi >= 8 ? hi - 16 : hi);
+        }
+}
+
+/*
+ * Integer GEMM: only the inner dimension is summed, so the per-token and per-out-channel scales
+ * stay outside the sum (Sec. 3.2, "Fine-Grained Quantization Granularity").
+ *   acc[g][m][n] = sum_{k in group g} xq[m][k] * wq[n][k]   (int32, exact)
+ * group = 0: one sum over all K (G = 1).
+ */
+void orc_gemm_i32(const int8_t *xq, const int8_t *wq, int64_t M, int N, int K, int group, int32_t *acc)
+{
+    int G = group > 0 ? K / group : 1;
+    int glen = group > 0 ? group : K;
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m)
+        for (int g = 0; g < G; ++g)
+            for (int n = 0; n < N; ++n) {
+                const int8_t *a = xq + m * K + g * glen;
+                const int8_t *b = wq + (int64_t)n * K + g * glen;
+                int32_t s = 0;
+                for (int k = 0; k < glen; ++k) s += (int32_t)a[k] * (int32_t)b[k];
+                acc[((int64_t)g * M + m) * N + n] = s;
+            }
+}
+
+/*
+ * Rescale + bias + bf16.
+ *   G == 1:  t = fl(a_scale[m] * w_scale[n]);  z = fl(float(acc) * t);  z = fl(z + bias[n])
+ *   G  > 1:  s = 0; for g ascending: s = fl(s + fl(float(acc_g) * a_scale[m][g]));
+ *            z = fl(fl(s * w_scale[n]) + bias[n])
+ * bias is bf16 bits or NULL (= 0).  Y is bf16 bits, row stride ldy.
+ */
+void orc_epilogue(const int32_t *acc, const float *a_scale, const float *w_scale, const uint16_t *bias,
+                  int64_t M, int N, int G, uint16_t *Y, int64_t ldy)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m)
+        for (int n = 0; n < N; ++n) {
+            float z;
+            if (G == 1) {
+                float t = a_scale[m] * w_scale[n];
+                z = (float)acc[m * N + n] * t;
+            } else {
+                float s = 0.0f;
+                for (int g = 0; g < G; ++g) {
+                    float p = (float)acc[((int64_t)g * M + m) * N + n] * a_scale[m * G + g];
+                    s = s + p;
+                }
+                z = s * w_scale[n];
+            }
+            if (bias) z = z + orc_bf16_to_f32(bias[n]);
+            Y[m * ldy + n] = orc_f32_to_bf16(z);
+        }
+}
+
+/*
+ * Post-local smoothing factors (Eq. "smooth_factor", alpha = 0.5 in the paper):
+ *   c_k = clip( max_m |(X H)_{m,k}|^alpha / max_n |(W H)_{n,k}|^(1-alpha), lo, hi ),
+ * both maxima taken in the rotated space with the normalized Hadamard, in fp64 from the bf16
+ * inputs; the signs v do not change absolute values.  0/0 -> 1.  Result rounded to fp32.
+ */
+void orc_smooth_factors(const uint16_t *Xcal, int64_t Mc, const uint16_t *W, int N, int K, double alpha,
+                        double lo, double hi, float *c)
+{
+    double *ax = (double *)calloc((size_t)K, sizeof(double));
+    double *aw = (double *)calloc((size_t)K, sizeof(double));
+    double *u = (double *)malloc(sizeof(double) * (size_t)K);
+    double nrm = 1.0 / sqrt((double)K);
+    for (int64_t m = 0; m < Mc; ++m) {
+        for (int k = 0; k < K; ++k) u[k] = (double)orc_bf16_to_f32(Xcal[m * K + k]);
+        orc_fwht_f64(u, K);
+        for (int k = 0; k < K; ++k) {
+            double a = fabs(u[k]) * nrm;
+            if (a > ax[k]) ax[k] = a;
+        }
+    }
+    for (int n = 0; n < N; ++n) {
+        for (int k = 0; k < K; ++k) u[k] = (double)orc_bf16_to_f32(W[(int64_t)n * K + k]);
+        orc_fwht_f64(u, K);
+        for (int k = 0; k < K; ++k) {
+            double a = fabs(u[k]) * nrm;
+            if (a > aw[k]) aw[k] = a;
+        }
+    }
+    for (int k = 0; k < K; ++k) {
+        double v;
+        if (ax[k] == 0.0 && aw[k] == 0.0) v = 1.0;
+        else v = pow(ax[k], alpha) / pow(aw[k], 1.0 - alpha);
+        if (!(v >= lo)) v = lo;
+        if (v > hi) v = hi;
+        c[k] = (float)v;
+    }
+    free(ax);
+    free(aw);
+    free(u);
+}
+
+/* fp64 rotated-and-scaled rows: out[m][k] = (x_m H_K)[k] * mul[k]  (for the invariance pins). */
+void orc_rotate_f64(const uint16_t *X, int64_t ldx, int64_t M, int K, const double *mul, double *out)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m) {
+        double *u = out + m * K;
+        for (int k = 0; k < K; ++k) u[k] = (double)orc_bf16_to_f32(X[m * ldx + k]);
+        orc_fwht_f64(u, K);
+        for (int k = 0; k < K; ++k) u[k] *= mul[k];
+    }
+}
+
+/* The unquantized layer Y = X W^T + b in fp64 from the bf16 inputs (information-only reference). */
+void orc_linear_f64(const uint16_t *X, const uint16_t *W, const uint16_t *bias, int64_t M, int N, int K,
+                    double *Y)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m)
+        for (int n = 0; n < N; ++n) {
+            double s = 0.0;
+            for (int k = 0; k < K; ++k)
+                s += (double)orc_bf16_to_f32(X[m * K + k]) * (double)orc_bf16_to_f32(W[(int64_t)n * K + k]);
+            if (bias) s += (double)orc_bf16_to_f32(bias[n]);
+            Y[m * N + n] = s;
+        }
+}

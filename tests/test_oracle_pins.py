@@ -1,0 +1,349 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, checked without the CUDA path.
+
+Each test names the passage it leans on.  Where a check recomputes something, it does so by a
+different route than the oracle (dense +-1 matrices from the closed form, numpy int64/fp64 matmul,
+pure-Python loops), never by retyping the oracle's own loop.
+"""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+import workload
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def f32_to_bf16_bits(a):
+    """Exact only for values already representable in bf16 (asserted)."""
+    a = np.asarray(a, np.float32)
+    u = a.view(np.uint32)
+    assert np.all((u & 0xFFFF) == 0), "test input is not bf16-representable"
+    return (u >> 16).astype(np.uint16)
+
+
+def sylvester(K):
+    """Closed form of the Kronecker recursion: H[i][j] = (-1)^popcount(i & j)."""
+    i = np.arange(K, dtype=np.int64)
+    x = i[:, None] & i[None, :]
+    pc = np.zeros_like(x)
+    while np.any(x):
+        pc += x & 1
+        x >>= 1
+    return (1 - 2 * (pc & 1)).astype(np.int64)
+
+
+def load_table(name):
+    rows = []
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                rows.append([float(t) for t in line.split()])
+    return np.array(rows)
+
+
+# ------------------------------------------------------------------ Hadamard (Sec. 3.2, Pre-Global-Rotation)
+def test_h8_matches_handwritten_kronecker_recursion():
+    H8 = load_table("sylvester_h8.txt")
+    assert H8.shape == (8, 8)
+    got = oracle.fwht_f32(np.eye(8, dtype=np.float32))  # row j = e_j H
+    assert np.array_equal(got, H8.astype(np.float32))
+    assert np.array_equal(sylvester(8), H8.astype(np.int64))  # the closed form used below agrees too
+
+
+@pytest.mark.parametrize("K", [2, 4, 16, 64, 1024, 4096])
+def test_fwht_of_unit_vectors_is_closed_form_column(K):
+    H = sylvester(K) if K <= 1024 else None
+    for j in sorted({j for j in (0, 1, 2, 3, K // 2, K - 1, (K // 3) | 1) if j < K}):
+        e = np.zeros(K, np.float32)
+        e[j] = 1.0
+        got = oracle.fwht_f32(e)
+        if H is not None:
+            want = H[j]
+        else:
+            i = np.arange(K)
+            want = 1 - 2 * (np.array([bin(v).count("1") for v in (i & j)]) & 1)
+        assert np.array_equal(got, want.astype(np.float32)), (K, j)
+
+
+@pytest.mark.parametrize("K", [2, 8, 64])
+def test_h_ht_equals_k_identity(K):
+    H = oracle.fwht_f64(np.eye(K))
+    assert np.array_equal(H @ H.T, K * np.eye(K))
+    assert np.array_equal(H, H.T)
+
+
+@pytest.mark.parametrize("K", [16, 1024, 4096])
+def test_fwht_twice_is_k_times_identity_on_small_integers(K):
+    rng = np.random.default_rng(K)
+    x = rng.integers(-8, 9, size=(3, K)).astype(np.float32)
+    assert np.array_equal(oracle.fwht_f32(oracle.fwht_f32(x)), K * x)
+
+
+@pytest.mark.parametrize("K", [64, 1024, 4096])
+def test_fwht_equals_dense_product_on_integer_inputs(K):
+    """Integer inputs keep every fp32 partial sum exact, so any butterfly order must match x @ H."""
+    rng = np.random.default_rng(7 + K)
+    x = rng.integers(-100, 101, size=(4, K)).astype(np.int64)
+    want = x @ sylvester(K)
+    got = oracle.fwht_f32(x.astype(np.float32))
+    assert np.array_equal(got.astype(np.int64), want)
+    got64 = oracle.fwht_f64(x.astype(np.float64))
+    assert np.array_equal(got64.astype(np.int64), want)
+
+
+@pytest.mark.parametrize("K", [1024, 4096])
+def test_fwht_f32_stays_within_rounding_bound_of_f64(K):
+    spec = workload.LinearSpec("t", K, 8, workload.DIST_NORMAL, 11, 0)
+    x = workload.bf16_to_f32(spec.x_rows(0, 6)).astype(np.float64)
+    u64 = oracle.fwht_f64(x)
+    u32 = oracle.fwht_f32(x.astype(np.float32)).astype(np.float64)
+    bound = np.log2(K) * 2.0 ** -24 * np.abs(x).sum(axis=1, keepdims=True) * 1.01
+    assert np.all(np.abs(u32 - u64) <= bound)
+    assert np.any(u32 != u64)  # the fp32 path really rounds (so the bound is not vacuous)
+
+
+def test_rotation_invariance_fp64():
+    """X W^T = (X H)(W H)^T for the random Hadamard H = K^-1/2 H_K diag(v), H^T H = I."""
+    K, M, N = 1024, 9, 7
+    spec = workload.LinearSpec("t", K, N, workload.DIST_NORMAL, 3, 0)
+    X, W = spec.x_rows(0, M), spec.weight()
+    v = workload.signs_i8(3, 9, K).astype(np.float64)
+    assert set(np.unique(v)) == {-1.0, 1.0}
+    mul = v / np.sqrt(K)
+    lhs = oracle.rotate_f64(X, mul) @ oracle.rotate_f64(W, mul).T
+    rhs = workload.bf16_to_f32(X).astype(np.float64) @ workload.bf16_to_f32(W).astype(np.float64).T
+    assert np.max(np.abs(lhs - rhs)) <= 1e-12 * np.max(np.abs(rhs))
+
+
+@pytest.mark.parametrize("K", [1024, 4096])
+def test_smoothing_invariance_fp64_with_oracle_multipliers(K):
+    """X W^T = (X H diag(c)^-1)(diag(c) H^T W^T) using the multipliers the oracle really applies."""
+    M, N = 6, 5
+    spec = workload.LinearSpec("t", K, N, workload.DIST_NORMAL, 5, 0)
+    X, W = spec.x_rows(0, M), spec.weight()
+    c = workload.loguniform_f32(5, 50, K, 1e-2, 1e2)
+    v = workload.signs_i8(5, 51, K)
+    amul, wmul = oracle.multipliers(c, v)
+    assert amul.dtype == np.float32 and np.all(np.sign(amul) == v) and np.all(np.sign(wmul) == v)
+    nrm = np.float32(2.0 ** -(np.log2(K) / 2))
+    assert np.array_equal(amul, (v * nrm).astype(np.float32) / c)  # one IEEE division
+    assert np.array_equal(wmul, (v * nrm).astype(np.float32) * c)
+    lhs = oracle.rotate_f64(X, amul.astype(np.float64)) @ oracle.rotate_f64(W, wmul.astype(np.float64)).T
+    rhs = workload.bf16_to_f32(X).astype(np.float64) @ workload.bf16_to_f32(W).astype(np.float64).T
+    # amul*wmul = (1/K)(1 + O(2^-23)) per channel, so the identity holds to fp32 rounding of c
+    assert np.max(np.abs(lhs - rhs)) <= 4e-7 * np.sum(np.abs(workload.bf16_to_f32(X[:, None, :]).astype(np.float64)
+                                                            * workload.bf16_to_f32(W[None]).astype(np.float64)), axis=2).max()
+
+
+def test_default_signs_are_plus_one():
+    c = workload.loguniform_f32(1, 2, 1024, 0.1, 10)
+    a0, w0 = oracle.multipliers(c, None)
+    a1, w1 = oracle.multipliers(c, np.ones(1024, np.int8))
+    assert np.array_equal(a0, a1) and np.array_equal(w0, w1) and np.all(a0 > 0)
+
+
+# ------------------------------------------------------------------ quantizer (Eq. "quantization", N = 4)
+def _rotated_y(X, mul):
+    u = oracle.fwht_f32(workload.bf16_to_f32(X))
+    return u * mul.astype(np.float32)[None, :]
+
+
+@pytest.mark.parametrize("K,group", [(1024, 0), (4096, 0), (1024, 128), (4096, 128)])
+def test_quantizer_error_bound_and_range(K, group):
+    spec = workload.LinearSpec("t", K, 8, workload.DIST_NORMAL, 21, 0)
+    X = spec.x_rows(0, 12)  # includes the five x100 special rows
+    c = workload.loguniform_f32(21, 5, K, 0.05, 20)
+    amul, _ = oracle.multipliers(c, workload.signs_i8(21, 6, K))
+    codes, scales = oracle.rotate_smooth_quantize(X, amul, group)
+    y = _rotated_y(X, amul).astype(np.float64)
+    G = K // group if group else 1
+    yg = y.reshape(12, G, -1)
+    qg = codes.reshape(12, G, -1).astype(np.float64)
+    sg = scales.reshape(12, G, 1).astype(np.float64)
+    assert np.all(np.abs(yg - sg * qg) <= sg / 2 * (1 + 2.0 ** -22))      # |x - Delta q| <= Delta / 2
+    amax = np.abs(yg).max(axis=2, keepdims=True)
+    assert np.array_equal(sg.astype(np.float32), (amax.astype(np.float32) / np.float32(7)))  # Delta = max|x| / 7
+    assert codes.min() >= -7 and codes.max() <= 7                           # -8 is never produced
+    hit = np.abs(yg) == amax
+    assert np.all(np.abs(qg[hit]) == 7)                                     # the absmax element maps to +-7
+    assert np.all(np.sign(qg[hit]) == np.sign(yg[hit]))
+
+
+def test_round_half_to_even_on_handbuilt_ties():
+    tab = load_table("round_ties.txt")
+    y, want = tab[:, 0], tab[:, 1].astype(np.int8)
+    K = len(y)
+    assert K == 16
+    x = (sylvester(K) @ y) / K                     # x H_K = y exactly (all partial sums are dyadic and small)
+    X = f32_to_bf16_bits(x.astype(np.float32))[None, :]
+    assert np.array_equal(oracle.fwht_f32(workload.bf16_to_f32(X))[0], y.astype(np.float32))
+    codes, scales = oracle.rotate_smooth_quantize(X, np.ones(K, np.float32), 0)
+    assert scales[0] == np.float32(1.0)
+    assert np.array_equal(codes[0], want)
+
+
+def test_zero_row_gives_zero_codes_and_floor_scale():
+    X = np.zeros((2, 1024), np.uint16)
+    X[1, 5] = 0x3F80
+    codes, scales = oracle.rotate_smooth_quantize(X, np.full(1024, 2.0 ** -5, np.float32), 0)
+    assert not codes[0].any() and scales[0] == np.float32(1e-8) / np.float32(7)
+    # a single 1.0 spreads to +-2^-5 everywhere: every code is +-7 and follows the Sylvester column
+    assert np.array_equal(codes[1], 7 * sylvester(1024)[5])
+    assert scales[1] == np.float32(2.0 ** -5) / np.float32(7)
+
+
+def test_group_equal_to_k_reduces_to_per_token():
+    K = 1024
+    spec = workload.LinearSpec("t", K, 8, workload.DIST_NORMAL, 2, 0)
+    X = spec.x_rows(0, 7)
+    amul, _ = oracle.multipliers(workload.loguniform_f32(2, 5, K, 0.1, 10))
+    c0, s0 = oracle.rotate_smooth_quantize(X, amul, 0)
+    c1, s1 = oracle.rotate_smooth_quantize(X, amul, K)
+    assert np.array_equal(c0, c1) and np.array_equal(s0, s1.reshape(-1))
+    acc0 = oracle.gemm_i32(c0, c0[:5], 0)
+    acc1 = oracle.gemm_i32(c0, c0[:5], K)
+    assert np.array_equal(acc0, acc1[0])
+
+
+def test_pack_layout_low_nibble_is_even_index():
+    codes = np.array([[1, -1, 7, -8, 0, 3, -7, 5]], np.int8)
+    packed = oracle.pack_int4(codes)
+    assert packed.tolist() == [[0xF1, 0x87, 0x30, 0x59]]
+    assert np.array_equal(oracle.unpack_int4(packed), codes)
+    rng = np.random.default_rng(0)
+    r = rng.integers(-8, 8, size=(5, 64)).astype(np.int8)
+    assert np.array_equal(oracle.unpack_int4(oracle.pack_int4(r)), r)
+
+
+# ------------------------------------------------------------------ integer GEMM (Sec. 3.2, granularity)
+def test_gemm_bruteforce_tiny():
+    rng = np.random.default_rng(1)
+    M, N, K = 3, 4, 8
+    a = rng.integers(-8, 8, size=(M, K)).astype(np.int8)
+    b = rng.integers(-8, 8, size=(N, K)).astype(np.int8)
+    want = [[sum(int(a[m, k]) * int(b[n, k]) for k in range(K)) for n in range(N)] for m in range(M)]
+    assert oracle.gemm_i32(a, b).tolist() == want
+    assert oracle.gemm_i32(a, b).shape == (M, N)  # [tokens, out channels], not transposed
+
+
+@pytest.mark.parametrize("K,group", [(1024, 0), (4096, 0), (1024, 128), (4096, 128)])
+def test_gemm_matches_int64_matmul_and_bound(K, group):
+    rng = np.random.default_rng(K + group)
+    M, N = 11, 13
+    a = rng.integers(-7, 8, size=(M, K)).astype(np.int8)
+    b = rng.integers(-7, 8, size=(N, K)).astype(np.int8)
+    a[0], b[0] = 7, -7                                    # extreme row: acc = -49 K
+    acc = oracle.gemm_i32(a, b, group)
+    if group:
+        G = K // group
+        want = np.einsum("mgk,ngk->gmn", a.reshape(M, G, -1).astype(np.int64), b.reshape(N, G, -1).astype(np.int64))
+        assert acc.shape == (G, M, N) and np.array_equal(acc, want)
+        assert np.array_equal(acc.sum(axis=0), a.astype(np.int64) @ b.astype(np.int64).T)
+    else:
+        assert np.array_equal(acc, a.astype(np.int64) @ b.astype(np.int64).T)
+        assert acc[0, 0] == -49 * K
+    assert np.abs(acc).max() <= 49 * K
+
+
+# ------------------------------------------------------------------ epilogue
+def bf16_neighbors_ok(got_bits, want_f64):
+    """got is the bf16 nearest to want_f64, or one of its two neighbours."""
+    got = oracle.bf16_to_f32(got_bits).astype(np.float64)
+    ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(want_f64), 1e-300))) - 7)
+    return np.abs(got - want_f64) <= ulp * 1.0000001
+
+
+def test_epilogue_against_fp64_recomputation():
+    rng = np.random.default_rng(4)
+    M, N = 17, 19
+    acc = rng.integers(-200000, 200001, size=(M, N)).astype(np.int32)
+    a_s = rng.uniform(0.01, 3.0, M).astype(np.float32)
+    w_s = rng.uniform(1e-4, 1e-2, N).astype(np.float32)
+    bias = workload.normal_bf16(4, 1, 1, N, 0.01).reshape(N)
+    Y = oracle.epilogue(acc, a_s, w_s, bias)
+    want = acc.astype(np.float64) * a_s[:, None].astype(np.float64) * w_s[None, :].astype(np.float64) \
+        + oracle.bf16_to_f32(bias).astype(np.float64)[None, :]
+    assert np.all(bf16_neighbors_ok(Y, want))
+    Y0 = oracle.epilogue(acc, a_s, w_s, None)
+    assert np.all(bf16_neighbors_ok(Y0, want - oracle.bf16_to_f32(bias).astype(np.float64)[None, :]))
+
+
+def test_epilogue_exact_special_cases():
+    N = 8
+    bias = workload.normal_bf16(9, 1, 1, N, 0.01).reshape(N)
+    zero = np.zeros((2, N), np.int32)
+    one = np.ones(2, np.float32)
+    assert np.array_equal(oracle.epilogue(zero, one, np.ones(N, np.float32), bias), np.tile(bias, (2, 1)))  # acc = 0 -> bias
+    acc = np.arange(-8, 8, dtype=np.int32).reshape(2, N) * 3
+    Y = oracle.epilogue(acc, 2 * one, np.full(N, 0.5, np.float32), None)       # scales cancel -> small integers, exact
+    assert np.array_equal(oracle.bf16_to_f32(Y), acc.astype(np.float32))
+    # per-token scale goes with the row, per-channel scale with the column
+    a_s = np.array([1.0, 4.0], np.float32)
+    w_s = np.array([1, 2, 1, 1, 1, 1, 1, 8], np.float32)
+    Y = oracle.bf16_to_f32(oracle.epilogue(np.ones((2, N), np.int32), a_s, w_s, None))
+    assert np.array_equal(Y, a_s[:, None] * w_s[None, :])
+
+
+def test_epilogue_groupwise_against_fp64():
+    rng = np.random.default_rng(6)
+    G, M, N = 8, 5, 6
+    acc = rng.integers(-6000, 6001, size=(G, M, N)).astype(np.int32)
+    a_s = rng.uniform(0.01, 3.0, (M, G)).astype(np.float32)
+    w_s = rng.uniform(1e-4, 1e-2, N).astype(np.float32)
+    bias = workload.normal_bf16(6, 1, 1, N, 0.01).reshape(N)
+    Y = oracle.bf16_to_f32(oracle.epilogue(acc, a_s, w_s, bias)).astype(np.float64)
+    terms = acc.astype(np.float64) * a_s.T[:, :, None].astype(np.float64)
+    want = terms.sum(axis=0) * w_s[None, :] + oracle.bf16_to_f32(bias)[None, :]
+    slack = 2.0 ** -7 * np.abs(want) + G * 2.0 ** -23 * np.abs(terms).sum(axis=0) * w_s[None, :]
+    assert np.all(np.abs(Y - want) <= slack)
+
+
+# ------------------------------------------------------------------ smoothing factors (Eq. "smooth_factor")
+def test_smooth_factors_against_dense_closed_form():
+    K, Mc, N = 64, 10, 12
+    X = workload.activations(8, 0, 0, Mc, K, workload.DIST_NORMAL, workload.outlier_gains(8, 1, K, 2), frame_rows=0)
+    W = workload.normal_bf16(8, 2, N, K, 0.02)
+    H = sylvester(K).astype(np.float64) / np.sqrt(K)
+    ax = np.abs(workload.bf16_to_f32(X).astype(np.float64) @ H).max(axis=0)
+    aw = np.abs(workload.bf16_to_f32(W).astype(np.float64) @ H).max(axis=0)
+    for alpha in (0.3, 0.5, 0.7):
+        want = np.clip(ax ** alpha / aw ** (1 - alpha), 1e-2, 1e2)
+        got = oracle.smooth_factors(X, W, alpha)
+        assert np.allclose(got, want, rtol=1e-6, atol=0)
+    # clipping and the 0/0 convention
+    Xz = np.zeros((3, K), np.uint16)
+    Wz = np.zeros((3, K), np.uint16)
+    assert np.array_equal(oracle.smooth_factors(Xz, Wz), np.ones(K, np.float32))
+    assert np.array_equal(oracle.smooth_factors(Xz, W), np.full(K, 1e-2, np.float32))
+    assert np.array_equal(oracle.smooth_factors(X, Wz), np.full(K, 1e2, np.float32))
+
+
+# ------------------------------------------------------------------ whole layer
+def test_linear_f64_is_x_wt_plus_b():
+    spec = workload.LinearSpec("t", 64, 5, workload.DIST_NORMAL, 1, 0)
+    X, W, b = spec.x_rows(0, 4), spec.weight(), spec.bias()
+    want = workload.bf16_to_f32(X).astype(np.float64) @ workload.bf16_to_f32(W).astype(np.float64).T \
+        + workload.bf16_to_f32(b).astype(np.float64)
+    assert np.allclose(oracle.linear_f64(X, W, b), want, rtol=1e-13, atol=1e-15)
+
+
+@pytest.mark.parametrize("group", [0, 128])
+def test_quantized_layer_approximates_the_fp_layer(group):
+    """Information-level sanity (parity unpinned by the paper): the W4A4 output tracks X W^T + b."""
+    spec = workload.LinearSpec("proj", 1024, 256, workload.DIST_NORMAL, 0, 1)
+    X, W, b = spec.x_rows(0, 64), spec.weight(), spec.bias()
+    c = oracle.smooth_factors(spec.x_calib(256), W)
+    prep = oracle.prepare_weights(W, c, None)
+    out = oracle.w4a4_linear(X, prep, b, group)
+    ref = oracle.linear_f64(X, W, b)
+    y = oracle.bf16_to_f32(out["y"]).astype(np.float64)
+    rel = np.linalg.norm(y - ref) / np.linalg.norm(ref)
+    assert rel < 0.25, rel
+    # dequantized integer sums reproduce the same numbers (scales factor out of the sum)
+    if not group:
+        deq = out["acc"].astype(np.float64) * out["a_scale"][:, None] * prep["w_scale"][None, :] \
+            + oracle.bf16_to_f32(b)[None, :]
+        assert np.all(bf16_neighbors_ok(out["y"], deq))
