@@ -1,0 +1,332 @@
+#!/usr/bin/env python
+"""Benchmark of the W4A4 linear path (QuantVGGT Dual-Smoothed Fine-Grained Quantization) on B200.
+
+One "step" = one pass of the whole online hot path over one batch: for each of the four linears of
+one aggregator block (qkv 1024->3072, proj 1024->1024, fc1 1024->4096, fc2 4096->1024) at 8 frames
+(M = 10992 tokens): rotate-smooth-quantize, then W4A4 GEMM + rescale + bias + bf16.  Weight
+preparation is offline and untimed.  Prints ONE JSON line (see the design doc for the fields).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workload  # noqa: E402
+
+FRAMES = 8
+NOMINAL_INT8_OVER_BF16 = 2.0      # dense tensor peaks: int8 4.5 POPS vs bf16 2.25 PFLOP/s (nominal ratio)
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS if k in p} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS, source="fallback")
+
+
+def layer_ops(M, spec):
+    return 2.0 * M * spec.N * spec.K
+
+
+def gemm_bytes(M, spec):
+    return M * spec.K / 2 + 4 * M + spec.N * spec.K / 2 + 6 * spec.N + 2.0 * M * spec.N
+
+
+def rsq_bytes(M, K):
+    return M * (2 * K + K / 2 + 4)
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([t.strip() for t in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], None, set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                smax = float(r[1])
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            except Exception:
+                pass
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": smax, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------ oracle arm
+def run_reference(args, rank, world):
+    """The CPU oracle, as it stands, on a bounded sample of the same workload (rank 0 only)."""
+    if rank != 0:
+        return
+    import oracle
+    specs = workload.block_specs(0, 0)
+    rows = args.ref_rows
+    prepared = []
+    for s in specs:
+        W = s.weight()
+        c = oracle.smooth_factors(s.x_calib(256), W)
+        prepared.append((s, oracle.prepare_weights(W, c, None), s.bias(), s.x_rows(0, rows)))
+    ops = sum(layer_ops(rows, s) for s in specs)
+
+    def step():
+        for s, prep, b, X in prepared:
+            oracle.w4a4_linear(X, prep, b, 0)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    tops = ops / dt / 1e12
+    sample = f"first {rows} token rows of the 8-frame batch through all four linears of one block"
+    print(json.dumps({
+        "impl": "reference", "metric": "w4a4_linear_tops", "value": tops, "unit": "TOPS", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int4 x int4 -> int32 (fp32 rotation and scales)",
+        "data": "synthetic", "tokens_per_s": rows / dt,
+        "config": {"workload": "aggregator block, 4 linears (qkv/proj/fc1/fc2), 8 frames M=10992 -- bounded sample", "sample": sample},
+        "cpu_baseline": {"value": tops, "unit": "TOPS", "cores": oracle.threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": tops, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def cpu_baseline(rows=workload.TOKENS_PER_FRAME):
+    import oracle
+    specs = workload.block_specs(0, 0)
+    ops, dt, timings = 0.0, 0.0, {}
+    for s in specs:
+        W = s.weight()
+        prep = oracle.prepare_weights(W, oracle.smooth_factors(s.x_calib(256), W), None)
+        X, b = s.x_rows(0, rows), s.bias()
+        t0 = time.perf_counter()
+        oracle.w4a4_linear(X, prep, b, 0, timings)
+        dt += time.perf_counter() - t0
+        ops += layer_ops(rows, s)
+    return {"value": ops / dt / 1e12, "unit": "TOPS", "cores": oracle.threads(), "kind": "oracle",
+            "sample": f"first {rows} token rows (one frame) of the batch through all four linears, one pass, {dt:.1f} s",
+            "tokens_per_s": rows / dt, "seconds": {k: round(v, 3) for k, v in timings.items()}}
+
+
+# ------------------------------------------------------------------------------------------------ CUDA arm
+def run_ours(args, rank, world, local_rank):
+    import torch
+    import paper_2509_21302_b200 as q
+
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    q.build()
+    peaks = load_peaks()
+    M = FRAMES * workload.TOKENS_PER_FRAME
+    specs = workload.block_specs(0, 0)
+    row0 = rank * M                                     # weak scaling: every rank gets its own 8 frames
+
+    def dev_bf16(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+    layers = []
+    NBUF = 2                                            # input/output buffer sets, alternated per step
+    for s in specs:
+        W = dev_bf16(s.weight())
+        c = q.calibrate_smooth(dev_bf16(s.x_calib()), W)
+        h = q.prepare_weights(W, dev_bf16(s.bias()), c, None)
+        host_x = torch.from_numpy(s.x_rows(row0, M).view(np.int16)).pin_memory()
+        xs = [host_x.cuda().view(torch.bfloat16) for _ in range(NBUF)]
+        layers.append(dict(spec=s, h=h, host_x=host_x, x=xs,
+                           xq=[torch.empty((M, s.K // 2), dtype=torch.uint8, device="cuda") for _ in range(NBUF)],
+                           a=[torch.empty((M,), dtype=torch.float32, device="cuda") for _ in range(NBUF)],
+                           y=[torch.empty((M, s.N), dtype=torch.bfloat16, device="cuda") for _ in range(NBUF)],
+                           host_y=torch.empty((M, s.N), dtype=torch.bfloat16).pin_memory()))
+    torch.cuda.synchronize()
+
+    def step(i, ev=None):
+        b = i % NBUF
+        for li, L in enumerate(layers):
+            if ev is not None:
+                ev[li][0].record()
+            q.rotate_smooth_quantize(L["h"], L["x"][b], 0, L["xq"][b], L["a"][b])
+            if ev is not None:
+                ev[li][1].record()
+            q.w4a4_linear(L["h"], L["xq"][b], L["a"][b], 0, L["y"][b])
+            if ev is not None:
+                ev[li][2].record()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+    # timed region: K steps, CUDA events on the launching stream; per-kernel events ride along
+    kev = [[[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in layers] for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    t_start, t_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_start.record()
+    for i in range(args.steps):
+        step(i, kev[i])
+    t_stop.record()
+    barrier()
+    clocks = sampler.stop()
+    total_ms = t_start.elapsed_time(t_stop)
+    if dist is not None:
+        t = torch.tensor([total_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    for L in layers:
+        assert L["h"].device_status() == 0, "a device-side wait expired"
+
+    rsq_ms = np.array([[kev[i][li][0].elapsed_time(kev[i][li][1]) for li in range(len(layers))] for i in range(args.steps)])
+    gemm_ms = np.array([[kev[i][li][1].elapsed_time(kev[i][li][2]) for li in range(len(layers))] for i in range(args.steps)])
+
+    # end-to-end: host buffers in, host buffers out, copies inside the timed region
+    def e2e_step(i):
+        b = i % NBUF
+        for L in layers:
+            L["x"][b].view(torch.int16).copy_(L["host_x"], non_blocking=True)
+            q.rotate_smooth_quantize(L["h"], L["x"][b], 0, L["xq"][b], L["a"][b])
+            q.w4a4_linear(L["h"], L["xq"][b], L["a"][b], 0, L["y"][b])
+            L["host_y"].copy_(L["y"][b], non_blocking=True)
+
+    e2e_steps = max(2, min(args.steps, 5))
+    e2e_step(0)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    ops_step = sum(layer_ops(M, s) for s in specs)
+    ms_per_step = total_ms / args.steps
+    tops = world * ops_step / (ms_per_step * 1e-3) / 1e12
+    gemm_ops = sum(layer_ops(M, s) for s in specs)
+    gemm_avg_ms = gemm_ms.mean(axis=0)                    # per layer
+    gemm_tops = gemm_ops / (gemm_avg_ms.sum() * 1e-3) / 1e12
+    int8_peak = peaks["bf16_tflops"] * NOMINAL_INT8_OVER_BF16
+    int8_peak_sus = peaks["bf16_tflops_sustained"] * NOMINAL_INT8_OVER_BF16
+    rsq_avg_ms = rsq_ms.mean(axis=0)
+    rsq_b = sum(rsq_bytes(M, s.K) for s in specs)
+    rsq_gbs = rsq_b / (rsq_avg_ms.sum() * 1e-3) / 1e9
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tpath):
+        with open(tpath) as f:
+            traffic = json.load(f).get("gemm_bytes_per_launch_avg")
+    per_layer = {}
+    for li, s in enumerate(specs):
+        t_g, t_r = gemm_avg_ms[li] * 1e-3, rsq_avg_ms[li] * 1e-3
+        bound = max(layer_ops(M, s) / (int8_peak * 1e12), gemm_bytes(M, s) / (peaks["hbm_gbs"] * 1e9))
+        per_layer[s.name] = {"gemm_us": round(t_g * 1e6, 2), "gemm_tops": round(layer_ops(M, s) / t_g / 1e12, 1),
+                             "gemm_roofline_frac": round(bound / t_g, 4),
+                             "rsq_us": round(t_r * 1e6, 2), "rsq_gbs": round(rsq_bytes(M, s.K) / t_r / 1e9, 1),
+                             "rsq_hbm_frac": round(rsq_bytes(M, s.K) / t_r / 1e9 / peaks["hbm_gbs"], 4)}
+    out = {
+        "metric": "w4a4_linear_tops", "value": tops, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int4 x int4 -> int32 (fp32 rotation and scales)", "data": "synthetic",
+        "tokens_per_s": world * M / (ms_per_step * 1e-3),
+        "config": {"workload": "aggregator block, 4 linears (qkv/proj/fc1/fc2), 8 frames M=10992 per GPU (BASELINE configs[1])",
+                   "l2": f"step working set ~400 MB > 126 MB L2; {NBUF} buffer sets alternated per step",
+                   "timed": "rotate-smooth-quantize + W4A4 GEMM/epilogue per linear; weight prep offline"},
+        "clocks": clocks,
+        "gpu_launches": int(2 * len(layers) * args.steps),
+        "e2e": {"value": world * ops_step / (e2e_ms * 1e-3) / 1e12, "unit": "TOPS", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": int(sum(M * s.K * 2 for s in specs)),
+                "d2h_bytes_per_step": int(sum(M * s.N * 2 for s in specs))},
+        "roofline": {"kernel": "gemm_w4a4_kernel (4 launches per step)", "bound": "tensor", "achieved": gemm_tops,
+                     "peak": int8_peak, "unit": "TOP/s", "frac": gemm_tops / int8_peak,
+                     "peak_note": f"int8 dense = {NOMINAL_INT8_OVER_BF16:g} x bf16 burst, of {peaks['source']}",
+                     "frac_of_sustained": gemm_tops / int8_peak_sus, "traffic": traffic},
+        "roofline_rsq": {"kernel": "rsq_kernel (4 launches per step)", "bound": "hbm", "achieved": rsq_gbs,
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": rsq_gbs / peaks["hbm_gbs"],
+                         "peak_note": f"of {peaks['source']}", "traffic": None},
+        "per_layer": per_layer,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline()
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--ref-rows", type=int, default=512, help="token rows per step of the oracle arm")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

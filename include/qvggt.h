@@ -1,0 +1,136 @@
+/*
+ * qvggt -- W4A4 linear layer of Dual-Smoothed Fine-Grained Quantization (QuantVGGT, Sec. 3.2)
+ * for NVIDIA B200 (sm_100a).  C ABI: plain pointers and sizes, no C++ or framework types.
+ *
+ * The layer computes an approximation of  Y = X W^T + b  (X: [M tokens, K], W: [N, K]) as
+ *
+ *   Y[m][n] = a_scale[m] * w_scale[n] * sum_k Xq[m][k] * Wq[n][k] + b[n]
+ *
+ * where, with the random Hadamard rotation H = K^{-1/2} H_K diag(v) ("Pre-Global-Rotation") and
+ * the per-rotated-channel smoothing factors c ("Post-Local-Smooth", Eq. "smooth_factor"),
+ *
+ *   Xq, a_scale = quant4_per_token  ( X H diag(c)^{-1} )      (online,  qvggt_rotate_smooth_quantize)
+ *   Wq, w_scale = quant4_per_channel( W H diag(c)      )      (offline, qvggt_prepare_weights)
+ *
+ * and quant4 is the symmetric quantizer of Eq. "quantization" with N = 4 bits:
+ * Delta = max|x| / 7, q = clamp(round(x / Delta), -8, 7), round = half-to-even.  Because only the
+ * inner dimension is summed, both scales stay outside the integer sum ("Fine-Grained Quantization
+ * Granularity"), which runs on the int8 tensor cores with int32 accumulation.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless stated otherwise; matrices are row-major; the caller
+ *     owns every buffer except the opaque weights handle.
+ *   - bf16 buffers are passed as void*; packed int4 buffers as unsigned char*: byte i of a row holds
+ *     code 2i in bits 0-3 and code 2i+1 in bits 4-7, two's complement.
+ *   - K must be 1024 or 4096 (the rotation is a power-of-two Hadamard; other sizes: QVGGT_ERR_SHAPE).
+ *     N must be a multiple of 128.  M >= 0 (M == 0 is a no-op).
+ *   - `group` selects the activation-scale granularity: 0 = one scale per token (the paper's
+ *     setting); 128 = one scale per token per 128 consecutive rotated channels (an extension; the
+ *     integer partial sums are rescaled per group in the epilogue).
+ *   - All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream); no call synchronises the device except where stated.
+ *   - Return value: QVGGT_OK or a negative qvggt_status_t.  Arguments are validated on the host
+ *     before anything is launched; nothing throws or exits.
+ *   - Device-side waits are bounded.  If one expires the kernel records a code in the handle's
+ *     status word and returns; read it with qvggt_device_status().
+ */
+#ifndef QVGGT_H
+#define QVGGT_H
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct qvggt_weights qvggt_weights_t; /* opaque; owns Wq, w_scale, amul, bias, status word on the device */
+
+typedef enum {
+    QVGGT_OK = 0,
+    QVGGT_ERR_NULL = -1,           /* a required pointer is NULL */
+    QVGGT_ERR_SHAPE = -2,          /* K not in {1024, 4096}, N not a multiple of 128, M < 0, bad leading dimension */
+    QVGGT_ERR_ALIGN = -3,          /* a pointer or leading dimension breaks the 16-byte alignment rule */
+    QVGGT_ERR_UNSUPPORTED = -4,    /* group not in {0, 128}; device is not sm_100 */
+    QVGGT_ERR_CUDA = -5,           /* a CUDA runtime call failed (launch, allocation, copy) */
+    QVGGT_ERR_DEVICE_TIMEOUT = -6, /* a bounded device-side wait expired (see qvggt_device_status) */
+    QVGGT_ERR_NOMEM = -7           /* device allocation failed */
+} qvggt_status_t;
+
+/*
+ * Offline weight path (Sec. 3.2: fold the rotation and the smoothing factors into W, then
+ * out-channel-wise symmetric int4).  Per weight row n:
+ *   u = FWHT_K(W[n][:])   un-normalised Sylvester transform, fp32 radix-2 butterflies, strides 1,2,4,..
+ *   y[k] = u[k] * wmul[k],  wmul[k] = (v[k] K^{-1/2}) * c[k]
+ *   w_scale[n] = max_k|y| / 7,  Wq[n][k] = round(y[k] * (7 / max_k|y|))
+ * Also stores amul[k] = (v[k] K^{-1/2}) / c[k] for the activation path and a copy of the bias.
+ *   W_bf16    [N, K] bf16, 16-byte aligned
+ *   bias_bf16 [N] bf16 or NULL (no bias)
+ *   smooth_c  [K] fp32, finite and > 0
+ *   sign_v    [K] int8 of +1/-1, or NULL (all +1)
+ *   out       receives a new handle (device memory is allocated here, on the current device);
+ *             release it with qvggt_free_weights.  The handle is bound to that device.
+ * Work is enqueued on the stream; the inputs may be released once the stream has passed this call.
+ */
+int qvggt_prepare_weights(const void *W_bf16, const void *bias_bf16, const float *smooth_c,
+                          const signed char *sign_v, int N, int K, int flags, void *cuda_stream,
+                          qvggt_weights_t **out);
+
+/*
+ * Online activation path (Sec. 3.2: X H diag(c)^{-1}, then dynamic token-wise symmetric int4).
+ * Per token row m:  u = FWHT_K(X[m][:]);  y[k] = u[k] * amul[k];  per scale group:
+ *   a_scale = max|y| / 7 (max floored at 1e-8),  Xq = round(y * (7 / max|y|)).
+ *   w        handle from qvggt_prepare_weights (supplies K and amul)
+ *   X_bf16   [M, K] bf16 with row stride ldx elements (ldx >= K, ldx % 8 == 0), 16-byte aligned
+ *   group    0 or 128
+ *   Xq       [M, K/2] packed int4, 16-byte aligned
+ *   a_scale  fp32 [M] (group 0) or [M, K/128] (group 128)
+ */
+int qvggt_rotate_smooth_quantize(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M,
+                                 int group, unsigned char *Xq, float *a_scale, void *cuda_stream);
+
+/*
+ * Integer GEMM + rescale + bias + bf16 (Sec. 3.2, granularity paragraph: scales factor out of the sum).
+ *   group 0:    Y[m][n] = bf16( float(acc[m][n]) * (a_scale[m] * w_scale[n]) + bias[n] ),
+ *               acc[m][n] = sum_k Xq[m][k] Wq[n][k]   (int32, exact)
+ *   group 128:  Y[m][n] = bf16( (sum_g float(acc_g[m][n]) * a_scale[m][g]) * w_scale[n] + bias[n] ),
+ *               g ascending over the K/128 groups
+ *   Xq, a_scale as written by qvggt_rotate_smooth_quantize with the same `group`
+ *   Y_bf16      [M, N] bf16 with row stride ldy elements (ldy >= N, ldy % 8 == 0), 16-byte aligned
+ *   acc_debug   NULL, or int32 [M, N] (group 0) / [K/128, M, N] (group 128): the raw integer sums
+ */
+int qvggt_w4a4_linear(const qvggt_weights_t *w, const unsigned char *Xq, const float *a_scale, int M,
+                      int group, void *Y_bf16, long long ldy, int *acc_debug, void *cuda_stream);
+
+/* Frees the handle and its device memory (synchronises the device first).  NULL is allowed. */
+void qvggt_free_weights(qvggt_weights_t *w);
+
+/*
+ * Device pointers into the handle, for inspection (any output pointer may be NULL to skip it):
+ * Wq [N, K/2] packed int4, w_scale fp32 [N], amul fp32 [K], bias bf16 [N] (NULL if none).
+ * The memory stays owned by the handle.
+ */
+int qvggt_weights_view(const qvggt_weights_t *w, const unsigned char **Wq, const float **w_scale,
+                       const float **amul, const void **bias_bf16, int *N, int *K);
+
+/*
+ * Synchronises `cuda_stream`, then reads the handle's device status word into *code (HOST pointer):
+ * 0 = no device-side wait has expired since the handle was created; otherwise a positive code
+ * naming the wait that gave up.  Returns QVGGT_ERR_DEVICE_TIMEOUT if *code != 0.
+ */
+int qvggt_device_status(const qvggt_weights_t *w, void *cuda_stream, int *code);
+
+/*
+ * Calibration helper (Eq. "smooth_factor"): c[k] = clip( ax[k]^alpha / aw[k]^(1-alpha), lo, hi ) with
+ * ax[k] = max_m |(X_calib H)[m][k]|, aw[k] = max_n |(W H)[n][k]| in the rotated space (fp32
+ * butterflies; 0/0 -> 1).
+ *   X_calib_bf16 [Mc, K] bf16, contiguous;  W_bf16 [N, K] bf16, contiguous;  smooth_c fp32 [K] output
+ *   colmax_scratch  fp32 [2*K] device scratch supplied by the caller (overwritten)
+ */
+int qvggt_calibrate_smooth(const void *X_calib_bf16, int Mc, const void *W_bf16, int N, int K, float alpha,
+                           float lo, float hi, float *colmax_scratch, float *smooth_c, void *cuda_stream);
+
+/* Static, NUL-terminated description of a status code. */
+const char *qvggt_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QVGGT_H */

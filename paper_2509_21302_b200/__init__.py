@@ -1,0 +1,10 @@
+"""B200-native W4A4 linear path of QuantVGGT's Dual-Smoothed Fine-Grained Quantization.
+
+CUDA kernels (sm_100a) behind a C ABI (include/qvggt.h) plus this thin binding.
+"""
+from .binding import (EXPORTS, QvggtError, Weights, calibrate_smooth, lib, prepare_weights,
+                      rotate_smooth_quantize, w4a4_linear)
+from .build import build
+
+__all__ = ["EXPORTS", "QvggtError", "Weights", "calibrate_smooth", "lib", "prepare_weights",
+           "rotate_smooth_quantize", "w4a4_linear", "build"]

@@ -1,0 +1,202 @@
+"""Thin Python binding of libqvggt (ctypes): argument marshalling only.
+
+Every step of the path runs in the CUDA kernels behind the C ABI declared in include/qvggt.h;
+PyTorch is used for device memory and streams.  There is no CPU fallback: if the shared library
+is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+OK = 0
+_STATUS_NAMES = {0: "QVGGT_OK", -1: "QVGGT_ERR_NULL", -2: "QVGGT_ERR_SHAPE", -3: "QVGGT_ERR_ALIGN",
+                 -4: "QVGGT_ERR_UNSUPPORTED", -5: "QVGGT_ERR_CUDA", -6: "QVGGT_ERR_DEVICE_TIMEOUT",
+                 -7: "QVGGT_ERR_NOMEM"}
+
+EXPORTS = ("qvggt_prepare_weights", "qvggt_rotate_smooth_quantize", "qvggt_w4a4_linear", "qvggt_free_weights",
+           "qvggt_weights_view", "qvggt_device_status", "qvggt_calibrate_smooth", "qvggt_status_string")
+
+
+class QvggtError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().qvggt_status_string(status).decode()
+        super().__init__(f"{where}: {_STATUS_NAMES.get(status, status)} ({msg})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libqvggt.so (built in-tree by `build.build()`); raises if it is not there."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB
+        if not os.path.exists(path):
+            raise RuntimeError(f"{path} is missing: run __graft_entry__.build() (nvcc, sm_100a) first; "
+                               "there is no fallback path")
+        L = ctypes.CDLL(path)
+        vp, i32, i64, f32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong, ctypes.c_float
+        L.qvggt_prepare_weights.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, ctypes.POINTER(vp)]
+        L.qvggt_rotate_smooth_quantize.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp]
+        L.qvggt_w4a4_linear.argtypes = [vp, vp, vp, i32, i32, vp, i64, vp, vp]
+        L.qvggt_free_weights.argtypes = [vp]
+        L.qvggt_free_weights.restype = None
+        L.qvggt_weights_view.argtypes = [vp] + [ctypes.POINTER(vp)] * 4 + [ctypes.POINTER(i32)] * 2
+        L.qvggt_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
+        L.qvggt_calibrate_smooth.argtypes = [vp, i32, vp, i32, i32, f32, f32, f32, vp, vp, vp]
+        L.qvggt_status_string.argtypes = [i32]
+        L.qvggt_status_string.restype = ctypes.c_char_p
+        for name in EXPORTS:
+            if name not in ("qvggt_free_weights", "qvggt_status_string"):
+                getattr(L, name).restype = i32
+        _lib = L
+    return _lib
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t: torch.Tensor | None) -> int | None:
+    if t is None:
+        return None
+    assert t.is_cuda, "device tensor expected"
+    return t.data_ptr()
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise QvggtError(status, where)
+
+
+class Weights:
+    """Owner of a qvggt_weights_t handle (prepared int4 weights of one linear layer)."""
+
+    def __init__(self, handle: int, N: int, K: int):
+        self._h = handle
+        self.N, self.K = N, K
+
+    @property
+    def handle(self) -> int:
+        if not self._h:
+            raise RuntimeError("weights handle already freed")
+        return self._h
+
+    def view(self) -> dict:
+        """Copies of the handle's device arrays as torch tensors: wq [N,K/2] u8, w_scale [N], amul [K], bias [N] or None."""
+        ptrs = [ctypes.c_void_p() for _ in range(4)]
+        n, k = ctypes.c_int(), ctypes.c_int()
+        _check(lib().qvggt_weights_view(self.handle, *[ctypes.byref(p) for p in ptrs], ctypes.byref(n), ctypes.byref(k)),
+               "qvggt_weights_view")
+        N, K = n.value, k.value
+
+        def wrap(p, nbytes, dtype, shape):
+            if not p.value:
+                return None
+            return _from_device_ptr(p.value, nbytes, dtype, shape)
+
+        return dict(wq=wrap(ptrs[0], N * K // 2, torch.uint8, (N, K // 2)),
+                    w_scale=wrap(ptrs[1], 4 * N, torch.float32, (N,)),
+                    amul=wrap(ptrs[2], 4 * K, torch.float32, (K,)),
+                    bias=wrap(ptrs[3], 2 * N, torch.bfloat16, (N,)))
+
+    def device_status(self) -> int:
+        code = ctypes.c_int(0)
+        st = lib().qvggt_device_status(self.handle, _stream(), ctypes.byref(code))
+        if st not in (OK, -6):
+            raise QvggtError(st, "qvggt_device_status")
+        return code.value
+
+    def free(self) -> None:
+        if self._h:
+            lib().qvggt_free_weights(self._h)
+            self._h = 0
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+class _DeviceArray:
+    """Minimal __cuda_array_interface__ carrier so torch can wrap a raw device pointer."""
+
+    def __init__(self, ptr: int, shape, typestr: str):
+        self.__cuda_array_interface__ = {"shape": tuple(shape), "typestr": typestr, "data": (ptr, False), "version": 2}
+
+
+def _from_device_ptr(ptr: int, nbytes: int, dtype: torch.dtype, shape) -> torch.Tensor:
+    """Copy of the device array at `ptr` as a fresh torch tensor (so it outlives the handle)."""
+    typestr = {torch.uint8: "|u1", torch.float32: "<f4", torch.bfloat16: "<i2"}[dtype]
+    t = torch.as_tensor(_DeviceArray(ptr, shape, typestr), device="cuda")
+    assert t.numel() * t.element_size() == nbytes
+    t = t.clone()
+    return t.view(torch.bfloat16) if dtype == torch.bfloat16 else t
+
+
+def prepare_weights(W: torch.Tensor, bias: torch.Tensor | None, smooth_c: torch.Tensor,
+                    sign_v: torch.Tensor | None = None) -> Weights:
+    """W [N,K] bf16, bias [N] bf16 or None, smooth_c [K] fp32, sign_v [K] int8 (+1/-1) or None."""
+    assert W.dim() == 2 and W.element_size() == 2 and W.is_contiguous()
+    N, K = W.shape
+    assert smooth_c.dtype == torch.float32 and smooth_c.numel() == K and smooth_c.is_contiguous()
+    if bias is not None:
+        assert bias.element_size() == 2 and bias.numel() == N and bias.is_contiguous()
+    if sign_v is not None:
+        assert sign_v.dtype == torch.int8 and sign_v.numel() == K and sign_v.is_contiguous()
+    h = ctypes.c_void_p()
+    _check(lib().qvggt_prepare_weights(_ptr(W), _ptr(bias), _ptr(smooth_c), _ptr(sign_v), N, K, 0, _stream(),
+                                       ctypes.byref(h)), "qvggt_prepare_weights")
+    return Weights(h.value, N, K)
+
+
+def rotate_smooth_quantize(w: Weights, X: torch.Tensor, group: int = 0, Xq: torch.Tensor | None = None,
+                           a_scale: torch.Tensor | None = None):
+    """X [M,K] bf16 (row stride may exceed K) -> (Xq [M,K/2] uint8, a_scale fp32 [M] or [M,K/128])."""
+    assert X.dim() == 2 and X.element_size() == 2 and X.stride(1) == 1 and X.shape[1] == w.K
+    M = X.shape[0]
+    if Xq is None:
+        Xq = torch.empty((M, w.K // 2), dtype=torch.uint8, device=X.device)
+    if a_scale is None:
+        a_scale = torch.empty((M, w.K // 128) if group else (M,), dtype=torch.float32, device=X.device)
+    ldx = X.stride(0) if M > 1 else w.K
+    _check(lib().qvggt_rotate_smooth_quantize(w.handle, _ptr(X), ldx, M, group, _ptr(Xq), _ptr(a_scale), _stream()),
+           "qvggt_rotate_smooth_quantize")
+    return Xq, a_scale
+
+
+def w4a4_linear(w: Weights, Xq: torch.Tensor, a_scale: torch.Tensor, group: int = 0, Y: torch.Tensor | None = None,
+                acc_debug: torch.Tensor | None = None) -> torch.Tensor:
+    """-> Y [M,N] bf16.  acc_debug: optional int32 [M,N] (group 0) or [K/128,M,N] receiving the integer sums."""
+    M = Xq.shape[0]
+    assert Xq.dtype == torch.uint8 and Xq.is_contiguous() and Xq.shape[1] == w.K // 2
+    assert a_scale.dtype == torch.float32 and a_scale.is_contiguous()
+    if Y is None:
+        Y = torch.empty((M, w.N), dtype=torch.bfloat16, device=Xq.device)
+    assert Y.element_size() == 2 and Y.stride(1) == 1 and Y.shape == (M, w.N)
+    ldy = Y.stride(0) if M > 1 else w.N
+    if acc_debug is not None:
+        assert acc_debug.dtype == torch.int32 and acc_debug.is_contiguous()
+    _check(lib().qvggt_w4a4_linear(w.handle, _ptr(Xq), _ptr(a_scale), M, group, _ptr(Y), ldy, _ptr(acc_debug), _stream()),
+           "qvggt_w4a4_linear")
+    return Y
+
+
+def calibrate_smooth(X_calib: torch.Tensor, W: torch.Tensor, alpha: float = 0.5, lo: float = 1e-2,
+                     hi: float = 1e2) -> torch.Tensor:
+    """Smoothing factors c [K] fp32 from calibration activations [Mc,K] bf16 and weights [N,K] bf16."""
+    assert X_calib.is_contiguous() and W.is_contiguous() and X_calib.element_size() == 2 and W.element_size() == 2
+    Mc, K = X_calib.shape
+    N = W.shape[0]
+    scratch = torch.empty(2 * K, dtype=torch.float32, device=W.device)
+    c = torch.empty(K, dtype=torch.float32, device=W.device)
+    _check(lib().qvggt_calibrate_smooth(_ptr(X_calib), Mc, _ptr(W), N, K, alpha, lo, hi, _ptr(scratch), _ptr(c), _stream()),
+           "qvggt_calibrate_smooth")
+    return c

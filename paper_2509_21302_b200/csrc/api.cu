@@ -1,0 +1,176 @@
+// C-ABI entry points of libqvggt: argument validation, handle management, kernel launches.
+#include <new>
+
+#include "qvggt_internal.cuh"
+
+namespace {
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool valid_k(int K) { return K == 1024 || K == 4096; }
+
+int device_is_sm100()
+{
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return 0;
+    return major == 10;
+}
+
+void release(qvggt_weights *w)
+{
+    if (!w) return;
+    cudaFree(w->Wq);
+    cudaFree(w->w_scale);
+    cudaFree(w->amul);
+    cudaFree(w->bias);
+    cudaFree(w->status);
+    delete w;
+}
+
+}  // namespace
+
+extern "C" {
+
+int qvggt_prepare_weights(const void *W_bf16, const void *bias_bf16, const float *smooth_c, const signed char *sign_v,
+                          int N, int K, int flags, void *cuda_stream, qvggt_weights_t **out)
+{
+    (void)flags;
+    if (!out) return QVGGT_ERR_NULL;
+    *out = nullptr;
+    if (!W_bf16 || !smooth_c) return QVGGT_ERR_NULL;
+    if (!valid_k(K) || N <= 0 || N % 128 != 0) return QVGGT_ERR_SHAPE;
+    if (!aligned16(W_bf16)) return QVGGT_ERR_ALIGN;
+    if (!device_is_sm100()) return QVGGT_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+
+    qvggt_weights *w = new (std::nothrow) qvggt_weights();
+    if (!w) return QVGGT_ERR_NOMEM;
+    w->N = N;
+    w->K = K;
+    w->Wq = nullptr; w->w_scale = nullptr; w->amul = nullptr; w->bias = nullptr; w->status = nullptr;
+    cudaGetDevice(&w->device);
+    float *wmul = nullptr;
+    bool ok = cudaMalloc(&w->Wq, (size_t)N * K / 2) == cudaSuccess &&
+              cudaMalloc(&w->w_scale, sizeof(float) * N) == cudaSuccess &&
+              cudaMalloc(&w->amul, sizeof(float) * K) == cudaSuccess &&
+              cudaMalloc(&w->status, sizeof(int)) == cudaSuccess &&
+              cudaMallocAsync(&wmul, sizeof(float) * K, st) == cudaSuccess &&
+              (!bias_bf16 || cudaMalloc(&w->bias, sizeof(uint16_t) * N) == cudaSuccess);
+    if (!ok) {
+        cudaGetLastError();
+        if (wmul) cudaFreeAsync(wmul, st);
+        release(w);
+        return QVGGT_ERR_NOMEM;
+    }
+    cudaError_t e = cudaMemsetAsync(w->status, 0, sizeof(int), st);
+    if (e == cudaSuccess && bias_bf16)
+        e = cudaMemcpyAsync(w->bias, bias_bf16, sizeof(uint16_t) * N, cudaMemcpyDeviceToDevice, st);
+    if (e == cudaSuccess) e = qvggt_launch_multipliers(smooth_c, sign_v, K, w->amul, wmul, st);
+    if (e == cudaSuccess) e = qvggt_launch_rsq(W_bf16, K, N, K, wmul, 0, w->Wq, w->w_scale, st);
+    // wmul is scratch: stream-ordered release so that the call stays asynchronous
+    if (cudaFreeAsync(wmul, st) != cudaSuccess) cudaGetLastError();
+    if (e != cudaSuccess) {
+        cudaStreamSynchronize(st);
+        release(w);
+        return QVGGT_ERR_CUDA;
+    }
+    *out = w;
+    return QVGGT_OK;
+}
+
+int qvggt_rotate_smooth_quantize(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M, int group,
+                                 unsigned char *Xq, float *a_scale, void *cuda_stream)
+{
+    if (!w) return QVGGT_ERR_NULL;
+    if (M < 0) return QVGGT_ERR_SHAPE;
+    if (group != 0 && group != 128) return QVGGT_ERR_UNSUPPORTED;
+    if (M == 0) return QVGGT_OK;
+    if (!X_bf16 || !Xq || !a_scale) return QVGGT_ERR_NULL;
+    if (ldx < w->K) return QVGGT_ERR_SHAPE;
+    if (ldx % 8 != 0 || !aligned16(X_bf16) || !aligned16(Xq) || (reinterpret_cast<uintptr_t>(a_scale) & 3u)) return QVGGT_ERR_ALIGN;
+    cudaError_t e = qvggt_launch_rsq(X_bf16, ldx, M, w->K, w->amul, group, Xq, a_scale, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
+}
+
+int qvggt_w4a4_linear(const qvggt_weights_t *w, const unsigned char *Xq, const float *a_scale, int M, int group,
+                      void *Y_bf16, long long ldy, int *acc_debug, void *cuda_stream)
+{
+    if (!w) return QVGGT_ERR_NULL;
+    if (M < 0) return QVGGT_ERR_SHAPE;
+    if (group != 0 && group != 128) return QVGGT_ERR_UNSUPPORTED;
+    if (M == 0) return QVGGT_OK;
+    if (!Xq || !a_scale || !Y_bf16) return QVGGT_ERR_NULL;
+    if (ldy < w->N) return QVGGT_ERR_SHAPE;
+    if (ldy % 8 != 0 || !aligned16(Xq) || !aligned16(Y_bf16) || (acc_debug && !aligned16(acc_debug)) ||
+        (reinterpret_cast<uintptr_t>(a_scale) & 3u))
+        return QVGGT_ERR_ALIGN;
+    cudaError_t e = qvggt_launch_gemm(w, Xq, a_scale, M, group, Y_bf16, ldy, acc_debug, static_cast<cudaStream_t>(cuda_stream));
+    if (e == cudaErrorNotSupported) return QVGGT_ERR_UNSUPPORTED;
+    return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
+}
+
+void qvggt_free_weights(qvggt_weights_t *w)
+{
+    if (!w) return;
+    int cur = 0;
+    cudaGetDevice(&cur);
+    if (cur != w->device) cudaSetDevice(w->device);
+    cudaDeviceSynchronize();
+    release(w);
+    if (cur != w->device) cudaSetDevice(cur);
+}
+
+int qvggt_weights_view(const qvggt_weights_t *w, const unsigned char **Wq, const float **w_scale, const float **amul,
+                       const void **bias_bf16, int *N, int *K)
+{
+    if (!w) return QVGGT_ERR_NULL;
+    if (Wq) *Wq = w->Wq;
+    if (w_scale) *w_scale = w->w_scale;
+    if (amul) *amul = w->amul;
+    if (bias_bf16) *bias_bf16 = w->bias;
+    if (N) *N = w->N;
+    if (K) *K = w->K;
+    return QVGGT_OK;
+}
+
+int qvggt_device_status(const qvggt_weights_t *w, void *cuda_stream, int *code)
+{
+    if (!w || !code) return QVGGT_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return QVGGT_ERR_CUDA;
+    if (cudaMemcpy(code, w->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return QVGGT_ERR_CUDA;
+    return *code == 0 ? QVGGT_OK : QVGGT_ERR_DEVICE_TIMEOUT;
+}
+
+int qvggt_calibrate_smooth(const void *X_calib_bf16, int Mc, const void *W_bf16, int N, int K, float alpha, float lo,
+                           float hi, float *colmax_scratch, float *smooth_c, void *cuda_stream)
+{
+    if (!X_calib_bf16 || !W_bf16 || !colmax_scratch || !smooth_c) return QVGGT_ERR_NULL;
+    if (!valid_k(K) || Mc <= 0 || N <= 0) return QVGGT_ERR_SHAPE;
+    if (!aligned16(X_calib_bf16) || !aligned16(W_bf16)) return QVGGT_ERR_ALIGN;
+    if (!device_is_sm100()) return QVGGT_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaMemsetAsync(colmax_scratch, 0, sizeof(float) * 2 * K, st);
+    if (e == cudaSuccess) e = qvggt_launch_colmax(X_calib_bf16, Mc, K, colmax_scratch, st);
+    if (e == cudaSuccess) e = qvggt_launch_colmax(W_bf16, N, K, colmax_scratch + K, st);
+    if (e == cudaSuccess) e = qvggt_launch_smooth_finalize(colmax_scratch, colmax_scratch + K, K, alpha, lo, hi, smooth_c, st);
+    return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
+}
+
+const char *qvggt_status_string(int status)
+{
+    switch (status) {
+        case QVGGT_OK: return "ok";
+        case QVGGT_ERR_NULL: return "a required pointer is NULL";
+        case QVGGT_ERR_SHAPE: return "unsupported shape (K must be 1024 or 4096, N a multiple of 128, M >= 0, ld >= row length)";
+        case QVGGT_ERR_ALIGN: return "pointer or leading dimension violates the 16-byte alignment rule";
+        case QVGGT_ERR_UNSUPPORTED: return "unsupported option or device (group must be 0 or 128; device must be sm_100)";
+        case QVGGT_ERR_CUDA: return "a CUDA runtime call failed";
+        case QVGGT_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+        case QVGGT_ERR_NOMEM: return "out of memory";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,38 @@
+// Internal declarations shared by the translation units of libqvggt (device code for sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/qvggt.h"
+
+struct qvggt_weights {
+    int N, K;
+    int device;
+    unsigned char *Wq;   // [N, K/2] packed int4
+    float *w_scale;      // [N]
+    float *amul;         // [K]
+    uint16_t *bias;      // [N] bf16 bits, or nullptr
+    int *status;         // device status word (0 = ok)
+};
+
+// Device status codes written by kernels whose bounded waits expire.
+enum : int {
+    QVGGT_DEV_OK = 0,
+    QVGGT_DEV_TIMEOUT_FULL = 1,    // MMA thread gave up waiting for a converted operand stage
+    QVGGT_DEV_TIMEOUT_EMPTY = 2,   // converter gave up waiting for a stage to be released
+    QVGGT_DEV_TIMEOUT_ACCUM = 3,   // epilogue gave up waiting for the accumulator
+    QVGGT_DEV_TIMEOUT_TMEM_FREE = 4 // MMA thread gave up waiting for the epilogue to drain TMEM
+};
+
+// rsq.cu
+cudaError_t qvggt_launch_multipliers(const float *c, const signed char *v, int K, float *amul, float *wmul,
+                                     cudaStream_t st);
+cudaError_t qvggt_launch_rsq(const void *X, long long ldx, int M, int K, const float *mul, int group,
+                             unsigned char *Xq, float *scales, cudaStream_t st);
+cudaError_t qvggt_launch_colmax(const void *X, int M, int K, float *colmax, cudaStream_t st);
+cudaError_t qvggt_launch_smooth_finalize(const float *ax, const float *aw, int K, float alpha, float lo, float hi,
+                                         float *c, cudaStream_t st);
+
+// gemm.cu
+cudaError_t qvggt_launch_gemm(const qvggt_weights *w, const unsigned char *Xq, const float *a_scale, int M,
+                              int group, void *Y, long long ldy, int *acc_debug, cudaStream_t st);

@@ -1,0 +1,287 @@
+// Rotate -> smooth -> 4-bit quantize (Sec. 3.2: pre-global rotation, post-local smooth, Eq. "quantization").
+//
+// One row of K bf16 values is transformed by the un-normalised Sylvester-Hadamard matrix with fp32
+// radix-2 butterflies in ascending-stride order (strides 1, 2, 4, ..., K/2), multiplied by a
+// per-rotated-channel factor, and quantized to signed 4-bit codes with one scale per row or per
+// 128 rotated channels.  The logical stage order and the rounding of every operation are fixed
+// (explicit round-to-nearest intrinsics, no FMA contraction), so codes and scales are reproducible
+// bit for bit; only the mapping of elements to lanes, registers and shared memory is free.
+//
+// The same kernel serves the activations (multiplier amul) and the weight rows (multiplier wmul).
+#include "qvggt_internal.cuh"
+
+namespace {
+
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ int padded(int i) { return i + (i >> 5); }
+
+// Five butterfly stages over the 32 values a thread holds; register bit b is stride 2^b.
+__device__ __forceinline__ void butterfly32(float (&r)[32])
+{
+#pragma unroll
+    for (int h = 1; h < 32; h <<= 1) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            if (!(i & h)) {
+                float a = r[i], b = r[i + h];
+                r[i] = __fadd_rn(a, b);
+                r[i + h] = __fsub_rn(a, b);
+            }
+        }
+    }
+}
+
+template <int K>
+struct RowGeom {
+    static constexpr int T = K / 32;             // threads per row
+    static constexpr int ROWS = kThreads / T;    // rows per CTA pass
+    static constexpr int PADDED = K + K / 32;    // floats of shared memory per row
+};
+
+__device__ __forceinline__ void row_sync(int T, int slot)
+{
+    if (T == 32) {
+        __syncwarp();
+    } else {
+        asm volatile("bar.sync %0, %1;" ::"r"(slot + 1), "r"(T) : "memory");
+    }
+}
+
+// Loads row `x` (bf16, K values), leaves the transformed row in shared memory `s` (padded fp32),
+// element i at s[padded(i)], already multiplied by mul[i] if mul != nullptr.
+template <int K>
+__device__ __forceinline__ void rotate_row_to_smem(const uint16_t *x, const float *mul, float *s, int t, int slot)
+{
+    constexpr int T = RowGeom<K>::T;
+    float r[32];
+    // strides 1..16: thread t holds elements 32t .. 32t+31
+    {
+        const uint4 *src = reinterpret_cast<const uint4 *>(x + t * 32);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            uint4 w = __ldg(src + q);
+            uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                r[q * 8 + 2 * e] = __uint_as_float(ww[e] << 16);
+                r[q * 8 + 2 * e + 1] = __uint_as_float(ww[e] & 0xFFFF0000u);
+            }
+        }
+    }
+    butterfly32(r);
+#pragma unroll
+    for (int j = 0; j < 32; ++j) s[padded(t * 32 + j)] = r[j];
+    row_sync(T, slot);
+    // strides 32..512: thread holds elements base + 32 j
+    const int base = (t >> 5) * 1024 + (t & 31);
+#pragma unroll
+    for (int j = 0; j < 32; ++j) r[j] = s[padded(base + 32 * j)];
+    butterfly32(r);
+    if (K == 1024) {
+        if (mul) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) r[j] = __fmul_rn(r[j], __ldg(mul + base + 32 * j));
+        }
+#pragma unroll
+        for (int j = 0; j < 32; ++j) s[padded(base + 32 * j)] = r[j];
+        row_sync(T, slot);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) s[padded(base + 32 * j)] = r[j];
+        row_sync(T, slot);
+        // strides 1024, 2048: thread holds elements 8t + e + 1024 q  (register 4e + q)
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) r[4 * e + q] = s[padded(8 * t + e + 1024 * q)];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            float a0 = r[4 * e], a1 = r[4 * e + 1], a2 = r[4 * e + 2], a3 = r[4 * e + 3];
+            float b0 = __fadd_rn(a0, a1), b1 = __fsub_rn(a0, a1);   // stride 1024
+            float b2 = __fadd_rn(a2, a3), b3 = __fsub_rn(a2, a3);
+            r[4 * e] = __fadd_rn(b0, b2);                            // stride 2048
+            r[4 * e + 2] = __fsub_rn(b0, b2);
+            r[4 * e + 1] = __fadd_rn(b1, b3);
+            r[4 * e + 3] = __fsub_rn(b1, b3);
+        }
+        if (mul) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) r[4 * e + q] = __fmul_rn(r[4 * e + q], __ldg(mul + 8 * t + e + 1024 * q));
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) s[padded(8 * t + e + 1024 * q)] = r[4 * e + q];
+        row_sync(T, slot);
+    }
+}
+
+template <int K, int GROUP>
+__global__ void __launch_bounds__(kThreads)
+rsq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float *__restrict__ mul,
+           unsigned char *__restrict__ Xq, float *__restrict__ scales)
+{
+    using G = RowGeom<K>;
+    __shared__ float smem[G::ROWS * G::PADDED];
+    __shared__ float red[G::ROWS][4];
+    const int slot = threadIdx.x / G::T;
+    const int t = threadIdx.x % G::T;
+    float *s = smem + slot * G::PADDED;
+
+    for (long long m0 = (long long)blockIdx.x * G::ROWS; m0 < M; m0 += (long long)gridDim.x * G::ROWS) {
+        const long long m = m0 + slot;
+        if (m < M) {
+            rotate_row_to_smem<K>(X + m * ldx, mul, s, t, slot);
+            float y[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) y[j] = s[padded(t * 32 + j)];
+            float amax = 0.0f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) amax = fmaxf(amax, fabsf(y[j]));
+            if (GROUP == 128) {
+                amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
+                amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
+            } else {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
+                if (G::T > 32) {
+                    if ((t & 31) == 0) red[slot][t >> 5] = amax;
+                    row_sync(G::T, slot);
+                    amax = fmaxf(fmaxf(red[slot][0], red[slot][1]), fmaxf(red[slot][2], red[slot][3]));
+                }
+            }
+            amax = fmaxf(amax, 1e-8f);
+            const float scale = __fdiv_rn(amax, 7.0f);
+            const float inv = __fdiv_rn(7.0f, amax);
+            uint32_t packed[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint32_t word = 0;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    // exact product + 1.5*2^23, rounded once (half-to-even): low mantissa bits = two's-complement code
+                    float f = __fmaf_rn(y[q * 8 + e], inv, 12582912.0f);
+                    word |= (__float_as_uint(f) & 0xFu) << (4 * e);
+                }
+                packed[q] = word;
+            }
+            *reinterpret_cast<uint4 *>(Xq + m * (K / 2) + t * 16) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+            if (GROUP == 128) {
+                if ((t & 3) == 0) scales[m * (K / 128) + (t >> 2)] = scale;
+            } else {
+                if (t == 0) scales[m] = scale;
+            }
+        }
+        // the row's shared memory is reused by the next pass
+        if (G::T == 32) __syncwarp(); else __syncthreads();
+    }
+}
+
+// Column-wise absolute maximum of the normalised rotated rows (calibration statistics for Eq. "smooth_factor").
+template <int K>
+__global__ void __launch_bounds__(kThreads)
+colmax_kernel(const uint16_t *__restrict__ X, int M, float *__restrict__ colmax)
+{
+    using G = RowGeom<K>;
+    __shared__ float smem[G::ROWS * G::PADDED];
+    const int slot = threadIdx.x / G::T;
+    const int t = threadIdx.x % G::T;
+    float *s = smem + slot * G::PADDED;
+    const float nrm = (K == 1024) ? 0.03125f : 0.015625f;
+    float best[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) best[j] = 0.0f;
+    for (long long m0 = (long long)blockIdx.x * G::ROWS; m0 < M; m0 += (long long)gridDim.x * G::ROWS) {
+        const long long m = m0 + slot;
+        if (m < M) {
+            rotate_row_to_smem<K>(X + m * (long long)K, nullptr, s, t, slot);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) best[j] = fmaxf(best[j], fabsf(s[padded(t * 32 + j)]));
+        }
+        if (G::T == 32) __syncwarp(); else __syncthreads();
+    }
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        // non-negative floats order like their bit patterns
+        atomicMax(reinterpret_cast<int *>(colmax) + t * 32 + j, __float_as_int(__fmul_rn(best[j], nrm)));
+    }
+}
+
+__global__ void multipliers_kernel(const float *__restrict__ c, const signed char *__restrict__ v, int K,
+                                   float *__restrict__ amul, float *__restrict__ wmul)
+{
+    int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= K) return;
+    const float nrm = (K == 1024) ? 0.03125f : 0.015625f;   // K^{-1/2}, exact
+    const float sgn = (v != nullptr && v[k] < 0) ? -nrm : nrm;
+    if (amul) amul[k] = __fdiv_rn(sgn, c[k]);
+    if (wmul) wmul[k] = __fmul_rn(sgn, c[k]);
+}
+
+__global__ void smooth_finalize_kernel(const float *__restrict__ ax, const float *__restrict__ aw, int K, float alpha,
+                                       float lo, float hi, float *__restrict__ c)
+{
+    int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= K) return;
+    float x = ax[k], w = aw[k], r;
+    if (x == 0.0f && w == 0.0f) r = 1.0f;
+    else r = powf(x, alpha) / powf(w, 1.0f - alpha);
+    if (!(r >= lo)) r = lo;
+    if (r > hi) r = hi;
+    c[k] = r;
+}
+
+int rsq_grid(int M, int rows_per_cta)
+{
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    long long need = ((long long)M + rows_per_cta - 1) / rows_per_cta;
+    long long cap = (long long)sms * 6;
+    return (int)(need < cap ? need : cap);
+}
+
+}  // namespace
+
+cudaError_t qvggt_launch_multipliers(const float *c, const signed char *v, int K, float *amul, float *wmul,
+                                     cudaStream_t st)
+{
+    multipliers_kernel<<<(K + 255) / 256, 256, 0, st>>>(c, v, K, amul, wmul);
+    return cudaGetLastError();
+}
+
+cudaError_t qvggt_launch_rsq(const void *X, long long ldx, int M, int K, const float *mul, int group,
+                             unsigned char *Xq, float *scales, cudaStream_t st)
+{
+    if (M == 0) return cudaSuccess;
+    const uint16_t *x = static_cast<const uint16_t *>(X);
+    if (K == 1024) {
+        int grid = rsq_grid(M, RowGeom<1024>::ROWS);
+        if (group == 128) rsq_kernel<1024, 128><<<grid, kThreads, 0, st>>>(x, ldx, M, mul, Xq, scales);
+        else rsq_kernel<1024, 0><<<grid, kThreads, 0, st>>>(x, ldx, M, mul, Xq, scales);
+    } else {
+        int grid = rsq_grid(M, RowGeom<4096>::ROWS);
+        if (group == 128) rsq_kernel<4096, 128><<<grid, kThreads, 0, st>>>(x, ldx, M, mul, Xq, scales);
+        else rsq_kernel<4096, 0><<<grid, kThreads, 0, st>>>(x, ldx, M, mul, Xq, scales);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t qvggt_launch_colmax(const void *X, int M, int K, float *colmax, cudaStream_t st)
+{
+    if (M == 0) return cudaSuccess;
+    const uint16_t *x = static_cast<const uint16_t *>(X);
+    if (K == 1024) colmax_kernel<1024><<<rsq_grid(M, RowGeom<1024>::ROWS), kThreads, 0, st>>>(x, M, colmax);
+    else colmax_kernel<4096><<<rsq_grid(M, RowGeom<4096>::ROWS), kThreads, 0, st>>>(x, M, colmax);
+    return cudaGetLastError();
+}
+
+cudaError_t qvggt_launch_smooth_finalize(const float *ax, const float *aw, int K, float alpha, float lo, float hi,
+                                         float *c, cudaStream_t st)
+{
+    smooth_finalize_kernel<<<(K + 255) / 256, 256, 0, st>>>(ax, aw, K, alpha, lo, hi, c);
+    return cudaGetLastError();
+}
