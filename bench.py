@@ -72,9 +72,15 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([t.strip() for t in line.split(",")])
+            self.rows.append((time.time(), [t.strip() for t in line.split(",")]))
 
-    def stop(self):
+    def wait_first_sample(self, timeout=5.0):
+        t0 = time.time()
+        while self.proc and not self.rows and time.time() - t0 < timeout:
+            time.sleep(0.02)
+
+    def stop(self, t_begin=0.0, t_end=float("inf")):
+        """Summary of the samples taken between wall-clock t_begin and t_end (the timed region)."""
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -83,7 +89,10 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         sm, smax, reasons = [], None, set()
-        for r in self.rows:
+        inside = [r for (t, r) in self.rows if t_begin <= t <= t_end]
+        if not inside:                       # region shorter than one sampling period: take the nearest samples
+            inside = [r for (_, r) in self.rows[-3:]]
+        for r in inside:
             try:
                 sm.append(float(r[0]))
                 smax = float(r[1])
@@ -134,7 +143,7 @@ def run_reference(args, rank, world):
     }))
 
 
-def cpu_baseline(rows=workload.TOKENS_PER_FRAME):
+def cpu_baseline(rows=FRAMES * workload.TOKENS_PER_FRAME):
     import oracle
     specs = workload.block_specs(0, 0)
     ops, dt, timings = 0.0, 0.0, {}
@@ -147,7 +156,7 @@ def cpu_baseline(rows=workload.TOKENS_PER_FRAME):
         dt += time.perf_counter() - t0
         ops += layer_ops(rows, s)
     return {"value": ops / dt / 1e12, "unit": "TOPS", "cores": oracle.threads(), "kind": "oracle",
-            "sample": f"first {rows} token rows (one frame) of the batch through all four linears, one pass, {dt:.1f} s",
+            "sample": f"the whole {rows}-token batch through all four linears, one pass, {dt:.1f} s of wall clock",
             "tokens_per_s": rows / dt, "seconds": {k: round(v, 3) for k, v in timings.items()}}
 
 
@@ -209,14 +218,17 @@ def run_ours(args, rank, world, local_rank):
     kev = [[[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in layers] for _ in range(args.steps)]
     sampler = ClockSampler(local_rank)
     sampler.start()
+    sampler.wait_first_sample()
     t_start, t_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    wall0 = time.time()
     t_start.record()
     for i in range(args.steps):
         step(i, kev[i])
     t_stop.record()
     barrier()
-    clocks = sampler.stop()
+    wall1 = time.time()
+    clocks = sampler.stop(wall0, wall1)
     total_ms = t_start.elapsed_time(t_stop)
     if dist is not None:
         t = torch.tensor([total_ms], device="cuda")
@@ -313,7 +325,7 @@ def run_ours(args, rank, world, local_rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--ref-rows", type=int, default=512, help="token rows per step of the oracle arm")
