@@ -127,6 +127,26 @@ int qvggt_device_status(const qvggt_weights_t *w, void *cuda_stream, int *code);
 int qvggt_calibrate_smooth(const void *X_calib_bf16, int Mc, const void *W_bf16, int N, int K, float alpha,
                            float lo, float hi, float *colmax_scratch, float *smooth_c, void *cuda_stream);
 
+/*
+ * Allocation-free variant of the weight quantization in qvggt_prepare_weights.  (The paper has no
+ * counterpart; this exists for deployment.)  For callers that cannot allocate device memory at this point:
+ * a process whose whole device memory already belongs to its own arena, or a section that cannot
+ * take the device-wide synchronisation cudaMalloc/cudaFree may imply.  It calls no cudaMalloc,
+ * cudaFree or any other allocating routine.  Same arithmetic and results as qvggt_prepare_weights:
+ *   Wq      [N, K/2] packed int4 (output, caller-allocated, 16-byte aligned)
+ *   w_scale fp32 [N] (output)        amul  fp32 [K] (output, for the activation path)
+ *   W_bf16 [N, K] bf16 16-byte aligned; smooth_c fp32 [K]; sign_v int8 [K] or NULL; any N >= 1.
+ * The temporary weight-side multipliers live in a fixed 16 KB device array inside the library
+ * (held by every GPU that loads it, until the process exits), which limits K to at most 4096:
+ * a larger K is refused with QVGGT_ERR_SHAPE.  The array is shared by all calls and keeps the
+ * previous call's contents; each call rewrites the part it reads, but two calls whose kernels
+ * overlap on the GPU (different streams) race on it -- serialise them.  The first call on each
+ * device looks up the array's device address (with that device current); make that first call
+ * before any stream capture begins.
+ */
+int qvggt_quantize_weights_static(const void *W_bf16, const float *smooth_c, const signed char *sign_v, int N,
+                                  int K, unsigned char *Wq, float *w_scale, float *amul, void *cuda_stream);
+
 /* Static, NUL-terminated description of a status code. */
 const char *qvggt_status_string(int status);
 

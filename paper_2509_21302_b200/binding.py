@@ -19,7 +19,8 @@ _STATUS_NAMES = {0: "QVGGT_OK", -1: "QVGGT_ERR_NULL", -2: "QVGGT_ERR_SHAPE", -3:
                  -7: "QVGGT_ERR_NOMEM"}
 
 EXPORTS = ("qvggt_prepare_weights", "qvggt_rotate_smooth_quantize", "qvggt_w4a4_linear", "qvggt_free_weights",
-           "qvggt_weights_view", "qvggt_device_status", "qvggt_calibrate_smooth", "qvggt_status_string")
+           "qvggt_weights_view", "qvggt_device_status", "qvggt_calibrate_smooth", "qvggt_status_string",
+           "qvggt_quantize_weights_static")
 
 
 class QvggtError(RuntimeError):
@@ -50,6 +51,7 @@ def lib() -> ctypes.CDLL:
         L.qvggt_weights_view.argtypes = [vp] + [ctypes.POINTER(vp)] * 4 + [ctypes.POINTER(i32)] * 2
         L.qvggt_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
         L.qvggt_calibrate_smooth.argtypes = [vp, i32, vp, i32, i32, f32, f32, f32, vp, vp, vp]
+        L.qvggt_quantize_weights_static.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp]
         L.qvggt_status_string.argtypes = [i32]
         L.qvggt_status_string.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -200,3 +202,20 @@ def calibrate_smooth(X_calib: torch.Tensor, W: torch.Tensor, alpha: float = 0.5,
     _check(lib().qvggt_calibrate_smooth(_ptr(X_calib), Mc, _ptr(W), N, K, alpha, lo, hi, _ptr(scratch), _ptr(c), _stream()),
            "qvggt_calibrate_smooth")
     return c
+
+
+def quantize_weights_static(W: torch.Tensor, smooth_c: torch.Tensor, sign_v: torch.Tensor | None, Wq: torch.Tensor,
+                            w_scale: torch.Tensor, amul: torch.Tensor) -> None:
+    """Weight quantization into caller-provided buffers without any device allocation.
+
+    For callers that cannot allocate (all device memory already owned by their own arena, or no
+    implicit device synchronisation allowed): the temporary multipliers live in a fixed array
+    inside the library, so K <= 4096 and concurrent calls on different streams must be serialised.
+    W [N,K] bf16, smooth_c [K] fp32, sign_v [K] int8 or None -> Wq [N,K/2] uint8, w_scale [N], amul [K].
+    """
+    N, K = W.shape
+    assert W.element_size() == 2 and W.is_contiguous() and smooth_c.dtype == torch.float32
+    assert Wq.dtype == torch.uint8 and Wq.shape == (N, K // 2) and Wq.is_contiguous()
+    assert w_scale.dtype == torch.float32 and w_scale.numel() == N and amul.dtype == torch.float32 and amul.numel() == K
+    _check(lib().qvggt_quantize_weights_static(_ptr(W), _ptr(smooth_c), _ptr(sign_v), N, K, _ptr(Wq), _ptr(w_scale),
+                                               _ptr(amul), _stream()), "qvggt_quantize_weights_static")
