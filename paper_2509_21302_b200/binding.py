@@ -11,7 +11,7 @@ import os
 
 import torch
 
-from . import build as _build
+from . import buildlib as _build
 
 OK = 0
 _STATUS_NAMES = {0: "QVGGT_OK", -1: "QVGGT_ERR_NULL", -2: "QVGGT_ERR_SHAPE", -3: "QVGGT_ERR_ALIGN",
