@@ -1,332 +1,380 @@
 // W4A4 GEMM + rescale + bias + bf16 for sm_100a (Sec. 3.2: integer sum over the inner dimension,
 // per-token and per-out-channel scales applied outside the sum).
 //
-// tcgen05 has no 4-bit integer kind, so the codes are fed to kind::i8.  Converter warps read the
-// packed codes straight from global memory (L2), expand every nibble into the HIGH half of a byte
-// (value 16*q, no sign extension needed) and write the int8 operand tiles into shared memory in
-// the 128-byte-swizzled K-major layout the tensor core reads.  The raw accumulator is therefore
-// 256 * sum(q_x q_w) (at most 2^26 in magnitude), shifted back exactly in the epilogue.  Even and
-// odd codes of a 32-code slice land in separate 16-byte chunks; the same permutation of K is
-// applied to both operands, so the dot product is unchanged.
+// tcgen05 has no 4-bit integer kind, so the codes are fed to kind::i8.  TMA stages tiles of packed
+// codes in shared memory; converter warps expand every nibble into the HIGH half of a byte (value
+// 16*q, so no sign extension is needed) and write the int8 operand tiles in the 128-byte-swizzled
+// K-major layout the tensor core reads.  The raw accumulator is therefore 256 * sum(q_x q_w) (at
+// most 2^26 in magnitude), undone exactly in the epilogue.  Even and odd codes of a 32-code slice
+// land in separate 16-byte chunks; the same permutation of K is applied to both operands, so the
+// dot product is unchanged.
+//
+// Persistent and warp-specialised.  A "worker" is one CTA (CG = 1: tile 128 tokens x 256 channels)
+// or a pair of CTAs on neighbouring SMs (CG = 2: tile 256 x 256, each CTA stages 128 token rows and
+// 128 weight rows, one thread of the leader CTA issues tcgen05.mma.cta_group::2 for both).
+//   warps 0-7    epilogue: TMEM -> registers -> scale, bias, bf16 -> swizzled staging -> TMA store
+//   warps 8-15   converters: packed stage -> registers -> int8 operand stage
+//   warp  16     one thread issues tcgen05.mma and the commits that release stages / publish accumulators
+//   warp  17     one thread issues the TMA loads of packed tiles
+// Every wait is bounded; on expiry the kernel records a code in *status and all roles fall through
+// to the common exit, where tensor memory is released.
+#include <cuda.h>
 #include <cuda_bf16.h>
 
 #include "qvggt_internal.cuh"
 #include "sm100_ptx.cuh"
 
-#ifdef QVGGT_PROFILE
-__device__ long long g_prof[32];
-extern "C" int qvggt_debug_read_prof(long long *host_out)
-{
-    return (int)cudaMemcpyFromSymbol(host_out, g_prof, sizeof(long long) * 32);
-}
-#define PROF_DECL(n) long long n = 0
-#define PROF_T0(t) long long t = clock64()
-#define PROF_ADD(acc, t) do { long long _n = clock64(); acc += _n - t; t = _n; } while (0)
-#define PROF_STORE(i, v) do { g_prof[i] = (v); } while (0)
-#else
-#define PROF_DECL(n)
-#define PROF_T0(t)
-#define PROF_ADD(acc, t)
-#define PROF_STORE(i, v)
-#endif
-
 namespace {
 
-constexpr int BM = 128;            // tokens per CTA tile (TMEM lanes)
+constexpr int BM = 128;            // token rows per CTA (TMEM lanes)
+constexpr int BN = 256;            // output channels per tile
 constexpr int BK = 128;            // codes along K per pipeline stage = one 128-byte swizzled row of int8
-constexpr int STAGES = 4;          // shared-memory operand ring; also the converter's register ring
-constexpr int PREFETCH = 3;        // K-blocks of packed codes in flight (in registers) per converter thread
+constexpr int EPI_WARPS = 8;       // warp w reads TMEM lanes 32*(w%4).., columns 128*(w/4)..
 constexpr int CONV_WARPS = 8;
-constexpr int CONV_THREADS = CONV_WARPS * 32;
-constexpr int MMA_WARP = CONV_WARPS;
-constexpr int EPI_WARP0 = CONV_WARPS + 1;
-constexpr int EPI_WARPS = 4;       // warp (EPI_WARP0 + i) owns TMEM lanes 32 * ((EPI_WARP0 + i) % 4) ..
-constexpr int EPI_THREADS = EPI_WARPS * 32;
-constexpr int THREADS = (CONV_WARPS + 1 + EPI_WARPS) * 32;
+constexpr int CONV_WARP0 = EPI_WARPS;
+constexpr int MMA_WARP = EPI_WARPS + CONV_WARPS;
+constexpr int TMA_WARP = MMA_WARP + 1;
+constexpr int THREADS = (TMA_WARP + 1) * 32;
 constexpr int ACC_BUFS = 2;        // TMEM accumulators: the epilogue of tile i overlaps the MMAs of tile i+1
+constexpr int STG_BYTES = 32 * 128;   // per epilogue warp: 32 rows x 64 bf16, 128-byte swizzled
 
-template <int BN>
-struct Tile {
-    static constexpr int A_BYTES = BM * 128;
-    static constexpr int B_BYTES = BN * 128;
-    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int CHUNKS = (BM + BN) * 4 / CONV_THREADS;   // 16-byte packed pieces per thread per stage
-    static constexpr int OFF_WSCALE = STAGES * STAGE_BYTES;
-    static constexpr int OFF_BIAS = OFF_WSCALE + BN * 4;
-    static constexpr int OFF_BAR = OFF_BIAS + BN * 4;             // full[STAGES], empty[STAGES], tfull[2], tempty[2]
-    static constexpr int NBARS = 2 * STAGES + 2 * ACC_BUFS;
+template <int CG>
+struct Cfg {
+    static constexpr int B_ROWS = BN / CG;                 // weight rows staged by one CTA
+    static constexpr int ROWS = BM + B_ROWS;
+    static constexpr int PK_STAGE = ROWS * (BK / 2);       // packed codes
+    static constexpr int UP_STAGE = ROWS * BK;             // int8 operands
+    static constexpr int PS = 4;                           // packed stages (cover the L2 latency)
+    static constexpr int US = (CG == 1) ? 2 : 4;           // operand stages (decouple converters and MMA)
+    // Converter warps form GROUPS independent groups; group g converts K-blocks g, g + GROUPS, ...  so the
+    // fixed costs of a stage (draining the stores, the proxy fence, barrier round trips) overlap.
+    static constexpr int GROUPS = (CG == 1) ? 2 : 4;
+    static constexpr int GROUP_WARPS = CONV_WARPS / GROUPS;
+    static constexpr int GROUP_THREADS = GROUP_WARPS * 32;
+    static constexpr int CHUNKS = ROWS * 4 / GROUP_THREADS;   // 16-byte packed pieces per thread per stage
+    static constexpr int BATCH = (CG == 1) ? 6 : 8;           // pieces held in registers at a time
+    static_assert(CHUNKS % BATCH == 0, "stage must split into whole register batches");
+    static constexpr int OFF_UP = 0;                       // operand stages first: they need 1024-byte alignment
+    static constexpr int OFF_STG = OFF_UP + US * UP_STAGE;
+    static constexpr int OFF_PK = OFF_STG + EPI_WARPS * STG_BYTES;
+    static constexpr int OFF_BAR = OFF_PK + PS * PK_STAGE; // pfull[PS] pempty[PS] ufull[US] uempty[US] tfull[2] tempty[2]
+    static constexpr int NBARS = 2 * PS + 2 * US + 2 * ACC_BUFS;
     static constexpr int OFF_TMEM = OFF_BAR + NBARS * 8;
     static constexpr int OFF_ABORT = OFF_TMEM + 4;
     static constexpr int BYTES = OFF_ABORT + 4;
-    static constexpr int DYN_SMEM = BYTES + 1024;                 // slack to align the base to 1024 bytes
-    static constexpr int TMEM_COLS = ACC_BUFS * BN;               // 512 (BN = 256) or 256 (BN = 128): powers of two
+    static constexpr int DYN_SMEM = BYTES + 1024;          // slack to align the base to 1024 bytes
+    static constexpr int TMEM_COLS = ACC_BUFS * BN;        // 512
+    static_assert(DYN_SMEM <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
+    static_assert(UP_STAGE % 1024 == 0 && (BM * BK) % 1024 == 0, "operand tiles must stay 1024-byte aligned");
 };
 
-__device__ __forceinline__ float bf16_bits_to_f32(uint16_t b) { return __uint_as_float(static_cast<uint32_t>(b) << 16); }
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
-// Persistent, warp-specialised: CTA b works on tiles b, b + gridDim.x, ... (n fastest, so CTAs that run
-// together share the token rows of A and all of W stays in L2).
-//   warps 0-7   converters: packed codes global -> registers (PREFETCH K-blocks ahead) -> int8 operand tiles in smem
-//   warp  8     one thread issues tcgen05.mma and the commits that release stages / publish accumulators
-//   warps 9-12  epilogue: TMEM -> registers -> scale, bias, bf16 -> global
-template <int BN>
+template <int CG>
 __global__ void __launch_bounds__(THREADS, 1)
-gemm_w4a4_kernel(const unsigned char *__restrict__ Xq, const unsigned char *__restrict__ Wq,
-                 const float *__restrict__ a_scale, const float *__restrict__ w_scale,
-                 const uint16_t *__restrict__ bias, uint16_t *__restrict__ Y, long long ldy,
-                 int *__restrict__ acc_debug, int M, int N, int K, int *status)
+gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                 const __grid_constant__ CUtensorMap map_y, const float *__restrict__ a_scale,
+                 const float *__restrict__ w_scale, const uint16_t *__restrict__ bias, int *__restrict__ acc_debug,
+                 int M, int N, int K, int *status)
 {
-    using T = Tile<BN>;
-    static_assert(STAGES == 4 && PREFETCH == 3, "the converter loop is unrolled for a 4-slot ring");
+    using C = Cfg<CG>;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = ptx::smem_addr(smem);
-    float *s_wscale = reinterpret_cast<float *>(smem + T::OFF_WSCALE);
-    float *s_bias = reinterpret_cast<float *>(smem + T::OFF_BIAS);
-    const uint32_t bar_full = sbase + T::OFF_BAR;
-    const uint32_t bar_empty = bar_full + STAGES * 8;
-    const uint32_t bar_tfull = bar_empty + STAGES * 8;
+    const uint32_t bar_pfull = sbase + C::OFF_BAR;
+    const uint32_t bar_pempty = bar_pfull + C::PS * 8;
+    const uint32_t bar_ufull = bar_pempty + C::PS * 8;
+    const uint32_t bar_uempty = bar_ufull + C::US * 8;
+    const uint32_t bar_tfull = bar_uempty + C::US * 8;
     const uint32_t bar_tempty = bar_tfull + ACC_BUFS * 8;
-    uint32_t *s_tmem = reinterpret_cast<uint32_t *>(smem + T::OFF_TMEM);
-    volatile int *s_abort = reinterpret_cast<volatile int *>(smem + T::OFF_ABORT);
+    uint32_t *s_tmem = reinterpret_cast<uint32_t *>(smem + C::OFF_TMEM);
+    volatile int *s_abort = reinterpret_cast<volatile int *>(smem + C::OFF_ABORT);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int KB = K / BK;                      // 8 or 32: a multiple of STAGES
-    const int row_bytes = K / 2;
-    const int n_tiles = N / BN;
-    const int total_tiles = ((M + BM - 1) / BM) * n_tiles;
-    const int my_tiles = (total_tiles > (int)blockIdx.x) ? (total_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    const uint32_t rank = (CG == 2) ? ptx::cluster_ctarank() : 0u;     // 0 = leader of the pair
+    const int worker = blockIdx.x / CG, workers = gridDim.x / CG;
+    const int KB = K / BK;
+    const int n_tiles = (N + BN - 1) / BN;
+    const int total_tiles = ((M + BM * CG - 1) / (BM * CG)) * n_tiles;
+    const int my_tiles = (total_tiles > worker) ? (total_tiles - 1 - worker) / workers + 1 : 0;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            ptx::mbar_init(bar_full + 8 * s, CONV_WARPS);     // one arrival per converter warp
-            ptx::mbar_init(bar_empty + 8 * s, 1);
+        for (int s = 0; s < C::PS; ++s) {
+            ptx::mbar_init(bar_pfull + 8 * s, 1);                    // the producer's arrive.expect_tx
+            ptx::mbar_init(bar_pempty + 8 * s, C::GROUP_WARPS);
+        }
+        for (int s = 0; s < C::US; ++s) {
+            ptx::mbar_init(bar_ufull + 8 * s, C::GROUP_WARPS * CG); // one converter group of every CTA of the worker
+            ptx::mbar_init(bar_uempty + 8 * s, 1);                   // tcgen05.commit
         }
         for (int b = 0; b < ACC_BUFS; ++b) {
-            ptx::mbar_init(bar_tfull + 8 * b, 1);
-            ptx::mbar_init(bar_tempty + 8 * b, EPI_WARPS);
+            ptx::mbar_init(bar_tfull + 8 * b, 1);                    // tcgen05.commit
+            ptx::mbar_init(bar_tempty + 8 * b, EPI_WARPS * CG);
         }
         *s_abort = 0;
         ptx::fence_mbar_init();
     }
     if (warp == MMA_WARP) {
-        ptx::tmem_alloc(ptx::smem_addr(s_tmem), T::TMEM_COLS);
-        ptx::tmem_relinquish();
+        if (CG == 2) { ptx::tmem_alloc_pair(ptx::smem_addr(s_tmem), C::TMEM_COLS); ptx::tmem_relinquish_pair(); }
+        else         { ptx::tmem_alloc(ptx::smem_addr(s_tmem), C::TMEM_COLS);      ptx::tmem_relinquish(); }
+    }
+    if (warp == TMA_WARP && lane == 0) {
+        ptx::prefetch_tensormap(&map_x);
+        ptx::prefetch_tensormap(&map_w);
+        ptx::prefetch_tensormap(&map_y);
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if (CG == 2) ptx::cluster_sync();        // the peer's barriers exist before anything arrives on them remotely
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *s_tmem;
 
-    if (warp < CONV_WARPS) {
-        // ------------------------------------------------------------ converters
-        int row_of[T::CHUNKS];          // row inside the A region (< BM) or BM + row inside the B region
-        uint32_t soff[T::CHUNKS];
-#pragma unroll
-        for (int i = 0; i < T::CHUNKS; ++i) {
-            const int c = threadIdx.x + CONV_THREADS * i;
-            const int row = c >> 2, piece = c & 3;
-            row_of[i] = row;
-            // even codes -> 16-byte chunk 2*piece, odd codes -> chunk 2*piece+1, both XOR (row mod 8)
-            soff[i] = (row < BM ? row * 128 : T::A_BYTES + (row - BM) * 128) + (((2 * piece) ^ (row & 7)) << 4);
-        }
-        const int piece_off = (threadIdx.x & 3) * 16;
-
-        // load cursor: walks (tile, kb) PREFETCH blocks ahead of the conversion
-        const unsigned char *lptr[T::CHUNKS];
-        int l_tile = 0, l_kb = 0;
-        auto set_tile_ptrs = [&](int t_local) {
-            const int tile = blockIdx.x + t_local * gridDim.x;
-            const int m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
-#pragma unroll
-            for (int i = 0; i < T::CHUNKS; ++i) {
-                if (row_of[i] < BM) {
-                    const int gm = m0 + row_of[i];
-                    lptr[i] = (gm < M) ? Xq + (long long)gm * row_bytes + piece_off : nullptr;
-                } else {
-                    lptr[i] = Wq + (long long)(n0 + row_of[i] - BM) * row_bytes + piece_off;
-                }
-            }
-        };
-        auto issue_load = [&](uint4 (&dst)[T::CHUNKS]) {
-            if (l_tile < my_tiles) {
-#pragma unroll
-                for (int i = 0; i < T::CHUNKS; ++i) {
-#ifdef QVGGT_PROBE_NO_LOADS
-                    dst[i] = make_uint4(l_kb, i, l_tile, 0);
-#else
-                    dst[i] = lptr[i] ? __ldg(reinterpret_cast<const uint4 *>(lptr[i] + l_kb * (BK / 2))) : make_uint4(0, 0, 0, 0);
-#endif
-                }
-                if (++l_kb == KB) {
-                    l_kb = 0;
-                    if (++l_tile < my_tiles) set_tile_ptrs(l_tile);
-                }
-            }
-        };
-        auto convert = [&](const uint4 (&src)[T::CHUNKS], unsigned char *stage) {
-#pragma unroll
-            for (int i = 0; i < T::CHUNKS; ++i) {
-                const uint4 w = src[i];
-                uint4 lo, hi;
-                lo.x = (w.x << 4) & 0xF0F0F0F0u; hi.x = w.x & 0xF0F0F0F0u;
-                lo.y = (w.y << 4) & 0xF0F0F0F0u; hi.y = w.y & 0xF0F0F0F0u;
-                lo.z = (w.z << 4) & 0xF0F0F0F0u; hi.z = w.z & 0xF0F0F0F0u;
-                lo.w = (w.w << 4) & 0xF0F0F0F0u; hi.w = w.w & 0xF0F0F0F0u;
-                *reinterpret_cast<uint4 *>(stage + soff[i]) = lo;
-                *reinterpret_cast<uint4 *>(stage + (soff[i] ^ 16)) = hi;
-            }
-        };
-
-        uint4 buf[STAGES][T::CHUNKS];
-        if (my_tiles > 0) set_tile_ptrs(0);
-        issue_load(buf[0]);
-        issue_load(buf[1]);
-        issue_load(buf[2]);
-        const int rounds = my_tiles * (KB / STAGES);
+    if (warp < EPI_WARPS) {
+        // ------------------------------------------------------------ epilogue
+        const int quarter = warp & 3, chalf = warp >> 2;   // TMEM lane quarter, column half
+        unsigned char *stg = smem + C::OFF_STG + warp * STG_BYTES;
+        const uint32_t stg_addr = sbase + C::OFF_STG + warp * STG_BYTES;
+        const uint32_t leader_tempty = (CG == 2) ? ptx::map_to_cta(bar_tempty, 0) : bar_tempty;
         bool alive = true;
-        PROF_DECL(p_load); PROF_DECL(p_wait); PROF_DECL(p_conv); PROF_DECL(p_fence); PROF_DECL(p_arrive);
-        PROF_T0(pt);
-        for (int r = 0; r < rounds && alive; ++r) {
+        for (int t = 0; t < my_tiles; ++t) {
+            const int tile = worker + t * workers;
+            const int m0 = (tile / n_tiles) * (BM * CG) + (int)rank * BM + quarter * 32;
+            const int n0 = (tile % n_tiles) * BN + chalf * 128;
+            const int b = t & 1;
+            const int gm = m0 + lane;
+            const bool row_ok = gm < M;
+            const bool cols_ok = n0 < N;                       // N is a multiple of 128: a half tile is all in or all out
+            // a_scale / 256: exact (power of two), cancels the factor 256 carried by the raw accumulator
+            const float as = row_ok ? __fmul_rn(__ldg(a_scale + gm), 0.00390625f) : 0.0f;
+            if (alive) alive = ptx::mbar_wait_warp(bar_tfull + 8 * b, (t >> 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM, lane, 32);
+            ptx::tc_fence_after_sync();
+            if (alive) {
+#pragma unroll 1
+                for (int box = 0; box < 2; ++box) {
+                    // the previous TMA store has finished reading the staging buffer
+                    if (lane == 0) ptx::tma_store_wait_read<0>();
+                    __syncwarp();
 #pragma unroll
-            for (int u = 0; u < STAGES; ++u) {
-                issue_load(buf[(u + PREFETCH) & (STAGES - 1)]);
-                PROF_ADD(p_load, pt);
-                if (r > 0) alive = alive && ptx::mbar_wait_warp(bar_empty + 8 * u, (r - 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_EMPTY, lane);
-                PROF_ADD(p_wait, pt);
-                if (alive) {
-                    convert(buf[u], smem + u * T::STAGE_BYTES);
-                    PROF_ADD(p_conv, pt);
-                    ptx::fence_proxy_async_smem();      // my generic-proxy writes -> visible to the tensor core's async proxy
-                    PROF_ADD(p_fence, pt);
+                    for (int c = 0; c < 2; ++c) {
+                        const int col = box * 64 + c * 32;                // within this warp's 128 columns
+                        uint32_t raw[32];
+                        ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + b * BN + chalf * 128 + col, raw);
+                        ptx::tmem_ld_wait();
+                        if (box == 1 && c == 1) {
+                            // last read of this accumulator: hand it back to the MMA thread before the math
+                            ptx::tc_fence_before_sync();
+                            __syncwarp();
+                            if (lane == 0) {
+                                if (CG == 2) ptx::mbar_arrive_cluster(leader_tempty + 8 * b);
+                                else ptx::mbar_arrive(bar_tempty + 8 * b);
+                            }
+                        }
+                        if (cols_ok) {
+                            const float4 *ws4 = reinterpret_cast<const float4 *>(w_scale + n0 + col);
+                            const uint2 *bs2 = reinterpret_cast<const uint2 *>(bias + n0 + col);
+                            uint32_t out[16];
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4) {
+                                const float4 ws = __ldg(ws4 + (j >> 2));
+                                float2 b01 = make_float2(0.0f, 0.0f), b23 = make_float2(0.0f, 0.0f);
+                                if (bias) {
+                                    const uint2 bb = __ldg(bs2 + (j >> 2));
+                                    b01 = make_float2(bf16_lo(bb.x), bf16_hi(bb.x));
+                                    b23 = make_float2(bf16_lo(bb.y), bf16_hi(bb.y));
+                                }
+                                const float2 t01 = ptx::mul_f32x2(make_float2(as, as), make_float2(ws.x, ws.y));
+                                const float2 t23 = ptx::mul_f32x2(make_float2(as, as), make_float2(ws.z, ws.w));
+                                float2 z01 = make_float2(static_cast<float>(static_cast<int>(raw[j])), static_cast<float>(static_cast<int>(raw[j + 1])));
+                                float2 z23 = make_float2(static_cast<float>(static_cast<int>(raw[j + 2])), static_cast<float>(static_cast<int>(raw[j + 3])));
+                                z01 = ptx::mul_f32x2(z01, t01);
+                                z23 = ptx::mul_f32x2(z23, t23);
+                                if (bias) {
+                                    z01 = ptx::add_f32x2(z01, b01);
+                                    z23 = ptx::add_f32x2(z23, b23);
+                                }
+                                out[j >> 1] = ptx::pack_bf16x2(z01.x, z01.y);
+                                out[(j >> 1) + 1] = ptx::pack_bf16x2(z23.x, z23.y);
+                            }
+                            // row `lane` of the staging tile, 16-byte chunk (4c + q) XOR (lane mod 8)
+#pragma unroll
+                            for (int q = 0; q < 4; ++q)
+                                *reinterpret_cast<uint4 *>(stg + lane * 128 + (((4 * c + q) ^ (lane & 7)) << 4)) =
+                                    make_uint4(out[4 * q], out[4 * q + 1], out[4 * q + 2], out[4 * q + 3]);
+                            if (acc_debug && row_ok) {
+                                uint4 *dbg = reinterpret_cast<uint4 *>(acc_debug + (long long)gm * N + n0 + col);
+#pragma unroll
+                                for (int q = 0; q < 8; ++q)
+                                    dbg[q] = make_uint4(static_cast<int>(raw[4 * q]) >> 8, static_cast<int>(raw[4 * q + 1]) >> 8,
+                                                        static_cast<int>(raw[4 * q + 2]) >> 8, static_cast<int>(raw[4 * q + 3]) >> 8);
+                            }
+                        }
+                    }
+                    ptx::fence_proxy_async_smem();          // staging writes -> visible to the TMA engine
+                    __syncwarp();
+                    if (lane == 0 && cols_ok && m0 < M) {
+                        ptx::tma_store_2d(&map_y, stg_addr, n0 + box * 64, m0);   // rows >= M are clipped by the tensor map
+                        ptx::tma_store_commit();
+                    }
                 }
-                __syncwarp();                            // orders the whole warp's writes before the single arrival
-                if (alive && lane == 0) ptx::mbar_arrive(bar_full + 8 * u);
-                PROF_ADD(p_arrive, pt);
             }
         }
-#ifdef QVGGT_PROFILE
-        if (blockIdx.x == 0 && threadIdx.x == 0) {
-            PROF_STORE(0, p_load); PROF_STORE(1, p_wait); PROF_STORE(2, p_conv); PROF_STORE(3, p_fence); PROF_STORE(4, p_arrive);
-            PROF_STORE(5, (long long)rounds * STAGES);
+        if (lane == 0) ptx::tma_store_wait_all();
+    } else if (warp < MMA_WARP) {
+        // ------------------------------------------------------------ converters
+        const int cw = warp - CONV_WARP0;
+        const int group = cw / C::GROUP_WARPS;
+        const int gt = (cw % C::GROUP_WARPS) * 32 + lane;                // thread within the group
+        const int row = gt >> 2, piece = gt & 3;                         // piece i of this thread: row + (GROUP_THREADS/4) i
+        constexpr int SRC_STEP = C::GROUP_THREADS * 16;                  // bytes between a thread's consecutive packed pieces
+        constexpr int DST_STEP = (C::GROUP_THREADS / 4) * 128;
+        const uint32_t src_off = gt * 16;
+        const uint32_t dst_off = row * 128 + (((2 * piece) ^ (row & 7)) << 4);   // even codes
+        const uint32_t dst_hi_off = dst_off ^ 16;                                // odd codes: the neighbouring 16-byte chunk
+        const uint32_t leader_ufull = (CG == 2) ? ptx::map_to_cta(bar_ufull, 0) : bar_ufull;
+        const int total_kb = my_tiles * KB;
+        bool alive = true;
+        for (int it = group; it < total_kb && alive; it += C::GROUPS) {
+            const int ps = it % C::PS, us = it % C::US;
+            alive = ptx::mbar_wait_warp(bar_pfull + 8 * ps, (it / C::PS) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_PACKED, lane);
+            if (!alive) break;
+            if (it >= C::US) {
+                alive = ptx::mbar_wait_warp(bar_uempty + 8 * us, ((it / C::US) - 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_EMPTY, lane);
+                if (!alive) break;
+            }
+            const unsigned char *src = smem + C::OFF_PK + ps * C::PK_STAGE + src_off;
+            unsigned char *dst = smem + C::OFF_UP + us * C::UP_STAGE;
+#pragma unroll 1
+            for (int b0 = 0; b0 < C::CHUNKS; b0 += C::BATCH) {
+                uint4 pk[C::BATCH];
+#pragma unroll
+                for (int i = 0; i < C::BATCH; ++i) pk[i] = *reinterpret_cast<const uint4 *>(src + SRC_STEP * (b0 + i));
+#pragma unroll
+                for (int i = 0; i < C::BATCH; ++i) {
+                    const uint4 w = pk[i];
+                    uint4 lo, hi;
+                    lo.x = (w.x << 4) & 0xF0F0F0F0u; hi.x = w.x & 0xF0F0F0F0u;
+                    lo.y = (w.y << 4) & 0xF0F0F0F0u; hi.y = w.y & 0xF0F0F0F0u;
+                    lo.z = (w.z << 4) & 0xF0F0F0F0u; hi.z = w.z & 0xF0F0F0F0u;
+                    lo.w = (w.w << 4) & 0xF0F0F0F0u; hi.w = w.w & 0xF0F0F0F0u;
+                    *reinterpret_cast<uint4 *>(dst + dst_off + DST_STEP * (b0 + i)) = lo;
+                    *reinterpret_cast<uint4 *>(dst + dst_hi_off + DST_STEP * (b0 + i)) = hi;
+                }
+            }
+            ptx::fence_proxy_async_smem();      // my generic-proxy writes -> visible to the tensor core's async proxy
+            __syncwarp();                        // orders the whole warp's reads and writes before the two arrivals
+            if (lane == 0) {
+                ptx::mbar_arrive(bar_pempty + 8 * ps);
+                if (CG == 2) ptx::mbar_arrive_cluster(leader_ufull + 8 * us);
+                else ptx::mbar_arrive(bar_ufull + 8 * us);
+            }
         }
-#endif
     } else if (warp == MMA_WARP) {
-        // ------------------------------------------------------------ MMA issuer (one thread)
-        if (lane == 0) {
-            constexpr uint32_t idesc = ptx::idesc_i8(BM, BN);
+        // ------------------------------------------------------------ MMA issuer (one thread of the leader CTA)
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = ptx::idesc_i8(BM * CG, BN);
             bool alive = true;
-            int g = 0;                                   // K-blocks consumed so far (all tiles)
-            PROF_DECL(p_tempty); PROF_DECL(p_full); PROF_DECL(p_issue);
-            PROF_T0(pt);
+            int us = 0;
+            uint32_t uph = 0;
             for (int t = 0; t < my_tiles && alive; ++t) {
                 const int b = t & 1;
                 if (t >= ACC_BUFS) {
-                    alive = ptx::mbar_wait(bar_tempty + 8 * b, ((t >> 1) - 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_TMEM_FREE);
+                    alive = ptx::mbar_wait_cluster(bar_tempty + 8 * b, ((t >> 1) - 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_TMEM_FREE);
                     if (!alive) break;
                     ptx::tc_fence_after_sync();
                 }
-                PROF_ADD(p_tempty, pt);
                 const uint32_t d_tmem = tmem_base + b * BN;
-                for (int kb = 0; kb < KB; ++kb, ++g) {
-                    const int s = g & (STAGES - 1);
-                    alive = ptx::mbar_wait(bar_full + 8 * s, (g / STAGES) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_FULL);
+                for (int kb = 0; kb < KB; ++kb) {
+                    alive = ptx::mbar_wait_cluster(bar_ufull + 8 * us, uph, s_abort, status, QVGGT_DEV_TIMEOUT_FULL);
                     if (!alive) break;
                     ptx::tc_fence_after_sync();
-                    PROF_ADD(p_full, pt);
-                    const uint32_t a_addr = sbase + s * T::STAGE_BYTES;
+                    const uint32_t a_addr = sbase + C::OFF_UP + us * C::UP_STAGE;
                     const uint64_t a_desc = ptx::smem_desc_k_sw128(a_addr);
-                    const uint64_t b_desc = ptx::smem_desc_k_sw128(a_addr + T::A_BYTES);
+                    const uint64_t b_desc = ptx::smem_desc_k_sw128(a_addr + BM * BK);
 #pragma unroll
                     for (int p = 0; p < BK / 32; ++p) {
                         // advance 32 bytes (one K = 32 slice) inside the swizzled row: +2 in 16-byte units
-                        ptx::mma_i8_ss(d_tmem, a_desc + 2 * p, b_desc + 2 * p, idesc, (kb | p) != 0);
+                        if (CG == 2) ptx::mma_i8_ss_pair(d_tmem, a_desc + 2 * p, b_desc + 2 * p, idesc, (kb | p) != 0);
+                        else ptx::mma_i8_ss(d_tmem, a_desc + 2 * p, b_desc + 2 * p, idesc, (kb | p) != 0);
                     }
-                    ptx::mma_commit(bar_empty + 8 * s);
-                    PROF_ADD(p_issue, pt);
+                    if (CG == 2) ptx::mma_commit_pair(bar_uempty + 8 * us, 3);
+                    else ptx::mma_commit(bar_uempty + 8 * us);
+                    if (++us == C::US) { us = 0; uph ^= 1; }
                 }
-                if (alive) ptx::mma_commit(bar_tfull + 8 * b);
+                if (alive) {
+                    if (CG == 2) ptx::mma_commit_pair(bar_tfull + 8 * b, 3);
+                    else ptx::mma_commit(bar_tfull + 8 * b);
+                }
             }
-#ifdef QVGGT_PROFILE
-            if (blockIdx.x == 0) { PROF_STORE(8, p_tempty); PROF_STORE(9, p_full); PROF_STORE(10, p_issue); }
-#endif
         }
         __syncwarp();
     } else {
-        // ------------------------------------------------------------ epilogue
-        const int et = threadIdx.x - EPI_WARP0 * 32;       // 0..127
-        const int lane_base = 32 * (warp & 3);
-        bool alive = true;
-        PROF_DECL(p_twait); PROF_DECL(p_work);
-        PROF_T0(pt);
-        for (int t = 0; t < my_tiles; ++t) {
-            const int tile = blockIdx.x + t * gridDim.x;
-            const int m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
-            const int b = t & 1;
-            // per-channel scale and bias of this tile's columns (previous tile's readers are past this barrier)
-            asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
-            for (int i = et; i < BN; i += EPI_THREADS) {
-                s_wscale[i] = w_scale[n0 + i];
-                s_bias[i] = bias ? bf16_bits_to_f32(bias[n0 + i]) : 0.0f;
-            }
-            asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
-            const int gm = m0 + lane_base + lane;
-            const bool row_ok = gm < M;
-            const float as = row_ok ? a_scale[gm] : 0.0f;
-            PROF_ADD(p_work, pt);
-            if (alive) alive = ptx::mbar_wait_warp(bar_tfull + 8 * b, (t >> 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM, lane, 32);
-            ptx::tc_fence_after_sync();
-            PROF_ADD(p_twait, pt);
-            if (alive) {
-#pragma unroll 1
-                for (int c = 0; c < BN; c += 32) {
-                    uint32_t raw[32];
-                    ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(lane_base) << 16) + b * BN + c, raw);
-                    ptx::tmem_ld_wait();
-#ifdef QVGGT_PROBE_NO_EPILOGUE_MATH
-                    if (row_ok && raw[0] == 0x7fffffffu) {
-#else
-                    if (row_ok) {
-#endif
-                        uint32_t out[16];
-#pragma unroll
-                        for (int j = 0; j < 32; j += 2) {
-                            const int a0 = static_cast<int>(raw[j]) >> 8, a1 = static_cast<int>(raw[j + 1]) >> 8;
-                            raw[j] = a0; raw[j + 1] = a1;
-                            float z0 = __fmul_rn(static_cast<float>(a0), __fmul_rn(as, s_wscale[c + j]));
-                            float z1 = __fmul_rn(static_cast<float>(a1), __fmul_rn(as, s_wscale[c + j + 1]));
-                            z0 = __fadd_rn(z0, s_bias[c + j]);
-                            z1 = __fadd_rn(z1, s_bias[c + j + 1]);
-                            __nv_bfloat162 p = __floats2bfloat162_rn(z0, z1);
-                            out[j >> 1] = *reinterpret_cast<uint32_t *>(&p);
-                        }
-                        uint4 *dst = reinterpret_cast<uint4 *>(Y + (long long)gm * ldy + n0 + c);
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) dst[q] = make_uint4(out[4 * q], out[4 * q + 1], out[4 * q + 2], out[4 * q + 3]);
-                        if (acc_debug) {
-                            uint4 *dbg = reinterpret_cast<uint4 *>(acc_debug + (long long)gm * N + n0 + c);
-#pragma unroll
-                            for (int q = 0; q < 8; ++q) dbg[q] = make_uint4(raw[4 * q], raw[4 * q + 1], raw[4 * q + 2], raw[4 * q + 3]);
-                        }
+        // ------------------------------------------------------------ TMA producer (one thread)
+        if (lane == 0) {
+            bool alive = true;
+            int ps = 0;
+            uint32_t pph = 0;
+            int it = 0;
+            for (int t = 0; t < my_tiles && alive; ++t) {
+                const int tile = worker + t * workers;
+                const int m0 = (tile / n_tiles) * (BM * CG) + (int)rank * BM;
+                const int n0 = (tile % n_tiles) * BN + (int)rank * C::B_ROWS;
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    if (it >= C::PS) {
+                        alive = ptx::mbar_wait(bar_pempty + 8 * ps, pph ^ 1, s_abort, status, QVGGT_DEV_TIMEOUT_PACKED_FREE, 32);
+                        if (!alive) break;
                     }
+                    const uint32_t dst = sbase + C::OFF_PK + ps * C::PK_STAGE;
+                    ptx::mbar_arrive_expect_tx(bar_pfull + 8 * ps, C::PK_STAGE);
+                    ptx::tma_load_2d(&map_x, bar_pfull + 8 * ps, dst, kb * (BK / 2), m0);
+                    ptx::tma_load_2d(&map_w, bar_pfull + 8 * ps, dst + BM * (BK / 2), kb * (BK / 2), n0);
+                    if (++ps == C::PS) { ps = 0; pph ^= 1; }
                 }
-                ptx::tc_fence_before_sync();
             }
-            __syncwarp();
-            if (alive && lane == 0) ptx::mbar_arrive(bar_tempty + 8 * b);
-            PROF_ADD(p_work, pt);
         }
-#ifdef QVGGT_PROFILE
-        if (blockIdx.x == 0 && et == 0) { PROF_STORE(16, p_twait); PROF_STORE(17, p_work); PROF_STORE(18, my_tiles); }
-#endif
+        __syncwarp();
     }
 
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if (CG == 2) ptx::cluster_sync();        // no remote arrival or multicast commit may target a CTA that has exited
     if (warp == MMA_WARP) {
         ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc(tmem_base, T::TMEM_COLS);
+        if (CG == 2) ptx::tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
+        else ptx::tmem_dealloc(tmem_base, C::TMEM_COLS);
     }
+}
+
+// ------------------------------------------------------------------------------------------------ host side
+using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// 2-D row-major tensor: `inner` elements per row, `rows` rows, `pitch_bytes` between rows.
+bool make_map(CUtensorMap *map, CUtensorMapDataType type, const void *base, uint64_t inner, uint64_t rows,
+              uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swizzle)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {inner, rows};
+    const cuuint64_t strides[1] = {pitch_bytes};
+    const cuuint32_t box[2] = {box_inner, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, type, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 int sm_count()
@@ -340,23 +388,55 @@ int sm_count()
     return sms;
 }
 
-template <int BN>
+template <int CG>
 cudaError_t launch(const qvggt_weights *w, const unsigned char *Xq, const float *a_scale, int M, void *Y, long long ldy,
                    int *acc_debug, cudaStream_t st)
 {
-    using T = Tile<BN>;
-    static bool configured = false;   // per process; one GPU type per process
+    using C = Cfg<CG>;
+    static int max_workers = 0;       // per process; one GPU type per process
     cudaError_t e;
-    if (!configured) {
-        e = cudaFuncSetAttribute(gemm_w4a4_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::DYN_SMEM);
+    if (!max_workers) {
+        e = cudaFuncSetAttribute(gemm_w4a4_kernel<CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::DYN_SMEM);
         if (e != cudaSuccess) return e;
-        configured = true;
+        if (CG == 1) {
+            max_workers = sm_count();
+        } else {
+            cudaLaunchConfig_t probe = {};
+            probe.gridDim = dim3(2 * sm_count());
+            probe.blockDim = dim3(THREADS);
+            probe.dynamicSmemBytes = C::DYN_SMEM;
+            cudaLaunchAttribute a;
+            a.id = cudaLaunchAttributeClusterDimension;
+            a.val.clusterDim.x = CG; a.val.clusterDim.y = 1; a.val.clusterDim.z = 1;
+            probe.attrs = &a;
+            probe.numAttrs = 1;
+            int clusters = 0;
+            e = cudaOccupancyMaxActiveClusters(&clusters, gemm_w4a4_kernel<CG>, &probe);
+            if (e != cudaSuccess) return e;
+            if (clusters < 1) return cudaErrorLaunchOutOfResources;
+            max_workers = clusters;
+        }
     }
-    const int total_tiles = ((M + BM - 1) / BM) * (w->N / BN);
-    const int grid = total_tiles < sm_count() ? total_tiles : sm_count();
-    gemm_w4a4_kernel<BN><<<grid, THREADS, T::DYN_SMEM, st>>>(Xq, w->Wq, a_scale, w->w_scale, w->bias,
-                                                             static_cast<uint16_t *>(Y), ldy, acc_debug, M, w->N, w->K, w->status);
-    return cudaGetLastError();
+    const int K = w->K, N = w->N;
+    CUtensorMap map_x, map_w, map_y;
+    if (!make_map(&map_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, Xq, K / 2, M, K / 2, BK / 2, BM, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !make_map(&map_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, w->Wq, K / 2, N, K / 2, BK / 2, C::B_ROWS, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !make_map(&map_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Y, N, M, (uint64_t)ldy * 2, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B))
+        return cudaErrorInvalidValue;
+    const int total_tiles = ((M + BM * CG - 1) / (BM * CG)) * ((N + BN - 1) / BN);
+    const int workers = total_tiles < max_workers ? total_tiles : max_workers;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(workers * CG);
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = C::DYN_SMEM;
+    cfg.stream = st;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = CG; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_w4a4_kernel<CG>, map_x, map_w, map_y, a_scale, (const float *)w->w_scale,
+                              (const uint16_t *)w->bias, acc_debug, M, N, K, w->status);
 }
 
 }  // namespace
@@ -366,6 +446,9 @@ cudaError_t qvggt_launch_gemm(const qvggt_weights *w, const unsigned char *Xq, c
 {
     if (M == 0) return cudaSuccess;
     if (group != 0) return cudaErrorNotSupported;
-    if (w->N % 256 == 0) return launch<256>(w, Xq, a_scale, M, Y, ldy, acc_debug, st);
-    return launch<128>(w, Xq, a_scale, M, Y, ldy, acc_debug, st);
+#ifdef QVGGT_GEMM_CG1
+    return launch<1>(w, Xq, a_scale, M, Y, ldy, acc_debug, st);
+#else
+    return launch<2>(w, Xq, a_scale, M, Y, ldy, acc_debug, st);
+#endif
 }

@@ -21,7 +21,9 @@ enum : int {
     QVGGT_DEV_TIMEOUT_FULL = 1,    // MMA thread gave up waiting for a converted operand stage
     QVGGT_DEV_TIMEOUT_EMPTY = 2,   // converter gave up waiting for a stage to be released
     QVGGT_DEV_TIMEOUT_ACCUM = 3,   // epilogue gave up waiting for the accumulator
-    QVGGT_DEV_TIMEOUT_TMEM_FREE = 4 // MMA thread gave up waiting for the epilogue to drain TMEM
+    QVGGT_DEV_TIMEOUT_TMEM_FREE = 4, // MMA thread gave up waiting for the epilogue to drain TMEM
+    QVGGT_DEV_TIMEOUT_PACKED = 5,    // converter gave up waiting for a TMA-loaded stage of packed codes
+    QVGGT_DEV_TIMEOUT_PACKED_FREE = 6 // TMA producer gave up waiting for a packed stage to be released
 };
 
 // rsq.cu
