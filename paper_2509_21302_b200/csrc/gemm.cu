@@ -52,8 +52,6 @@ struct Cfg {
     static constexpr int GROUP_WARPS = CONV_WARPS / GROUPS;
     static constexpr int GROUP_THREADS = GROUP_WARPS * 32;
     static constexpr int CHUNKS = ROWS * 4 / GROUP_THREADS;   // 16-byte packed pieces per thread per stage
-    static constexpr int BATCH = (CG == 1) ? 6 : 8;           // pieces held in registers at a time
-    static_assert(CHUNKS % BATCH == 0, "stage must split into whole register batches");
     static constexpr int OFF_UP = 0;                       // operand stages first: they need 1024-byte alignment
     static constexpr int OFF_STG = OFF_UP + US * UP_STAGE;
     static constexpr int OFF_PK = OFF_STG + EPI_WARPS * STG_BYTES;
@@ -238,33 +236,38 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             const int ps = it % C::PS, us = it % C::US;
             alive = ptx::mbar_wait_warp(bar_pfull + 8 * ps, (it / C::PS) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_PACKED, lane);
             if (!alive) break;
+            // the whole share of the stage goes to registers first, so the packed stage is handed back
+            // to the TMA producer before the (longer) conversion starts
+            const unsigned char *src = smem + C::OFF_PK + ps * C::PK_STAGE + src_off;
+            uint4 pk[C::CHUNKS];
+#pragma unroll
+            for (int i = 0; i < C::CHUNKS; ++i) pk[i] = *reinterpret_cast<const uint4 *>(src + SRC_STEP * i);
+            // consume one value of every load: the loads have completed before the stage is released
+            uint32_t seen = 0;
+#pragma unroll
+            for (int i = 0; i < C::CHUNKS; ++i) seen |= pk[i].x;
+            asm volatile("" ::"r"(seen) : "memory");
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar_pempty + 8 * ps);
             if (it >= C::US) {
                 alive = ptx::mbar_wait_warp(bar_uempty + 8 * us, ((it / C::US) - 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_EMPTY, lane);
                 if (!alive) break;
             }
-            const unsigned char *src = smem + C::OFF_PK + ps * C::PK_STAGE + src_off;
             unsigned char *dst = smem + C::OFF_UP + us * C::UP_STAGE;
-#pragma unroll 1
-            for (int b0 = 0; b0 < C::CHUNKS; b0 += C::BATCH) {
-                uint4 pk[C::BATCH];
 #pragma unroll
-                for (int i = 0; i < C::BATCH; ++i) pk[i] = *reinterpret_cast<const uint4 *>(src + SRC_STEP * (b0 + i));
-#pragma unroll
-                for (int i = 0; i < C::BATCH; ++i) {
-                    const uint4 w = pk[i];
-                    uint4 lo, hi;
-                    lo.x = (w.x << 4) & 0xF0F0F0F0u; hi.x = w.x & 0xF0F0F0F0u;
-                    lo.y = (w.y << 4) & 0xF0F0F0F0u; hi.y = w.y & 0xF0F0F0F0u;
-                    lo.z = (w.z << 4) & 0xF0F0F0F0u; hi.z = w.z & 0xF0F0F0F0u;
-                    lo.w = (w.w << 4) & 0xF0F0F0F0u; hi.w = w.w & 0xF0F0F0F0u;
-                    *reinterpret_cast<uint4 *>(dst + dst_off + DST_STEP * (b0 + i)) = lo;
-                    *reinterpret_cast<uint4 *>(dst + dst_hi_off + DST_STEP * (b0 + i)) = hi;
-                }
+            for (int i = 0; i < C::CHUNKS; ++i) {
+                const uint4 w = pk[i];
+                uint4 lo, hi;
+                lo.x = (w.x << 4) & 0xF0F0F0F0u; hi.x = w.x & 0xF0F0F0F0u;
+                lo.y = (w.y << 4) & 0xF0F0F0F0u; hi.y = w.y & 0xF0F0F0F0u;
+                lo.z = (w.z << 4) & 0xF0F0F0F0u; hi.z = w.z & 0xF0F0F0F0u;
+                lo.w = (w.w << 4) & 0xF0F0F0F0u; hi.w = w.w & 0xF0F0F0F0u;
+                *reinterpret_cast<uint4 *>(dst + dst_off + DST_STEP * i) = lo;
+                *reinterpret_cast<uint4 *>(dst + dst_hi_off + DST_STEP * i) = hi;
             }
             ptx::fence_proxy_async_smem();      // my generic-proxy writes -> visible to the tensor core's async proxy
             __syncwarp();                        // orders the whole warp's reads and writes before the two arrivals
             if (lane == 0) {
-                ptx::mbar_arrive(bar_pempty + 8 * ps);
                 if (CG == 2) ptx::mbar_arrive_cluster(leader_ufull + 8 * us);
                 else ptx::mbar_arrive(bar_ufull + 8 * us);
             }
@@ -321,7 +324,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const int n0 = (tile % n_tiles) * BN + (int)rank * C::B_ROWS;
                 for (int kb = 0; kb < KB; ++kb, ++it) {
                     if (it >= C::PS) {
-                        alive = ptx::mbar_wait(bar_pempty + 8 * ps, pph ^ 1, s_abort, status, QVGGT_DEV_TIMEOUT_PACKED_FREE, 32);
+                        alive = ptx::mbar_wait(bar_pempty + 8 * ps, pph ^ 1, s_abort, status, QVGGT_DEV_TIMEOUT_PACKED_FREE);
                         if (!alive) break;
                     }
                     const uint32_t dst = sbase + C::OFF_PK + ps * C::PK_STAGE;
