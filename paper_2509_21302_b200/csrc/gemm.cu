@@ -36,7 +36,7 @@ constexpr int MMA_WARP = EPI_WARPS + CONV_WARPS;
 constexpr int TMA_WARP = MMA_WARP + 1;
 constexpr int THREADS = (TMA_WARP + 1) * 32;
 constexpr int ACC_BUFS = 2;        // TMEM accumulators: the epilogue of tile i overlaps the MMAs of tile i+1
-constexpr int STG_BYTES = 32 * 128;   // per epilogue warp: 32 rows x 64 bf16, 128-byte swizzled
+constexpr int STG_BYTES = 32 * 64;    // per epilogue warp: 32 rows x 32 bf16, 64-byte swizzled
 
 template <int CG>
 struct Cfg {
@@ -48,26 +48,29 @@ struct Cfg {
     static constexpr int US = (CG == 1) ? 2 : 4;           // operand stages (decouple converters and MMA)
     // Converter warps form GROUPS independent groups; group g converts K-blocks g, g + GROUPS, ...  so the
     // fixed costs of a stage (draining the stores, the proxy fence, barrier round trips) overlap.
+#ifdef QVGGT_GROUPS
+    static constexpr int GROUPS = QVGGT_GROUPS;
+#else
     static constexpr int GROUPS = (CG == 1) ? 2 : 4;
+#endif
     static constexpr int GROUP_WARPS = CONV_WARPS / GROUPS;
     static constexpr int GROUP_THREADS = GROUP_WARPS * 32;
     static constexpr int CHUNKS = ROWS * 4 / GROUP_THREADS;   // 16-byte packed pieces per thread per stage
     static constexpr int OFF_UP = 0;                       // operand stages first: they need 1024-byte alignment
     static constexpr int OFF_STG = OFF_UP + US * UP_STAGE;
-    static constexpr int OFF_PK = OFF_STG + EPI_WARPS * STG_BYTES;
+    static constexpr int OFF_CH = OFF_STG + EPI_WARPS * STG_BYTES;   // per-channel scale and bias of two tiles, fp32
+    static constexpr int OFF_PK = OFF_CH + 2 * ACC_BUFS * BN * 4;
     static constexpr int OFF_BAR = OFF_PK + PS * PK_STAGE; // pfull[PS] pempty[PS] ufull[US] uempty[US] tfull[2] tempty[2]
     static constexpr int NBARS = 2 * PS + 2 * US + 2 * ACC_BUFS;
     static constexpr int OFF_TMEM = OFF_BAR + NBARS * 8;
     static constexpr int OFF_ABORT = OFF_TMEM + 4;
-    static constexpr int BYTES = OFF_ABORT + 4;
+    static constexpr int OFF_FLAGS = OFF_ABORT + 4;        // outcome words of the group waits: epilogue, converter groups
+    static constexpr int BYTES = OFF_FLAGS + 8 * (1 + CONV_WARPS);
     static constexpr int DYN_SMEM = BYTES + 1024;          // slack to align the base to 1024 bytes
     static constexpr int TMEM_COLS = ACC_BUFS * BN;        // 512
     static_assert(DYN_SMEM <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
     static_assert(UP_STAGE % 1024 == 0 && (BM * BK) % 1024 == 0, "operand tiles must stay 1024-byte aligned");
 };
-
-__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
 template <int CG>
 __global__ void __launch_bounds__(THREADS, 1)
@@ -88,6 +91,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     const uint32_t bar_tempty = bar_tfull + ACC_BUFS * 8;
     uint32_t *s_tmem = reinterpret_cast<uint32_t *>(smem + C::OFF_TMEM);
     volatile int *s_abort = reinterpret_cast<volatile int *>(smem + C::OFF_ABORT);
+    volatile int *s_flags = reinterpret_cast<volatile int *>(smem + C::OFF_FLAGS);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = (CG == 2) ? ptx::cluster_ctarank() : 0u;     // 0 = leader of the pair
@@ -133,86 +137,95 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         const int quarter = warp & 3, chalf = warp >> 2;   // TMEM lane quarter, column half
         unsigned char *stg = smem + C::OFF_STG + warp * STG_BYTES;
         const uint32_t stg_addr = sbase + C::OFF_STG + warp * STG_BYTES;
+        float *s_ws = reinterpret_cast<float *>(smem + C::OFF_CH);          // [2][BN] per-channel scale of the tile
+        float *s_bs = s_ws + ACC_BUFS * BN;                                   // [2][BN] bias as fp32
         const uint32_t leader_tempty = (CG == 2) ? ptx::map_to_cta(bar_tempty, 0) : bar_tempty;
         bool alive = true;
+        uint32_t toggle = 0;
         for (int t = 0; t < my_tiles; ++t) {
             const int tile = worker + t * workers;
             const int m0 = (tile / n_tiles) * (BM * CG) + (int)rank * BM + quarter * 32;
-            const int n0 = (tile % n_tiles) * BN + chalf * 128;
+            const int nt0 = (tile % n_tiles) * BN;             // first channel of the tile
+            const int n0 = nt0 + chalf * 128;                  // first channel of this warp's half
             const int b = t & 1;
             const int gm = m0 + lane;
             const bool row_ok = gm < M;
             const bool cols_ok = n0 < N;                       // N is a multiple of 128: a half tile is all in or all out
+            // per-channel scale and bias of the tile -> shared memory; buffer b was last read two tiles ago,
+            // and every epilogue warp has passed the group barrier of the tile in between since then
+            {
+                const int e = threadIdx.x;                     // 0..255: one channel each
+                const bool ch_ok = nt0 + e < N;
+                s_ws[b * BN + e] = ch_ok ? __ldg(w_scale + nt0 + e) : 0.0f;
+                s_bs[b * BN + e] = (ch_ok && bias) ? __uint_as_float(static_cast<uint32_t>(__ldg(bias + nt0 + e)) << 16) : 0.0f;
+            }
             // a_scale / 256: exact (power of two), cancels the factor 256 carried by the raw accumulator
             const float as = row_ok ? __fmul_rn(__ldg(a_scale + gm), 0.00390625f) : 0.0f;
-            if (alive) alive = ptx::mbar_wait_warp(bar_tfull + 8 * b, (t >> 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM, lane, 32);
+            const uint64_t as2 = ptx::f32x2_pack(as, as);
+            // one thread polls for all epilogue warps (named barrier 1); the barrier also publishes s_ws / s_bs
+            alive = ptx::mbar_wait_group(bar_tfull + 8 * b, (t >> 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM,
+                                         threadIdx.x == 0, 1, EPI_WARPS * 32, s_flags, toggle, 64) && alive;
             ptx::tc_fence_after_sync();
             if (alive) {
+                const float *wsb = s_ws + b * BN + chalf * 128;
+                const float *bsb = s_bs + b * BN + chalf * 128;
 #pragma unroll 1
-                for (int box = 0; box < 2; ++box) {
-                    // the previous TMA store has finished reading the staging buffer
-                    if (lane == 0) ptx::tma_store_wait_read<0>();
-                    __syncwarp();
-#pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        const int col = box * 64 + c * 32;                // within this warp's 128 columns
-                        uint32_t raw[32];
-                        ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + b * BN + chalf * 128 + col, raw);
-                        ptx::tmem_ld_wait();
-                        if (box == 1 && c == 1) {
-                            // last read of this accumulator: hand it back to the MMA thread before the math
-                            ptx::tc_fence_before_sync();
-                            __syncwarp();
-                            if (lane == 0) {
-                                if (CG == 2) ptx::mbar_arrive_cluster(leader_tempty + 8 * b);
-                                else ptx::mbar_arrive(bar_tempty + 8 * b);
-                            }
-                        }
-                        if (cols_ok) {
-                            const float4 *ws4 = reinterpret_cast<const float4 *>(w_scale + n0 + col);
-                            const uint2 *bs2 = reinterpret_cast<const uint2 *>(bias + n0 + col);
-                            uint32_t out[16];
-#pragma unroll
-                            for (int j = 0; j < 32; j += 4) {
-                                const float4 ws = __ldg(ws4 + (j >> 2));
-                                float2 b01 = make_float2(0.0f, 0.0f), b23 = make_float2(0.0f, 0.0f);
-                                if (bias) {
-                                    const uint2 bb = __ldg(bs2 + (j >> 2));
-                                    b01 = make_float2(bf16_lo(bb.x), bf16_hi(bb.x));
-                                    b23 = make_float2(bf16_lo(bb.y), bf16_hi(bb.y));
-                                }
-                                const float2 t01 = ptx::mul_f32x2(make_float2(as, as), make_float2(ws.x, ws.y));
-                                const float2 t23 = ptx::mul_f32x2(make_float2(as, as), make_float2(ws.z, ws.w));
-                                float2 z01 = make_float2(static_cast<float>(static_cast<int>(raw[j])), static_cast<float>(static_cast<int>(raw[j + 1])));
-                                float2 z23 = make_float2(static_cast<float>(static_cast<int>(raw[j + 2])), static_cast<float>(static_cast<int>(raw[j + 3])));
-                                z01 = ptx::mul_f32x2(z01, t01);
-                                z23 = ptx::mul_f32x2(z23, t23);
-                                if (bias) {
-                                    z01 = ptx::add_f32x2(z01, b01);
-                                    z23 = ptx::add_f32x2(z23, b23);
-                                }
-                                out[j >> 1] = ptx::pack_bf16x2(z01.x, z01.y);
-                                out[(j >> 1) + 1] = ptx::pack_bf16x2(z23.x, z23.y);
-                            }
-                            // row `lane` of the staging tile, 16-byte chunk (4c + q) XOR (lane mod 8)
-#pragma unroll
-                            for (int q = 0; q < 4; ++q)
-                                *reinterpret_cast<uint4 *>(stg + lane * 128 + (((4 * c + q) ^ (lane & 7)) << 4)) =
-                                    make_uint4(out[4 * q], out[4 * q + 1], out[4 * q + 2], out[4 * q + 3]);
-                            if (acc_debug && row_ok) {
-                                uint4 *dbg = reinterpret_cast<uint4 *>(acc_debug + (long long)gm * N + n0 + col);
-#pragma unroll
-                                for (int q = 0; q < 8; ++q)
-                                    dbg[q] = make_uint4(static_cast<int>(raw[4 * q]) >> 8, static_cast<int>(raw[4 * q + 1]) >> 8,
-                                                        static_cast<int>(raw[4 * q + 2]) >> 8, static_cast<int>(raw[4 * q + 3]) >> 8);
-                            }
+                for (int c = 0; c < 4; ++c) {
+                    const int col = c * 32;                               // within this warp's 128 columns
+                    uint32_t raw[32];
+                    ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + b * BN + chalf * 128 + col, raw);
+                    ptx::tmem_ld_wait();
+                    if (c == 3) {
+                        // last read of this accumulator: hand it back to the MMA thread before the math
+                        ptx::tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) {
+                            if (CG == 2) ptx::mbar_arrive_cluster(leader_tempty + 8 * b);
+                            else ptx::mbar_arrive(bar_tempty + 8 * b);
                         }
                     }
-                    ptx::fence_proxy_async_smem();          // staging writes -> visible to the TMA engine
-                    __syncwarp();
-                    if (lane == 0 && cols_ok && m0 < M) {
-                        ptx::tma_store_2d(&map_y, stg_addr, n0 + box * 64, m0);   // rows >= M are clipped by the tensor map
-                        ptx::tma_store_commit();
+                    if (cols_ok) {
+                        uint32_t out[16];
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            const ulonglong2 w2 = *reinterpret_cast<const ulonglong2 *>(wsb + col + j);
+                            const ulonglong2 b2 = *reinterpret_cast<const ulonglong2 *>(bsb + col + j);
+                            uint64_t z01 = ptx::f32x2_pack(static_cast<float>(static_cast<int>(raw[j])), static_cast<float>(static_cast<int>(raw[j + 1])));
+                            uint64_t z23 = ptx::f32x2_pack(static_cast<float>(static_cast<int>(raw[j + 2])), static_cast<float>(static_cast<int>(raw[j + 3])));
+                            // fl(fl(float(acc) * fl(a_scale * w_scale)) + bias), every operation rounded to nearest.
+                            // The additions are scalar intrinsics: a packed multiply feeding a packed add was
+                            // observed to be contracted into one fused operation (single rounding).
+                            z01 = ptx::f32x2_mul(z01, ptx::f32x2_mul(as2, w2.x));
+                            z23 = ptx::f32x2_mul(z23, ptx::f32x2_mul(as2, w2.y));
+                            float y0, y1, y2, y3, c0, c1, c2, c3;
+                            ptx::f32x2_unpack(z01, y0, y1);
+                            ptx::f32x2_unpack(z23, y2, y3);
+                            ptx::f32x2_unpack(b2.x, c0, c1);
+                            ptx::f32x2_unpack(b2.y, c2, c3);
+                            out[j >> 1] = ptx::pack_bf16x2(__fadd_rn(y0, c0), __fadd_rn(y1, c1));
+                            out[(j >> 1) + 1] = ptx::pack_bf16x2(__fadd_rn(y2, c2), __fadd_rn(y3, c3));
+                        }
+                        // the previous TMA store has finished reading the staging buffer
+                        if (lane == 0) ptx::tma_store_wait_read<0>();
+                        __syncwarp();
+                        // row `lane` of the staging tile (64-byte rows, 64-byte swizzle): 16-byte chunk q XOR ((lane / 2) mod 4)
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            *reinterpret_cast<uint4 *>(stg + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4)) =
+                                make_uint4(out[4 * q], out[4 * q + 1], out[4 * q + 2], out[4 * q + 3]);
+                        if (acc_debug && row_ok) {
+                            uint4 *dbg = reinterpret_cast<uint4 *>(acc_debug + (long long)gm * N + n0 + col);
+#pragma unroll
+                            for (int q = 0; q < 8; ++q)
+                                dbg[q] = make_uint4(static_cast<int>(raw[4 * q]) >> 8, static_cast<int>(raw[4 * q + 1]) >> 8,
+                                                    static_cast<int>(raw[4 * q + 2]) >> 8, static_cast<int>(raw[4 * q + 3]) >> 8);
+                        }
+                        ptx::fence_proxy_async_smem();          // staging writes -> visible to the TMA engine
+                        __syncwarp();
+                        if (lane == 0 && m0 < M) {
+                            ptx::tma_store_2d(&map_y, stg_addr, n0 + col, m0);   // rows >= M are clipped by the tensor map
+                            ptx::tma_store_commit();
+                        }
                     }
                 }
             }
@@ -232,9 +245,11 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         const uint32_t leader_ufull = (CG == 2) ? ptx::map_to_cta(bar_ufull, 0) : bar_ufull;
         const int total_kb = my_tiles * KB;
         bool alive = true;
+        uint32_t toggle = 0;
         for (int it = group; it < total_kb && alive; it += C::GROUPS) {
             const int ps = it % C::PS, us = it % C::US;
-            alive = ptx::mbar_wait_warp(bar_pfull + 8 * ps, (it / C::PS) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_PACKED, lane);
+            alive = ptx::mbar_wait_group(bar_pfull + 8 * ps, (it / C::PS) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_PACKED, gt == 0,
+                                         2 + group, C::GROUP_THREADS, s_flags + 2 + 2 * group, toggle, 20);
             if (!alive) break;
             // the whole share of the stage goes to registers first, so the packed stage is handed back
             // to the TMA producer before the (longer) conversion starts
@@ -250,7 +265,8 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(bar_pempty + 8 * ps);
             if (it >= C::US) {
-                alive = ptx::mbar_wait_warp(bar_uempty + 8 * us, ((it / C::US) - 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_EMPTY, lane);
+                alive = ptx::mbar_wait_group(bar_uempty + 8 * us, ((it / C::US) - 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_EMPTY,
+                                             gt == 0, 2 + group, C::GROUP_THREADS, s_flags + 2 + 2 * group, toggle, 20);
                 if (!alive) break;
             }
             unsigned char *dst = smem + C::OFF_UP + us * C::UP_STAGE;
@@ -324,7 +340,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const int n0 = (tile % n_tiles) * BN + (int)rank * C::B_ROWS;
                 for (int kb = 0; kb < KB; ++kb, ++it) {
                     if (it >= C::PS) {
-                        alive = ptx::mbar_wait(bar_pempty + 8 * ps, pph ^ 1, s_abort, status, QVGGT_DEV_TIMEOUT_PACKED_FREE);
+                        alive = ptx::mbar_wait(bar_pempty + 8 * ps, pph ^ 1, s_abort, status, QVGGT_DEV_TIMEOUT_PACKED_FREE, 20);
                         if (!alive) break;
                     }
                     const uint32_t dst = sbase + C::OFF_PK + ps * C::PK_STAGE;
@@ -424,7 +440,7 @@ cudaError_t launch(const qvggt_weights *w, const unsigned char *Xq, const float 
     CUtensorMap map_x, map_w, map_y;
     if (!make_map(&map_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, Xq, K / 2, M, K / 2, BK / 2, BM, CU_TENSOR_MAP_SWIZZLE_NONE) ||
         !make_map(&map_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, w->Wq, K / 2, N, K / 2, BK / 2, C::B_ROWS, CU_TENSOR_MAP_SWIZZLE_NONE) ||
-        !make_map(&map_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Y, N, M, (uint64_t)ldy * 2, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B))
+        !make_map(&map_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Y, N, M, (uint64_t)ldy * 2, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B))
         return cudaErrorInvalidValue;
     const int total_tiles = ((M + BM * CG - 1) / (BM * CG)) * ((N + BN - 1) / BN);
     const int workers = total_tiles < max_workers ? total_tiles : max_workers;

@@ -90,7 +90,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 }
 
 // Same wait, polled by lane 0 only; the other lanes park at the shuffle instead of hammering the
-// barrier (128 spinning epilogue threads measurably slow the converter warps' shared-memory stores).
+// barrier (every poll is a shared-memory operation that competes with the operand traffic).
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
                                                int code, int lane, unsigned sleep_ns = 0)
 {
@@ -99,6 +99,23 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
     ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
     __syncwarp();   // memory ordering between lane 0's acquire and the other lanes' reads
     return ok != 0;
+}
+
+// Same wait for a group of `nthreads` threads (whole warps) that share named barrier `bar_id`:
+// one thread polls, the rest sleep in the hardware barrier.  `leader` is true for exactly one
+// thread of the group; `flags` are two shared-memory words of the group that carry the outcome,
+// used alternately (`toggle` is a per-thread call counter) so that the leader's next result
+// cannot overwrite a word that a slower thread has not read yet.  Every thread of the group must
+// make every call: the outcome is uniform, so they all leave their loop together.
+__device__ __forceinline__ bool mbar_wait_group(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code,
+                                                bool leader, int bar_id, int nthreads, volatile int *flags, uint32_t &toggle,
+                                                unsigned sleep_ns = 0)
+{
+    volatile int *flag = flags + (toggle & 1);
+    ++toggle;
+    if (leader) *flag = mbar_wait(bar, parity, abort_flag, status, code, sleep_ns) ? 1 : 0;
+    asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(nthreads) : "memory");
+    return *flag != 0;
 }
 
 // Generic-proxy shared-memory writes -> visible to the async proxy (tcgen05.mma operand reads).
@@ -375,6 +392,40 @@ __device__ __forceinline__ float2 sub_f32x2(float2 a, float2 b)
         "}\n"
         : "=f"(d.x), "=f"(d.y)
         : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return d;
+}
+
+// The same operations on pairs kept in 64-bit registers (no packing moves around each operation).
+__device__ __forceinline__ uint64_t f32x2_pack(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+
+__device__ __forceinline__ void f32x2_unpack(uint64_t v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+
+__device__ __forceinline__ uint64_t f32x2_mul(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+__device__ __forceinline__ uint64_t f32x2_add(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+__device__ __forceinline__ uint64_t f32x2_sub(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
 
