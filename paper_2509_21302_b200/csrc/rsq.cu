@@ -9,6 +9,7 @@
 //
 // The same kernel serves the activations (multiplier amul) and the weight rows (multiplier wmul).
 #include "qvggt_internal.cuh"
+#include "sm100_ptx.cuh"
 
 namespace {
 
@@ -180,6 +181,174 @@ rsq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float *__
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// K = 1024, one warp per row, 32 values per lane, packed fp32 pairs (two IEEE operations per issue
+// slot).  Element i = e + 8 t + 256 q (e < 8, lane t < 32, q < 4): a lane loads and stores 16-byte
+// pieces that are contiguous across the warp.  The ten stages run in ascending stride in three
+// register phases with two 32 x 32 transposes through shared memory in between:
+//   strides 1, 2, 4        on e   (lane holds p = 8 q + e)
+//   strides 8 .. 128       on t   (lane p holds all 32 values of t)
+//   strides 256, 512       on q   (lane t holds p again)
+// Transpose tiles keep 16-byte chunk c of row r at chunk c XOR (r mod 8): scalar stores of a
+// column and 16-byte loads of a row are both free of bank conflicts.
+
+// (a0, a1) <- (a0 + b0, a1 + b1), (b0, b1) <- (a0 - b0, a1 - b1): two butterflies per instruction pair
+__device__ __forceinline__ void bfly2(float &a0, float &a1, float &b0, float &b1)
+{
+#ifdef RSQ_SCALAR
+    const float x0 = a0, x1 = a1, y0 = b0, y1 = b1;
+    a0 = __fadd_rn(x0, y0); a1 = __fadd_rn(x1, y1); b0 = __fsub_rn(x0, y0); b1 = __fsub_rn(x1, y1);
+#else
+    const uint64_t A = ptx::f32x2_pack(a0, a1), B = ptx::f32x2_pack(b0, b1);
+    ptx::f32x2_unpack(ptx::f32x2_add(A, B), a0, a1);
+    ptx::f32x2_unpack(ptx::f32x2_sub(A, B), b0, b1);
+#endif
+}
+
+constexpr int kFastWarps = 8;
+
+template <int GROUP>
+__global__ void __launch_bounds__(kFastWarps * 32)
+rsq1024_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float *__restrict__ mul,
+               unsigned char *__restrict__ Xq, float *__restrict__ scales)
+{
+    __shared__ __align__(16) float tiles[kFastWarps][1024];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float *S = tiles[warp];
+    // the multipliers of this lane's 32 elements never change: registers
+    float m[32];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const float4 lo = __ldg(reinterpret_cast<const float4 *>(mul + 256 * q + 8 * lane));
+        const float4 hi = __ldg(reinterpret_cast<const float4 *>(mul + 256 * q + 8 * lane + 4));
+        m[8 * q + 0] = lo.x; m[8 * q + 1] = lo.y; m[8 * q + 2] = lo.z; m[8 * q + 3] = lo.w;
+        m[8 * q + 4] = hi.x; m[8 * q + 5] = hi.y; m[8 * q + 6] = hi.z; m[8 * q + 7] = hi.w;
+    }
+    const long long stride = (long long)gridDim.x * kFastWarps;
+    long long row = (long long)blockIdx.x * kFastWarps + warp;
+    uint4 nx[4];
+    if (row < M) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) nx[q] = __ldg(reinterpret_cast<const uint4 *>(X + row * ldx + 256 * q + 8 * lane));
+    }
+    for (; row < M; row += stride) {
+        float r[32];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t w[4] = {nx[q].x, nx[q].y, nx[q].z, nx[q].w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                r[8 * q + 2 * j] = __uint_as_float(w[j] << 16);
+                r[8 * q + 2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+            }
+        }
+        const long long next = row + stride;
+        if (next < M) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) nx[q] = __ldg(reinterpret_cast<const uint4 *>(X + next * ldx + 256 * q + 8 * lane));
+        }
+        // ---- strides 1, 2, 4 (bits of e); pairs run across q (p, p + 8)
+#pragma unroll
+        for (int h = 1; h < 8; h <<= 1)
+#pragma unroll
+            for (int qp = 0; qp < 32; qp += 16)
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                    if (!(e & h)) bfly2(r[qp + e], r[qp + 8 + e], r[qp + e + h], r[qp + 8 + e + h]);
+        // ---- transpose: lane t writes column t of row p; lane p reads row p
+#pragma unroll
+        for (int p = 0; p < 32; ++p) S[p * 32 + ((((lane >> 2) ^ (p & 7)) << 2) | (lane & 3))] = r[p];
+        __syncwarp();
+        float v[32];
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+            const float4 f = *reinterpret_cast<const float4 *>(S + lane * 32 + ((g ^ (lane & 7)) << 2));
+            v[4 * g] = f.x; v[4 * g + 1] = f.y; v[4 * g + 2] = f.z; v[4 * g + 3] = f.w;
+        }
+        __syncwarp();
+        // ---- strides 8 .. 128 (bits of t).  Stride 8 joins neighbours of a pair: scalar; the rest pairs (t, t + 1)
+#pragma unroll
+        for (int t = 0; t < 32; t += 2) {
+            const float a = v[t], b = v[t + 1];
+            v[t] = __fadd_rn(a, b);
+            v[t + 1] = __fsub_rn(a, b);
+        }
+#pragma unroll
+        for (int h = 2; h < 32; h <<= 1)
+#pragma unroll
+            for (int t = 0; t < 32; t += 2)
+                if (!(t & h)) bfly2(v[t], v[t + 1], v[t + h], v[t + 1 + h]);
+        // ---- transpose back: lane p writes column p of row t; lane t reads row t
+#pragma unroll
+        for (int t = 0; t < 32; ++t) S[t * 32 + ((((lane >> 2) ^ (t & 7)) << 2) | (lane & 3))] = v[t];
+        __syncwarp();
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+            const float4 f = *reinterpret_cast<const float4 *>(S + lane * 32 + ((g ^ (lane & 7)) << 2));
+            r[4 * g] = f.x; r[4 * g + 1] = f.y; r[4 * g + 2] = f.z; r[4 * g + 3] = f.w;
+        }
+        __syncwarp();
+        // ---- strides 256, 512 (bits of q); pairs run across e (e, e + 1)
+#pragma unroll
+        for (int h = 8; h < 32; h <<= 1)
+#pragma unroll
+            for (int p = 0; p < 32; p += 2)
+                if (!(p & h)) bfly2(r[p], r[p + 1], r[p + h], r[p + 1 + h]);
+        // ---- smoothing multiplier, absolute maximum, 4-bit codes
+#pragma unroll
+        for (int p = 0; p < 32; p += 2) {
+            const uint64_t y = ptx::f32x2_mul(ptx::f32x2_pack(r[p], r[p + 1]), ptx::f32x2_pack(m[p], m[p + 1]));
+            ptx::f32x2_unpack(y, r[p], r[p + 1]);
+        }
+        float amax[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            float a = 0.0f;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) a = fmaxf(a, fabsf(r[8 * q + e]));
+            amax[q] = a;
+        }
+        if (GROUP == 128) {
+            // group of element i is i / 128 = 2 q + (lane / 16): reduce over each half warp
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) amax[q] = fmaxf(amax[q], __shfl_xor_sync(0xFFFFFFFFu, amax[q], o));
+        } else {
+            float a = fmaxf(fmaxf(amax[0], amax[1]), fmaxf(amax[2], amax[3]));
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, o));
+            amax[0] = amax[1] = amax[2] = amax[3] = a;
+        }
+        uint32_t word[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const float am = fmaxf(amax[q], 1e-8f);
+            const float inv = __fdiv_rn(7.0f, am);
+            amax[q] = am;
+            uint32_t wv = 0;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                // exact product + 1.5*2^23, rounded once (half-to-even): low mantissa bits = two's-complement code
+                const float f = __fmaf_rn(r[8 * q + e], inv, 12582912.0f);
+                wv = __funnelshift_r(wv, __float_as_uint(f), 4);       // shift in the low nibble from the top
+            }
+            word[q] = wv;
+        }
+        unsigned char *dst = Xq + row * 512 + 4 * lane;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) *reinterpret_cast<uint32_t *>(dst + 128 * q) = word[q];
+        if (GROUP == 128) {
+            if ((lane & 15) == 0) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) scales[row * 8 + 2 * q + (lane >> 4)] = __fdiv_rn(amax[q], 7.0f);
+            }
+        } else {
+            if (lane == 0) scales[row] = __fdiv_rn(amax[0], 7.0f);
+        }
+    }
+}
+
 // Column-wise absolute maximum of the normalised rotated rows (calibration statistics for Eq. "smooth_factor").
 template <int K>
 __global__ void __launch_bounds__(kThreads)
@@ -259,9 +428,9 @@ cudaError_t qvggt_launch_rsq(const void *X, long long ldx, int M, int K, const f
     if (M == 0) return cudaSuccess;
     const uint16_t *x = static_cast<const uint16_t *>(X);
     if (K == 1024) {
-        int grid = rsq_grid(M, RowGeom<1024>::ROWS);
-        if (group == 128) rsq_kernel<1024, 128><<<grid, kThreads, 0, st>>>(x, ldx, M, mul, Xq, scales);
-        else rsq_kernel<1024, 0><<<grid, kThreads, 0, st>>>(x, ldx, M, mul, Xq, scales);
+        int grid = rsq_grid(M, kFastWarps);
+        if (group == 128) rsq1024_kernel<128><<<grid, kFastWarps * 32, 0, st>>>(x, ldx, M, mul, Xq, scales);
+        else rsq1024_kernel<0><<<grid, kFastWarps * 32, 0, st>>>(x, ldx, M, mul, Xq, scales);
     } else {
         int grid = rsq_grid(M, RowGeom<4096>::ROWS);
         if (group == 128) rsq_kernel<4096, 128><<<grid, kThreads, 0, st>>>(x, ldx, M, mul, Xq, scales);
