@@ -120,231 +120,202 @@ __device__ __forceinline__ void rotate_row_to_smem(const uint16_t *x, const floa
     }
 }
 
-template <int K, int GROUP>
-__global__ void __launch_bounds__(kThreads)
-rsq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float *__restrict__ mul,
-           unsigned char *__restrict__ Xq, float *__restrict__ scales)
-{
-    using G = RowGeom<K>;
-    __shared__ float smem[G::ROWS * G::PADDED];
-    __shared__ float red[G::ROWS][4];
-    const int slot = threadIdx.x / G::T;
-    const int t = threadIdx.x % G::T;
-    float *s = smem + slot * G::PADDED;
-
-    for (long long m0 = (long long)blockIdx.x * G::ROWS; m0 < M; m0 += (long long)gridDim.x * G::ROWS) {
-        const long long m = m0 + slot;
-        if (m < M) {
-            rotate_row_to_smem<K>(X + m * ldx, mul, s, t, slot);
-            float y[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) y[j] = s[padded(t * 32 + j)];
-            float amax = 0.0f;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) amax = fmaxf(amax, fabsf(y[j]));
-            if (GROUP == 128) {
-                amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
-                amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
-            } else {
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
-                if (G::T > 32) {
-                    if ((t & 31) == 0) red[slot][t >> 5] = amax;
-                    row_sync(G::T, slot);
-                    amax = fmaxf(fmaxf(red[slot][0], red[slot][1]), fmaxf(red[slot][2], red[slot][3]));
-                }
-            }
-            amax = fmaxf(amax, 1e-8f);
-            const float scale = __fdiv_rn(amax, 7.0f);
-            const float inv = __fdiv_rn(7.0f, amax);
-            uint32_t packed[4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                uint32_t word = 0;
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    // exact product + 1.5*2^23, rounded once (half-to-even): low mantissa bits = two's-complement code
-                    float f = __fmaf_rn(y[q * 8 + e], inv, 12582912.0f);
-                    word |= (__float_as_uint(f) & 0xFu) << (4 * e);
-                }
-                packed[q] = word;
-            }
-            *reinterpret_cast<uint4 *>(Xq + m * (K / 2) + t * 16) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-            if (GROUP == 128) {
-                if ((t & 3) == 0) scales[m * (K / 128) + (t >> 2)] = scale;
-            } else {
-                if (t == 0) scales[m] = scale;
-            }
-        }
-        // the row's shared memory is reused by the next pass
-        if (G::T == 32) __syncwarp(); else __syncthreads();
-    }
-}
-
-// ------------------------------------------------------------------------------------------------
-// K = 1024, one warp per row, 32 values per lane, packed fp32 pairs (two IEEE operations per issue
-// slot).  Element i = e + 8 t + 256 q (e < 8, lane t < 32, q < 4): a lane loads and stores 16-byte
-// pieces that are contiguous across the warp.  The ten stages run in ascending stride in three
-// register phases with two 32 x 32 transposes through shared memory in between:
-//   strides 1, 2, 4        on e   (lane holds p = 8 q + e)
-//   strides 8 .. 128       on t   (lane p holds all 32 values of t)
-//   strides 256, 512       on q   (lane t holds p again)
-// Transpose tiles keep 16-byte chunk c of row r at chunk c XOR (r mod 8): scalar stores of a
-// column and 16-byte loads of a row are both free of bank conflicts.
-
 // (a0, a1) <- (a0 + b0, a1 + b1), (b0, b1) <- (a0 - b0, a1 - b1): two butterflies per instruction pair
 __device__ __forceinline__ void bfly2(float &a0, float &a1, float &b0, float &b1)
 {
-#ifdef RSQ_SCALAR
-    const float x0 = a0, x1 = a1, y0 = b0, y1 = b1;
-    a0 = __fadd_rn(x0, y0); a1 = __fadd_rn(x1, y1); b0 = __fsub_rn(x0, y0); b1 = __fsub_rn(x1, y1);
-#else
     const uint64_t A = ptx::f32x2_pack(a0, a1), B = ptx::f32x2_pack(b0, b1);
     ptx::f32x2_unpack(ptx::f32x2_add(A, B), a0, a1);
     ptx::f32x2_unpack(ptx::f32x2_sub(A, B), b0, b1);
-#endif
 }
 
-constexpr int kFastWarps = 8;
-
-template <int GROUP>
-__global__ void __launch_bounds__(kFastWarps * 32)
-rsq1024_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float *__restrict__ mul,
-               unsigned char *__restrict__ Xq, float *__restrict__ scales)
+// ------------------------------------------------------------------------------------------------
+// K = T * T (T = 32: one warp per row; T = 64: two warps per row), T values per thread, a single
+// transpose.  The bf16 row is staged in shared memory with 16-byte asynchronous copies (coalesced
+// in global memory, double-buffered), so that thread t can start from the T contiguous elements
+// T t .. T t + T - 1:
+//   strides 1 .. T/2      in registers (element T t + j, bits of j)
+//   T x T transpose through shared memory (16-byte chunk c of row r kept at chunk c XOR (r mod 8))
+//   strides T .. T*T/2    in registers (thread t' holds elements T t + t', bits of t)
+// The codes of thread t' then belong to elements T t + t': eight neighbouring lanes exchange
+// nibbles with three shuffle steps so that every lane ends up with whole 32-bit output words.
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
 {
-    __shared__ __align__(16) float tiles[kFastWarps][1024];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    float *S = tiles[warp];
-    // the multipliers of this lane's 32 elements never change: registers
-    float m[32];
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ptx::smem_addr(smem_dst)), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+template <int LOGT>
+struct SqGeom {
+    static constexpr int T = 1 << LOGT;              // threads per row = values per thread
+    static constexpr int K = T * T;
+    static constexpr int CTA_THREADS = 128;
+    static constexpr int ROWS = CTA_THREADS / T;     // rows in flight per CTA
+    static constexpr int CH = T / 8;                 // 16-byte pieces of bf16 per thread
+    static constexpr int STAGE_BYTES = 2 * K;        // one bf16 row
+    static constexpr int ROW_SMEM = 2 * STAGE_BYTES + 4 * K + 256;  // two stages, fp32 transpose tile, 2 x 32 reduction words
+    static constexpr int SMEM = ROWS * ROW_SMEM;
+};
+
+template <int T>
+__device__ __forceinline__ void group_sync(int slot)
+{
+    if (T == 32) __syncwarp();
+    else asm volatile("bar.sync %0, %1;" ::"r"(slot + 1), "r"(T) : "memory");
+}
+
+// In-register stages over n values: the first joins neighbours (scalar), the others pair (k, k + 1).
+template <int N>
+__device__ __forceinline__ void stages_in_registers(float (&v)[N])
+{
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        const float4 lo = __ldg(reinterpret_cast<const float4 *>(mul + 256 * q + 8 * lane));
-        const float4 hi = __ldg(reinterpret_cast<const float4 *>(mul + 256 * q + 8 * lane + 4));
-        m[8 * q + 0] = lo.x; m[8 * q + 1] = lo.y; m[8 * q + 2] = lo.z; m[8 * q + 3] = lo.w;
-        m[8 * q + 4] = hi.x; m[8 * q + 5] = hi.y; m[8 * q + 6] = hi.z; m[8 * q + 7] = hi.w;
+    for (int k = 0; k < N; k += 2) {
+        const float a = v[k], b = v[k + 1];
+        v[k] = __fadd_rn(a, b);
+        v[k + 1] = __fsub_rn(a, b);
     }
-    const long long stride = (long long)gridDim.x * kFastWarps;
-    long long row = (long long)blockIdx.x * kFastWarps + warp;
-    uint4 nx[4];
+#pragma unroll
+    for (int h = 2; h < N; h <<= 1)
+#pragma unroll
+        for (int k = 0; k < N; k += 2)
+            if (!(k & h)) bfly2(v[k], v[k + 1], v[k + h], v[k + 1 + h]);
+}
+
+template <int LOGT, int GROUP>
+__global__ void __launch_bounds__(SqGeom<LOGT>::CTA_THREADS, LOGT == 5 ? 4 : 3)
+rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float *__restrict__ mul,
+              unsigned char *__restrict__ Xq, float *__restrict__ scales)
+{
+    using G = SqGeom<LOGT>;
+    constexpr int T = G::T, K = G::K, CH = G::CH;
+    constexpr int NG = (GROUP == 128) ? K / 128 : 1;           // scale groups per row
+    constexpr int GREGS = (GROUP == 128) ? 128 / T : T;        // consecutive registers of one thread in the same group
+    extern __shared__ __align__(16) unsigned char dsm[];
+    const int slot = threadIdx.x / T, t = threadIdx.x % T, lane = threadIdx.x & 31;
+    unsigned char *stage = dsm + slot * G::ROW_SMEM;
+    float *Tm = reinterpret_cast<float *>(stage + 2 * G::STAGE_BYTES);
+    float *red = Tm + K;                                       // cross-warp maxima (T = 64 only)
+
+    float m[T];                                                // multipliers of elements T k + t
+#pragma unroll
+    for (int k = 0; k < T; ++k) m[k] = __ldg(mul + T * k + t);
+
+    // staging copy: 16-byte piece cg = t + T j belongs to thread cg / CH, piece cg % CH of its T values
+    uint32_t cp_dst[CH];
+#pragma unroll
+    for (int j = 0; j < CH; ++j) {
+        const int cg = t + T * j, to = cg / CH, c = cg % CH;
+        const int sw = (T == 32) ? ((to >> 1) & 3) : (to & 7);
+        cp_dst[j] = to * (2 * T) + ((c ^ sw) << 4);
+    }
+    const int my_sw = (T == 32) ? ((t >> 1) & 3) : (t & 7);
+    // nibble exchange between the 8 lanes that share (t / 8): per step d the lane keeps half of its nibbles
+    uint32_t nb_send[3], nb_keep[3], nb_rot[3];
+#pragma unroll
+    for (int i = 0; i < 3; ++i) {
+        const uint32_t m0 = (i == 0) ? 0x0F0F0F0Fu : (i == 1) ? 0x00FF00FFu : 0x0000FFFFu;   // nibble index bit clear
+        const bool up = (lane >> i) & 1;
+        nb_send[i] = up ? m0 : ~m0;
+        nb_keep[i] = up ? ~m0 : m0;
+        nb_rot[i] = up ? (4u << i) : 32u - (4u << i);
+    }
+
+    const long long stride = (long long)gridDim.x * G::ROWS;
+    long long row = (long long)blockIdx.x * G::ROWS + slot;
     if (row < M) {
+        const unsigned char *src = reinterpret_cast<const unsigned char *>(X + row * ldx);
 #pragma unroll
-        for (int q = 0; q < 4; ++q) nx[q] = __ldg(reinterpret_cast<const uint4 *>(X + row * ldx + 256 * q + 8 * lane));
+        for (int j = 0; j < CH; ++j) cp_async16(stage + cp_dst[j], src + 16 * (t + T * j));
     }
-    for (; row < M; row += stride) {
-        float r[32];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const uint32_t w[4] = {nx[q].x, nx[q].y, nx[q].z, nx[q].w};
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                r[8 * q + 2 * j] = __uint_as_float(w[j] << 16);
-                r[8 * q + 2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
-            }
-        }
+    cp_async_commit();
+    int buf = 0;
+    for (; row < M; row += stride, buf ^= 1) {
         const long long next = row + stride;
         if (next < M) {
+            const unsigned char *src = reinterpret_cast<const unsigned char *>(X + next * ldx);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) nx[q] = __ldg(reinterpret_cast<const uint4 *>(X + next * ldx + 256 * q + 8 * lane));
+            for (int j = 0; j < CH; ++j) cp_async16(stage + (buf ^ 1) * G::STAGE_BYTES + cp_dst[j], src + 16 * (t + T * j));
         }
-        // ---- strides 1, 2, 4 (bits of e); pairs run across q (p, p + 8)
+        cp_async_commit();
+        cp_async_wait<1>();                 // this row's copies (mine) have landed; the barrier covers the others'
+        group_sync<T>(slot);
+        float v[T];
+        {
+            const unsigned char *mine = stage + buf * G::STAGE_BYTES + t * (2 * T);
 #pragma unroll
-        for (int h = 1; h < 8; h <<= 1)
+            for (int c = 0; c < CH; ++c) {
+                const uint4 w4 = *reinterpret_cast<const uint4 *>(mine + ((c ^ my_sw) << 4));
+                const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
-            for (int qp = 0; qp < 32; qp += 16)
+                for (int j = 0; j < 4; ++j) {
+                    v[8 * c + 2 * j] = __uint_as_float(w[j] << 16);
+                    v[8 * c + 2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+                }
+            }
+        }
+        stages_in_registers<T>(v);          // strides 1 .. T/2
 #pragma unroll
-                for (int e = 0; e < 8; ++e)
-                    if (!(e & h)) bfly2(r[qp + e], r[qp + 8 + e], r[qp + e + h], r[qp + 8 + e + h]);
-        // ---- transpose: lane t writes column t of row p; lane p reads row p
+        for (int j = 0; j < T; ++j) Tm[j * T + ((((t >> 2) ^ (j & 7)) << 2) | (t & 3))] = v[j];
+        group_sync<T>(slot);
 #pragma unroll
-        for (int p = 0; p < 32; ++p) S[p * 32 + ((((lane >> 2) ^ (p & 7)) << 2) | (lane & 3))] = r[p];
-        __syncwarp();
-        float v[32];
-#pragma unroll
-        for (int g = 0; g < 8; ++g) {
-            const float4 f = *reinterpret_cast<const float4 *>(S + lane * 32 + ((g ^ (lane & 7)) << 2));
+        for (int g = 0; g < T / 4; ++g) {
+            const float4 f = *reinterpret_cast<const float4 *>(Tm + t * T + ((g ^ (t & 7)) << 2));
             v[4 * g] = f.x; v[4 * g + 1] = f.y; v[4 * g + 2] = f.z; v[4 * g + 3] = f.w;
         }
-        __syncwarp();
-        // ---- strides 8 .. 128 (bits of t).  Stride 8 joins neighbours of a pair: scalar; the rest pairs (t, t + 1)
+        stages_in_registers<T>(v);          // strides T .. K/2: v[k] is element T k + t
 #pragma unroll
-        for (int t = 0; t < 32; t += 2) {
-            const float a = v[t], b = v[t + 1];
-            v[t] = __fadd_rn(a, b);
-            v[t + 1] = __fsub_rn(a, b);
+        for (int k = 0; k < T; k += 2) {
+            const uint64_t y = ptx::f32x2_mul(ptx::f32x2_pack(v[k], v[k + 1]), ptx::f32x2_pack(m[k], m[k + 1]));
+            ptx::f32x2_unpack(y, v[k], v[k + 1]);
         }
+        // absolute maxima: one per row, or one per 128 consecutive elements (GREGS registers of every thread)
+        float am[NG];
 #pragma unroll
-        for (int h = 2; h < 32; h <<= 1)
-#pragma unroll
-            for (int t = 0; t < 32; t += 2)
-                if (!(t & h)) bfly2(v[t], v[t + 1], v[t + h], v[t + 1 + h]);
-        // ---- transpose back: lane p writes column p of row t; lane t reads row t
-#pragma unroll
-        for (int t = 0; t < 32; ++t) S[t * 32 + ((((lane >> 2) ^ (t & 7)) << 2) | (lane & 3))] = v[t];
-        __syncwarp();
-#pragma unroll
-        for (int g = 0; g < 8; ++g) {
-            const float4 f = *reinterpret_cast<const float4 *>(S + lane * 32 + ((g ^ (lane & 7)) << 2));
-            r[4 * g] = f.x; r[4 * g + 1] = f.y; r[4 * g + 2] = f.z; r[4 * g + 3] = f.w;
-        }
-        __syncwarp();
-        // ---- strides 256, 512 (bits of q); pairs run across e (e, e + 1)
-#pragma unroll
-        for (int h = 8; h < 32; h <<= 1)
-#pragma unroll
-            for (int p = 0; p < 32; p += 2)
-                if (!(p & h)) bfly2(r[p], r[p + 1], r[p + h], r[p + 1 + h]);
-        // ---- smoothing multiplier, absolute maximum, 4-bit codes
-#pragma unroll
-        for (int p = 0; p < 32; p += 2) {
-            const uint64_t y = ptx::f32x2_mul(ptx::f32x2_pack(r[p], r[p + 1]), ptx::f32x2_pack(m[p], m[p + 1]));
-            ptx::f32x2_unpack(y, r[p], r[p + 1]);
-        }
-        float amax[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        for (int g = 0; g < NG; ++g) {
             float a = 0.0f;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) a = fmaxf(a, fabsf(r[8 * q + e]));
-            amax[q] = a;
-        }
-        if (GROUP == 128) {
-            // group of element i is i / 128 = 2 q + (lane / 16): reduce over each half warp
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-#pragma unroll
-                for (int o = 8; o > 0; o >>= 1) amax[q] = fmaxf(amax[q], __shfl_xor_sync(0xFFFFFFFFu, amax[q], o));
-        } else {
-            float a = fmaxf(fmaxf(amax[0], amax[1]), fmaxf(amax[2], amax[3]));
+            for (int k = 0; k < GREGS; ++k) a = fmaxf(a, fabsf(v[g * GREGS + k]));
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, o));
-            amax[0] = amax[1] = amax[2] = amax[3] = a;
+            am[g] = a;
         }
-        uint32_t word[4];
+        if (T == 64) {
+            if (lane == 0) {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const float am = fmaxf(amax[q], 1e-8f);
-            const float inv = __fdiv_rn(7.0f, am);
-            amax[q] = am;
-            uint32_t wv = 0;
+                for (int g = 0; g < NG; ++g) red[(t >> 5) * NG + g] = am[g];
+            }
+            group_sync<T>(slot);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
+            for (int g = 0; g < NG; ++g) am[g] = fmaxf(red[g], red[NG + g]);
+        }
+        uint32_t word[T / 8];
+#pragma unroll
+        for (int g = 0; g < NG; ++g) {
+            am[g] = fmaxf(am[g], 1e-8f);
+            const float inv = __fdiv_rn(7.0f, am[g]);
+#pragma unroll
+            for (int k = g * GREGS; k < (g + 1) * GREGS; ++k) {
                 // exact product + 1.5*2^23, rounded once (half-to-even): low mantissa bits = two's-complement code
-                const float f = __fmaf_rn(r[8 * q + e], inv, 12582912.0f);
-                wv = __funnelshift_r(wv, __float_as_uint(f), 4);       // shift in the low nibble from the top
+                const float f = __fmaf_rn(v[k], inv, 12582912.0f);
+                word[k >> 3] = __funnelshift_r((k & 7) ? word[k >> 3] : 0u, __float_as_uint(f), 4);
             }
-            word[q] = wv;
         }
-        unsigned char *dst = Xq + row * 512 + 4 * lane;
+        // word[kk] holds the codes of elements T (8 kk + n) + t in nibble n; after the exchange it holds the
+        // codes of elements T (8 kk + e) + 8 (t / 8) + n, e = t mod 8: one whole output word
 #pragma unroll
-        for (int q = 0; q < 4; ++q) *reinterpret_cast<uint32_t *>(dst + 128 * q) = word[q];
-        if (GROUP == 128) {
-            if ((lane & 15) == 0) {
+        for (int kk = 0; kk < T / 8; ++kk) {
+            uint32_t x = word[kk];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) scales[row * 8 + 2 * q + (lane >> 4)] = __fdiv_rn(amax[q], 7.0f);
+            for (int i = 0; i < 3; ++i) {
+                const uint32_t send = __funnelshift_l(x & nb_send[i], x & nb_send[i], nb_rot[i]);
+                x = (x & nb_keep[i]) | __shfl_xor_sync(0xFFFFFFFFu, send, 1 << i);
             }
-        } else {
-            if (lane == 0) scales[row] = __fdiv_rn(amax[0], 7.0f);
+            *reinterpret_cast<uint32_t *>(Xq + row * (K / 2) + 4 * ((T / 8) * (8 * kk + (t & 7)) + (t >> 3))) = x;
+        }
+        if (t == 0) {
+#pragma unroll
+            for (int g = 0; g < NG; ++g) scales[row * NG + g] = __fdiv_rn(am[g], 7.0f);
         }
     }
 }
@@ -403,13 +374,13 @@ __global__ void smooth_finalize_kernel(const float *__restrict__ ax, const float
     c[k] = r;
 }
 
-int rsq_grid(int M, int rows_per_cta)
+int rsq_grid(int M, int rows_per_cta, int ctas_per_sm = 6)
 {
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     long long need = ((long long)M + rows_per_cta - 1) / rows_per_cta;
-    long long cap = (long long)sms * 6;
+    long long cap = (long long)sms * ctas_per_sm;
     return (int)(need < cap ? need : cap);
 }
 
@@ -427,14 +398,23 @@ cudaError_t qvggt_launch_rsq(const void *X, long long ldx, int M, int K, const f
 {
     if (M == 0) return cudaSuccess;
     const uint16_t *x = static_cast<const uint16_t *>(X);
+    static bool configured = false;       // per process
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(rsq_sq_kernel<6, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SqGeom<6>::SMEM);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(rsq_sq_kernel<6, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, SqGeom<6>::SMEM);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
     if (K == 1024) {
-        int grid = rsq_grid(M, kFastWarps);
-        if (group == 128) rsq1024_kernel<128><<<grid, kFastWarps * 32, 0, st>>>(x, ldx, M, mul, Xq, scales);
-        else rsq1024_kernel<0><<<grid, kFastWarps * 32, 0, st>>>(x, ldx, M, mul, Xq, scales);
+        using G = SqGeom<5>;
+        const int grid = rsq_grid(M, G::ROWS, 4);
+        if (group == 128) rsq_sq_kernel<5, 128><<<grid, G::CTA_THREADS, G::SMEM, st>>>(x, ldx, M, mul, Xq, scales);
+        else rsq_sq_kernel<5, 0><<<grid, G::CTA_THREADS, G::SMEM, st>>>(x, ldx, M, mul, Xq, scales);
     } else {
-        int grid = rsq_grid(M, RowGeom<4096>::ROWS);
-        if (group == 128) rsq_kernel<4096, 128><<<grid, kThreads, 0, st>>>(x, ldx, M, mul, Xq, scales);
-        else rsq_kernel<4096, 0><<<grid, kThreads, 0, st>>>(x, ldx, M, mul, Xq, scales);
+        using G = SqGeom<6>;
+        const int grid = rsq_grid(M, G::ROWS, 3);
+        if (group == 128) rsq_sq_kernel<6, 128><<<grid, G::CTA_THREADS, G::SMEM, st>>>(x, ldx, M, mul, Xq, scales);
+        else rsq_sq_kernel<6, 0><<<grid, G::CTA_THREADS, G::SMEM, st>>>(x, ldx, M, mul, Xq, scales);
     }
     return cudaGetLastError();
 }
