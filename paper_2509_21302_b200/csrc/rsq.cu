@@ -165,7 +165,8 @@ __device__ __forceinline__ void group_sync(int slot)
     else asm volatile("bar.sync %0, %1;" ::"r"(slot + 1), "r"(T) : "memory");
 }
 
-// In-register stages over n values: the first joins neighbours (scalar), the others pair (k, k + 1).
+// In-register stages over n values: the first joins neighbours (scalar: packing it costs more register
+// moves than it saves), the others pair (k, k + 1).
 template <int N>
 __device__ __forceinline__ void stages_in_registers(float (&v)[N])
 {
@@ -273,9 +274,9 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
         float am[NG];
 #pragma unroll
         for (int g = 0; g < NG; ++g) {
-            float a = 0.0f;
+            float a = fmaxf(fabsf(v[g * GREGS]), fabsf(v[g * GREGS + 1]));
 #pragma unroll
-            for (int k = 0; k < GREGS; ++k) a = fmaxf(a, fabsf(v[g * GREGS + k]));
+            for (int k = 2; k < GREGS; k += 2) a = fmaxf(fmaxf(a, fabsf(v[g * GREGS + k])), fabsf(v[g * GREGS + k + 1]));
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, o));
             am[g] = a;
@@ -295,10 +296,15 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
             am[g] = fmaxf(am[g], 1e-8f);
             const float inv = __fdiv_rn(7.0f, am[g]);
 #pragma unroll
-            for (int k = g * GREGS; k < (g + 1) * GREGS; ++k) {
+            const uint64_t inv2 = ptx::f32x2_pack(inv, inv), magic2 = ptx::f32x2_pack(12582912.0f, 12582912.0f);
+#pragma unroll
+            for (int k = g * GREGS; k < (g + 1) * GREGS; k += 2) {
                 // exact product + 1.5*2^23, rounded once (half-to-even): low mantissa bits = two's-complement code
-                const float f = __fmaf_rn(v[k], inv, 12582912.0f);
-                word[k >> 3] = __funnelshift_r((k & 7) ? word[k >> 3] : 0u, __float_as_uint(f), 4);
+                float f0, f1;
+                ptx::f32x2_unpack(ptx::f32x2_fma(ptx::f32x2_pack(v[k], v[k + 1]), inv2, magic2), f0, f1);
+                uint32_t w = (k & 7) ? word[k >> 3] : 0u;
+                w = __funnelshift_r(w, __float_as_uint(f0), 4);        // shift the low nibble in from the top
+                word[k >> 3] = __funnelshift_r(w, __float_as_uint(f1), 4);
             }
         }
         // word[kk] holds the codes of elements T (8 kk + n) + t in nibble n; after the exchange it holds the

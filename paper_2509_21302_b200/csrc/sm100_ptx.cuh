@@ -429,6 +429,14 @@ __device__ __forceinline__ uint64_t f32x2_sub(uint64_t a, uint64_t b)
     return d;
 }
 
+// d = a * b + c on both halves, each rounded once (an explicit fused operation, where the arithmetic asks for one)
+__device__ __forceinline__ uint64_t f32x2_fma(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
 // two fp32 -> packed bf16 pair, round-to-nearest-even; `lo` lands in bits 0-15
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
