@@ -23,6 +23,7 @@
 
 #include "qvggt_internal.cuh"
 #include "sm100_ptx.cuh"
+#include "tensor_map.cuh"
 
 namespace {
 
@@ -65,7 +66,7 @@ struct Cfg {
     static constexpr int OFF_TMEM = OFF_BAR + NBARS * 8;
     static constexpr int OFF_ABORT = OFF_TMEM + 4;
     static constexpr int OFF_FLAGS = OFF_ABORT + 4;        // outcome words of the group waits: epilogue, converter groups
-    static constexpr int BYTES = OFF_FLAGS + 8 * (1 + CONV_WARPS);
+    static constexpr int BYTES = OFF_FLAGS + 8 * (2 + CONV_WARPS);
     static constexpr int DYN_SMEM = BYTES + 1024;          // slack to align the base to 1024 bytes
     static constexpr int TMEM_COLS = ACC_BUFS * BN;        // 512
     static_assert(DYN_SMEM <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
@@ -261,7 +262,9 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             uint32_t seen = 0;
 #pragma unroll
             for (int i = 0; i < C::CHUNKS; ++i) seen |= pk[i].x;
-            asm volatile("" ::"r"(seen) : "memory");
+            // a real (if never taken) use of every loaded value: the loads must have returned before
+            // this branch resolves, hence before the arrival below lets the TMA overwrite the stage
+            if (seen == 0x9E3779B9u) s_flags[1 + 2 * CONV_WARPS] = 1;
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(bar_pempty + 8 * ps);
             if (it >= C::US) {
@@ -364,49 +367,6 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     }
 }
 
-// ------------------------------------------------------------------------------------------------ host side
-using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = [] {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess)
-            p = nullptr;
-        return reinterpret_cast<EncodeTiledFn>(p);
-    }();
-    return fn;
-}
-
-// 2-D row-major tensor: `inner` elements per row, `rows` rows, `pitch_bytes` between rows.
-bool make_map(CUtensorMap *map, CUtensorMapDataType type, const void *base, uint64_t inner, uint64_t rows,
-              uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swizzle)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[2] = {inner, rows};
-    const cuuint64_t strides[1] = {pitch_bytes};
-    const cuuint32_t box[2] = {box_inner, box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(map, type, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-int sm_count()
-{
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    }
-    return sms;
-}
-
 template <int CG>
 cudaError_t launch(const qvggt_weights *w, const unsigned char *Xq, const float *a_scale, int M, void *Y, long long ldy,
                    int *acc_debug, cudaStream_t st)
@@ -418,10 +378,10 @@ cudaError_t launch(const qvggt_weights *w, const unsigned char *Xq, const float 
         e = cudaFuncSetAttribute(gemm_w4a4_kernel<CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::DYN_SMEM);
         if (e != cudaSuccess) return e;
         if (CG == 1) {
-            max_workers = sm_count();
+            max_workers = qvggt_sm_count();
         } else {
             cudaLaunchConfig_t probe = {};
-            probe.gridDim = dim3(2 * sm_count());
+            probe.gridDim = dim3(2 * qvggt_sm_count());
             probe.blockDim = dim3(THREADS);
             probe.dynamicSmemBytes = C::DYN_SMEM;
             cudaLaunchAttribute a;
@@ -438,9 +398,9 @@ cudaError_t launch(const qvggt_weights *w, const unsigned char *Xq, const float 
     }
     const int K = w->K, N = w->N;
     CUtensorMap map_x, map_w, map_y;
-    if (!make_map(&map_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, Xq, K / 2, M, K / 2, BK / 2, BM, CU_TENSOR_MAP_SWIZZLE_NONE) ||
-        !make_map(&map_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, w->Wq, K / 2, N, K / 2, BK / 2, C::B_ROWS, CU_TENSOR_MAP_SWIZZLE_NONE) ||
-        !make_map(&map_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Y, N, M, (uint64_t)ldy * 2, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+    if (!qvggt_make_map(&map_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, Xq, K / 2, M, K / 2, BK / 2, BM, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !qvggt_make_map(&map_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, w->Wq, K / 2, N, K / 2, BK / 2, C::B_ROWS, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !qvggt_make_map(&map_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Y, N, M, (uint64_t)ldy * 2, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B))
         return cudaErrorInvalidValue;
     const int total_tiles = ((M + BM * CG - 1) / (BM * CG)) * ((N + BN - 1) / BN);
     const int workers = total_tiles < max_workers ? total_tiles : max_workers;
@@ -464,6 +424,7 @@ cudaError_t qvggt_launch_gemm(const qvggt_weights *w, const unsigned char *Xq, c
                               void *Y, long long ldy, int *acc_debug, cudaStream_t st)
 {
     if (M == 0) return cudaSuccess;
+    if (group == 128) return qvggt_launch_gemm_grouped(w, Xq, a_scale, M, Y, ldy, acc_debug, st);
     if (group != 0) return cudaErrorNotSupported;
 #ifdef QVGGT_GEMM_CG1
     return launch<1>(w, Xq, a_scale, M, Y, ldy, acc_debug, st);

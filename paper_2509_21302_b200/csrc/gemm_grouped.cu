@@ -1,0 +1,328 @@
+// W4A4 GEMM with one activation scale per token per 128 consecutive rotated channels (an extension of
+// the paper's token-wise granularity; the weights keep one scale per output channel).  Because the
+// scale changes along the inner dimension, the integer sum of every 128-wide K-group is rescaled on
+// its own before it joins the fp32 running sum:
+//   Y[m][n] = bf16( (sum_g float(acc_g[m][n]) * a_scale[m][g]) * w_scale[n] + bias[n] ),  g ascending.
+//
+// Same building blocks as the token-wise kernel (TMA-staged packed codes, converter warps, int8
+// tcgen05.mma with the codes in the high nibble, bounded waits), with these differences:
+//   - one CTA per tile of 128 tokens x 128 channels (tcgen05.mma.cta_group::1, M = 128, N = 128);
+//   - every K-block of 128 codes is one scale group: it accumulates into its own TMEM buffer (two
+//     buffers of 128 columns, ping-pong), which the epilogue warps drain while the next group runs;
+//   - an epilogue thread keeps the running sums of its row's 64 columns in registers.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "qvggt_internal.cuh"
+#include "sm100_ptx.cuh"
+#include "tensor_map.cuh"
+
+namespace {
+
+constexpr int BM = 128, BN = 128, BK = 128;
+constexpr int EPI_WARPS = 8;       // warp w: TMEM lanes 32*(w%4).., columns 64*(w/4)..
+constexpr int CONV_WARPS = 8;
+constexpr int CONV_WARP0 = EPI_WARPS;
+constexpr int MMA_WARP = EPI_WARPS + CONV_WARPS;
+constexpr int TMA_WARP = MMA_WARP + 1;
+constexpr int THREADS = (TMA_WARP + 1) * 32;
+constexpr int ACC_BUFS = 2;
+constexpr int STG_BYTES = 32 * 64;             // per epilogue warp: 32 rows x 32 bf16, 64-byte swizzled
+constexpr int ROWS = BM + BN;                  // packed / operand rows per stage: tokens, then channels
+constexpr int PK_STAGE = ROWS * (BK / 2);
+constexpr int UP_STAGE = ROWS * BK;
+constexpr int PS = 4, US = 4;
+constexpr int GROUPS = 4;                      // converter groups, as in the token-wise kernel
+constexpr int GROUP_WARPS = CONV_WARPS / GROUPS;
+constexpr int GROUP_THREADS = GROUP_WARPS * 32;
+constexpr int CHUNKS = ROWS * 4 / GROUP_THREADS;
+constexpr int OFF_UP = 0;
+constexpr int OFF_STG = OFF_UP + US * UP_STAGE;
+constexpr int OFF_CH = OFF_STG + EPI_WARPS * STG_BYTES;      // [2][BN] channel scales, [2][BN] bias, fp32
+constexpr int OFF_PK = OFF_CH + 2 * 2 * BN * 4;
+constexpr int OFF_BAR = OFF_PK + PS * PK_STAGE;              // pfull[PS] pempty[PS] ufull[US] uempty[US] tfull[2] tempty[2]
+constexpr int NBARS = 2 * PS + 2 * US + 2 * ACC_BUFS;
+constexpr int OFF_TMEM = OFF_BAR + NBARS * 8;
+constexpr int OFF_ABORT = OFF_TMEM + 4;
+constexpr int OFF_FLAGS = OFF_ABORT + 4;
+constexpr int SMEM_BYTES = OFF_FLAGS + 8 * (2 + CONV_WARPS);
+constexpr int DYN_SMEM = SMEM_BYTES + 1024;
+constexpr int TMEM_COLS = ACC_BUFS * BN;                     // 256
+static_assert(DYN_SMEM <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
+
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_w4a4_grouped_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                         const __grid_constant__ CUtensorMap map_y, const float *__restrict__ a_scale,
+                         const float *__restrict__ w_scale, const uint16_t *__restrict__ bias, int *__restrict__ acc_debug,
+                         int M, int N, int K, int *status)
+{
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = ptx::smem_addr(smem);
+    const uint32_t bar_pfull = sbase + OFF_BAR;
+    const uint32_t bar_pempty = bar_pfull + PS * 8;
+    const uint32_t bar_ufull = bar_pempty + PS * 8;
+    const uint32_t bar_uempty = bar_ufull + US * 8;
+    const uint32_t bar_tfull = bar_uempty + US * 8;
+    const uint32_t bar_tempty = bar_tfull + ACC_BUFS * 8;
+    uint32_t *s_tmem = reinterpret_cast<uint32_t *>(smem + OFF_TMEM);
+    volatile int *s_abort = reinterpret_cast<volatile int *>(smem + OFF_ABORT);
+    volatile int *s_flags = reinterpret_cast<volatile int *>(smem + OFF_FLAGS);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int worker = blockIdx.x, workers = gridDim.x;
+    const int KB = K / BK;                                    // = number of scale groups
+    const int n_tiles = N / BN;
+    const int total_tiles = ((M + BM - 1) / BM) * n_tiles;
+    const int my_tiles = (total_tiles > worker) ? (total_tiles - 1 - worker) / workers + 1 : 0;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < PS; ++s) {
+            ptx::mbar_init(bar_pfull + 8 * s, 1);
+            ptx::mbar_init(bar_pempty + 8 * s, GROUP_WARPS);
+        }
+        for (int s = 0; s < US; ++s) {
+            ptx::mbar_init(bar_ufull + 8 * s, GROUP_WARPS);
+            ptx::mbar_init(bar_uempty + 8 * s, 1);
+        }
+        for (int b = 0; b < ACC_BUFS; ++b) {
+            ptx::mbar_init(bar_tfull + 8 * b, 1);
+            ptx::mbar_init(bar_tempty + 8 * b, EPI_WARPS);
+        }
+        *s_abort = 0;
+        ptx::fence_mbar_init();
+    }
+    if (warp == MMA_WARP) {
+        ptx::tmem_alloc(ptx::smem_addr(s_tmem), TMEM_COLS);
+        ptx::tmem_relinquish();
+    }
+    if (warp == TMA_WARP && lane == 0) {
+        ptx::prefetch_tensormap(&map_x);
+        ptx::prefetch_tensormap(&map_w);
+        ptx::prefetch_tensormap(&map_y);
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *s_tmem;
+
+    if (warp < EPI_WARPS) {
+        // ------------------------------------------------------------ epilogue
+        const int quarter = warp & 3, chalf = warp >> 2;   // TMEM lane quarter, column half (64 columns)
+        unsigned char *stg = smem + OFF_STG + warp * STG_BYTES;
+        const uint32_t stg_addr = sbase + OFF_STG + warp * STG_BYTES;
+        float *s_ws = reinterpret_cast<float *>(smem + OFF_CH);    // [2][BN]
+        float *s_bs = s_ws + 2 * BN;                                // [2][BN]
+        bool alive = true;
+        uint32_t toggle = 0;
+        int it = 0;                                                 // K-blocks seen so far (all tiles)
+        for (int t = 0; t < my_tiles; ++t) {
+            const int tile = worker + t * workers;
+            const int m0 = (tile / n_tiles) * BM + quarter * 32;
+            const int nt0 = (tile % n_tiles) * BN;
+            const int n0 = nt0 + chalf * 64;
+            const int tb = t & 1;
+            const int gm = m0 + lane;
+            const bool row_ok = gm < M;
+            if (threadIdx.x < BN) {
+                // buffer tb was last read two tiles ago; every epilogue warp has passed a group barrier since
+                const int e = threadIdx.x;
+                s_ws[tb * BN + e] = __ldg(w_scale + nt0 + e);
+                s_bs[tb * BN + e] = bias ? __uint_as_float(static_cast<uint32_t>(__ldg(bias + nt0 + e)) << 16) : 0.0f;
+            }
+            float sum[64];
+#pragma unroll
+            for (int j = 0; j < 64; ++j) sum[j] = 0.0f;
+#pragma unroll 1
+            for (int kb = 0; kb < KB; ++kb, ++it) {
+                const int b = it & 1;
+                // a_scale / 256: exact, cancels the factor 256 carried by the raw accumulator
+                const float as = row_ok ? __fmul_rn(__ldg(a_scale + (long long)gm * KB + kb), 0.00390625f) : 0.0f;
+                alive = ptx::mbar_wait_group(bar_tfull + 8 * b, (it >> 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM,
+                                             threadIdx.x == 0, 1, EPI_WARPS * 32, s_flags, toggle, 20) && alive;
+                ptx::tc_fence_after_sync();
+                if (alive) {
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t raw[32];
+                        ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + b * BN + chalf * 64 + c * 32, raw);
+                        ptx::tmem_ld_wait();
+                        if (c == 1) {
+                            ptx::tc_fence_before_sync();
+                            __syncwarp();
+                            if (lane == 0) ptx::mbar_arrive(bar_tempty + 8 * b);
+                        }
+                        // s = fl(s + fl(float(acc_g) * a_scale[m][g])): separate multiply and add
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            sum[32 * c + j] = __fadd_rn(sum[32 * c + j], __fmul_rn(static_cast<float>(static_cast<int>(raw[j])), as));
+                        if (acc_debug && row_ok) {
+                            uint4 *dbg = reinterpret_cast<uint4 *>(acc_debug + ((long long)kb * M + gm) * N + n0 + c * 32);
+#pragma unroll
+                            for (int q = 0; q < 8; ++q)
+                                dbg[q] = make_uint4(static_cast<int>(raw[4 * q]) >> 8, static_cast<int>(raw[4 * q + 1]) >> 8,
+                                                    static_cast<int>(raw[4 * q + 2]) >> 8, static_cast<int>(raw[4 * q + 3]) >> 8);
+                        }
+                    }
+                }
+            }
+            if (alive) {
+                const float *wsb = s_ws + tb * BN + chalf * 64;
+                const float *bsb = s_bs + tb * BN + chalf * 64;
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t out[16];
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        const float z0 = __fadd_rn(__fmul_rn(sum[32 * c + j], wsb[32 * c + j]), bsb[32 * c + j]);
+                        const float z1 = __fadd_rn(__fmul_rn(sum[32 * c + j + 1], wsb[32 * c + j + 1]), bsb[32 * c + j + 1]);
+                        out[j >> 1] = ptx::pack_bf16x2(z0, z1);
+                    }
+                    if (lane == 0) ptx::tma_store_wait_read<0>();      // the previous store has read the staging tile
+                    __syncwarp();
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        *reinterpret_cast<uint4 *>(stg + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4)) =
+                            make_uint4(out[4 * q], out[4 * q + 1], out[4 * q + 2], out[4 * q + 3]);
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0 && m0 < M) {
+                        ptx::tma_store_2d(&map_y, stg_addr, n0 + c * 32, m0);     // rows >= M are clipped by the tensor map
+                        ptx::tma_store_commit();
+                    }
+                }
+            }
+        }
+        if (lane == 0) ptx::tma_store_wait_all();
+    } else if (warp < MMA_WARP) {
+        // ------------------------------------------------------------ converters (see the token-wise kernel)
+        const int cw = warp - CONV_WARP0;
+        const int group = cw / GROUP_WARPS;
+        const int gt = (cw % GROUP_WARPS) * 32 + lane;
+        const int row = gt >> 2, piece = gt & 3;
+        constexpr int SRC_STEP = GROUP_THREADS * 16;
+        constexpr int DST_STEP = (GROUP_THREADS / 4) * 128;
+        const uint32_t src_off = gt * 16;
+        const uint32_t dst_off = row * 128 + (((2 * piece) ^ (row & 7)) << 4);   // even codes
+        const uint32_t dst_hi_off = dst_off ^ 16;                                // odd codes
+        const int total_kb = my_tiles * KB;
+        bool alive = true;
+        uint32_t toggle = 0;
+        for (int it = group; it < total_kb && alive; it += GROUPS) {
+            const int ps = it % PS, us = it % US;
+            alive = ptx::mbar_wait_group(bar_pfull + 8 * ps, (it / PS) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_PACKED, gt == 0,
+                                         2 + group, GROUP_THREADS, s_flags + 2 + 2 * group, toggle, 20);
+            if (!alive) break;
+            const unsigned char *src = smem + OFF_PK + ps * PK_STAGE + src_off;
+            uint4 pk[CHUNKS];
+#pragma unroll
+            for (int i = 0; i < CHUNKS; ++i) pk[i] = *reinterpret_cast<const uint4 *>(src + SRC_STEP * i);
+            uint32_t seen = 0;
+#pragma unroll
+            for (int i = 0; i < CHUNKS; ++i) seen |= pk[i].x;
+            // a real (if never taken) use of every loaded value: the loads must have returned before
+            // this branch resolves, hence before the arrival below lets the TMA overwrite the stage
+            if (seen == 0x9E3779B9u) s_flags[1 + 2 * CONV_WARPS] = 1;
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar_pempty + 8 * ps);
+            if (it >= US) {
+                alive = ptx::mbar_wait_group(bar_uempty + 8 * us, ((it / US) - 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_EMPTY,
+                                             gt == 0, 2 + group, GROUP_THREADS, s_flags + 2 + 2 * group, toggle, 20);
+                if (!alive) break;
+            }
+            unsigned char *dst = smem + OFF_UP + us * UP_STAGE;
+#pragma unroll
+            for (int i = 0; i < CHUNKS; ++i) {
+                const uint4 w = pk[i];
+                uint4 lo, hi;
+                lo.x = (w.x << 4) & 0xF0F0F0F0u; hi.x = w.x & 0xF0F0F0F0u;
+                lo.y = (w.y << 4) & 0xF0F0F0F0u; hi.y = w.y & 0xF0F0F0F0u;
+                lo.z = (w.z << 4) & 0xF0F0F0F0u; hi.z = w.z & 0xF0F0F0F0u;
+                lo.w = (w.w << 4) & 0xF0F0F0F0u; hi.w = w.w & 0xF0F0F0F0u;
+                *reinterpret_cast<uint4 *>(dst + dst_off + DST_STEP * i) = lo;
+                *reinterpret_cast<uint4 *>(dst + dst_hi_off + DST_STEP * i) = hi;
+            }
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar_ufull + 8 * us);
+        }
+    } else if (warp == MMA_WARP) {
+        // ------------------------------------------------------------ MMA issuer: one accumulator per K-block
+        if (lane == 0) {
+            constexpr uint32_t idesc = ptx::idesc_i8(BM, BN);
+            bool alive = true;
+            const int total_kb = my_tiles * KB;
+            for (int it = 0; it < total_kb && alive; ++it) {
+                const int b = it & 1, us = it % US;
+                if (it >= ACC_BUFS) {
+                    alive = ptx::mbar_wait(bar_tempty + 8 * b, ((it >> 1) - 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_TMEM_FREE);
+                    if (!alive) break;
+                }
+                alive = ptx::mbar_wait(bar_ufull + 8 * us, (it / US) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_FULL);
+                if (!alive) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t a_addr = sbase + OFF_UP + us * UP_STAGE;
+                const uint64_t a_desc = ptx::smem_desc_k_sw128(a_addr);
+                const uint64_t b_desc = ptx::smem_desc_k_sw128(a_addr + BM * BK);
+#pragma unroll
+                for (int p = 0; p < BK / 32; ++p) ptx::mma_i8_ss(tmem_base + b * BN, a_desc + 2 * p, b_desc + 2 * p, idesc, p != 0);
+                ptx::mma_commit(bar_uempty + 8 * us);
+                ptx::mma_commit(bar_tfull + 8 * b);
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            bool alive = true;
+            int it = 0;
+            for (int t = 0; t < my_tiles && alive; ++t) {
+                const int tile = worker + t * workers;
+                const int m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    const int ps = it % PS;
+                    if (it >= PS) {
+                        alive = ptx::mbar_wait(bar_pempty + 8 * ps, ((it / PS) - 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_PACKED_FREE, 20);
+                        if (!alive) break;
+                    }
+                    const uint32_t dst = sbase + OFF_PK + ps * PK_STAGE;
+                    ptx::mbar_arrive_expect_tx(bar_pfull + 8 * ps, PK_STAGE);
+                    ptx::tma_load_2d(&map_x, bar_pfull + 8 * ps, dst, kb * (BK / 2), m0);
+                    ptx::tma_load_2d(&map_w, bar_pfull + 8 * ps, dst + BM * (BK / 2), kb * (BK / 2), n0);
+                }
+            }
+        }
+        __syncwarp();
+    }
+
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == MMA_WARP) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace
+
+cudaError_t qvggt_launch_gemm_grouped(const qvggt_weights *w, const unsigned char *Xq, const float *a_scale, int M, void *Y,
+                                      long long ldy, int *acc_debug, cudaStream_t st)
+{
+    static bool configured = false;       // per process
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_w4a4_grouped_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DYN_SMEM);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    const int K = w->K, N = w->N;
+    CUtensorMap map_x, map_w, map_y;
+    if (!qvggt_make_map(&map_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, Xq, K / 2, M, K / 2, BK / 2, BM, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !qvggt_make_map(&map_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, w->Wq, K / 2, N, K / 2, BK / 2, BN, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !qvggt_make_map(&map_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Y, N, M, (uint64_t)ldy * 2, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+        return cudaErrorInvalidValue;
+    const int total_tiles = ((M + BM - 1) / BM) * (N / BN);
+    const int grid = total_tiles < qvggt_sm_count() ? total_tiles : qvggt_sm_count();
+    gemm_w4a4_grouped_kernel<<<grid, THREADS, DYN_SMEM, st>>>(map_x, map_w, map_y, a_scale, w->w_scale, w->bias, acc_debug, M, N,
+                                                              K, w->status);
+    return cudaGetLastError();
+}

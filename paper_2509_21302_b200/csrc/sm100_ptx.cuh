@@ -115,7 +115,13 @@ __device__ __forceinline__ bool mbar_wait_group(uint32_t bar, uint32_t parity, v
     ++toggle;
     if (leader) *flag = mbar_wait(bar, parity, abort_flag, status, code, sleep_ns) ? 1 : 0;
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(nthreads) : "memory");
-    return *flag != 0;
+    const bool ok = *flag != 0;
+    // Every thread observes the completed phase itself (it cannot advance again before this group has
+    // consumed it): what the phase publishes through the async proxy (TMA data, tensor-core results) is
+    // only guaranteed visible to threads that performed the wait, not to threads released by the barrier.
+    if (ok && !leader)
+        for (int i = 0; i < 4096 && !mbar_try_wait(bar, parity); ++i) {}
+    return ok;
 }
 
 // Generic-proxy shared-memory writes -> visible to the async proxy (tcgen05.mma operand reads).

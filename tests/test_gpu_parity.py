@@ -163,6 +163,24 @@ def test_w4a4_linear_parity(K, N, M):
     assert frac == 0.0, f"{frac:.3e} of the outputs differ in the last bit (allowed, but unexpected)"
 
 
+@pytest.mark.parametrize("K,N,M", [(1024, 128, 1), (1024, 384, 257), (4096, 256, 300), (1024, 1024, 1374)])
+def test_w4a4_linear_group128_parity(K, N, M):
+    """One activation scale per token per 128 rotated channels: per-group integer sums bit-exact,
+    outputs against the oracle's ascending-group fp32 accumulation."""
+    spec = workload.LinearSpec("gg", K, N, workload.DIST_GELU if K == 4096 else workload.DIST_NORMAL, 11, 1)
+    L = make_layer(spec, use_signs=(N == 256))
+    X = spec.x_rows(0, M)
+    ref = oracle.w4a4_linear(X, L["prep"], L["b"], 128)
+    Xq, a_scale = q.rotate_smooth_quantize(L["h"], dev_bf16(X), 128)
+    assert np.array_equal(a_scale.cpu().numpy(), ref["a_scale"])
+    acc = torch.full((K // 128, M, N), -123456, dtype=torch.int32, device="cuda")
+    Y = q.w4a4_linear(L["h"], Xq, a_scale, 128, acc_debug=acc)
+    assert L["h"].device_status() == 0
+    assert np.array_equal(acc.cpu().numpy(), ref["acc"])               # per-group int32 sums bit-exact
+    frac = assert_bf16_within_one_ulp(host_bits(Y), ref["y"])
+    assert frac == 0.0, f"{frac:.3e} of the outputs differ in the last bit (allowed, but unexpected)"
+
+
 def test_w4a4_linear_extreme_codes():
     """Codes of magnitude 7 everywhere: the sums reach +-49 K, the largest possible; plus a zero token."""
     K, N, M = 4096, 128, 130
