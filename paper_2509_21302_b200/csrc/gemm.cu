@@ -73,7 +73,9 @@ struct Cfg {
     static_assert(UP_STAGE % 1024 == 0 && (BM * BK) % 1024 == 0, "operand tiles must stay 1024-byte aligned");
 };
 
-template <int CG>
+// DUMP: also write the int32 sums to acc_debug (a separate instantiation keeps that code, and the registers it
+// pins, out of the production kernel)
+template <int CG, bool DUMP>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                  const __grid_constant__ CUtensorMap map_y, const float *__restrict__ a_scale,
@@ -214,7 +216,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                         for (int q = 0; q < 4; ++q)
                             *reinterpret_cast<uint4 *>(stg + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4)) =
                                 make_uint4(out[4 * q], out[4 * q + 1], out[4 * q + 2], out[4 * q + 3]);
-                        if (acc_debug && row_ok) {
+                        if (DUMP && acc_debug && row_ok) {
                             uint4 *dbg = reinterpret_cast<uint4 *>(acc_debug + (long long)gm * N + n0 + col);
 #pragma unroll
                             for (int q = 0; q < 8; ++q)
@@ -367,7 +369,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     }
 }
 
-template <int CG>
+template <int CG, bool DUMP>
 cudaError_t launch(const qvggt_weights *w, const unsigned char *Xq, const float *a_scale, int M, void *Y, long long ldy,
                    int *acc_debug, cudaStream_t st)
 {
@@ -375,7 +377,7 @@ cudaError_t launch(const qvggt_weights *w, const unsigned char *Xq, const float 
     static int max_workers = 0;       // per process; one GPU type per process
     cudaError_t e;
     if (!max_workers) {
-        e = cudaFuncSetAttribute(gemm_w4a4_kernel<CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::DYN_SMEM);
+        e = cudaFuncSetAttribute(gemm_w4a4_kernel<CG, DUMP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::DYN_SMEM);
         if (e != cudaSuccess) return e;
         if (CG == 1) {
             max_workers = qvggt_sm_count();
@@ -390,7 +392,7 @@ cudaError_t launch(const qvggt_weights *w, const unsigned char *Xq, const float 
             probe.attrs = &a;
             probe.numAttrs = 1;
             int clusters = 0;
-            e = cudaOccupancyMaxActiveClusters(&clusters, gemm_w4a4_kernel<CG>, &probe);
+            e = cudaOccupancyMaxActiveClusters(&clusters, gemm_w4a4_kernel<CG, DUMP>, &probe);
             if (e != cudaSuccess) return e;
             if (clusters < 1) return cudaErrorLaunchOutOfResources;
             max_workers = clusters;
@@ -414,7 +416,7 @@ cudaError_t launch(const qvggt_weights *w, const unsigned char *Xq, const float 
     attr.val.clusterDim.x = CG; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_w4a4_kernel<CG>, map_x, map_w, map_y, a_scale, (const float *)w->w_scale,
+    return cudaLaunchKernelEx(&cfg, gemm_w4a4_kernel<CG, DUMP>, map_x, map_w, map_y, a_scale, (const float *)w->w_scale,
                               (const uint16_t *)w->bias, acc_debug, M, N, K, w->status);
 }
 
@@ -427,8 +429,8 @@ cudaError_t qvggt_launch_gemm(const qvggt_weights *w, const unsigned char *Xq, c
     if (group == 128) return qvggt_launch_gemm_grouped(w, Xq, a_scale, M, Y, ldy, acc_debug, st);
     if (group != 0) return cudaErrorNotSupported;
 #ifdef QVGGT_GEMM_CG1
-    return launch<1>(w, Xq, a_scale, M, Y, ldy, acc_debug, st);
+    return acc_debug ? launch<1, true>(w, Xq, a_scale, M, Y, ldy, acc_debug, st) : launch<1, false>(w, Xq, a_scale, M, Y, ldy, acc_debug, st);
 #else
-    return launch<2>(w, Xq, a_scale, M, Y, ldy, acc_debug, st);
+    return acc_debug ? launch<2, true>(w, Xq, a_scale, M, Y, ldy, acc_debug, st) : launch<2, false>(w, Xq, a_scale, M, Y, ldy, acc_debug, st);
 #endif
 }
