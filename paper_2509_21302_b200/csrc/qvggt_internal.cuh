@@ -42,3 +42,4 @@ cudaError_t qvggt_launch_gemm(const qvggt_weights *w, const unsigned char *Xq, c
 // gemm_grouped.cu (group = 128: one activation scale per token per 128 rotated channels)
 cudaError_t qvggt_launch_gemm_grouped(const qvggt_weights *w, const unsigned char *Xq, const float *a_scale, int M, void *Y,
                                       long long ldy, int *acc_debug, cudaStream_t st);
+

@@ -116,11 +116,12 @@ __device__ __forceinline__ bool mbar_wait_group(uint32_t bar, uint32_t parity, v
     if (leader) *flag = mbar_wait(bar, parity, abort_flag, status, code, sleep_ns) ? 1 : 0;
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(nthreads) : "memory");
     const bool ok = *flag != 0;
-    // Every thread observes the completed phase itself (it cannot advance again before this group has
-    // consumed it): what the phase publishes through the async proxy (TMA data, tensor-core results) is
-    // only guaranteed visible to threads that performed the wait, not to threads released by the barrier.
-    if (ok && !leader)
+    // One thread of every warp observes the completed phase itself (it cannot advance again before this
+    // group has consumed it) and orders the rest of its warp behind it: what the phase publishes through
+    // the async proxy (TMA data, tensor-core results) is tied to the wait, not to the hardware barrier.
+    if (ok && !leader && (threadIdx.x & 31) == 0)
         for (int i = 0; i < 4096 && !mbar_try_wait(bar, parity); ++i) {}
+    __syncwarp();
     return ok;
 }
 
