@@ -51,6 +51,27 @@ def rsq_bytes(M, K):
     return M * (2 * K + K / 2 + 4)
 
 
+def rank_row0(rank: int, rows_per_rank: int) -> int:
+    """Weak scaling over token rows: rank r owns rows [r * rows_per_rank, (r + 1) * rows_per_rank) of the virtual
+    activation matrix (whole frames); weights are replicated; there is no collective on the data path."""
+    return rank * rows_per_rank
+
+
+def max_over_ranks(value: float, dist, device: str) -> float:
+    """The slowest rank decides: MAX all-reduce of a per-rank time (no-op without a process group)."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, ops_per_rank: float, ms_per_step: float) -> float:
+    """TOPS of the whole job: every rank does ops_per_rank per step in ms_per_step (the max over ranks)."""
+    return world * ops_per_rank / (ms_per_step * 1e-3) / 1e12
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
 
@@ -174,7 +195,7 @@ def run_ours(args, rank, world, local_rank):
     peaks = load_peaks()
     M = FRAMES * workload.TOKENS_PER_FRAME
     specs = workload.block_specs(0, 0)
-    row0 = rank * M                                     # weak scaling: every rank gets its own 8 frames
+    row0 = rank_row0(rank, M)                           # weak scaling: every rank gets its own 8 frames
 
     def dev_bf16(bits):
         return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
@@ -229,11 +250,7 @@ def run_ours(args, rank, world, local_rank):
     barrier()
     wall1 = time.time()
     clocks = sampler.stop(wall0, wall1)
-    total_ms = t_start.elapsed_time(t_stop)
-    if dist is not None:
-        t = torch.tensor([total_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(t_start.elapsed_time(t_stop), dist, "cuda")
     for L in layers:
         assert L["h"].device_status() == 0, "a device-side wait expired"
 
@@ -258,11 +275,7 @@ def run_ours(args, rank, world, local_rank):
         e2e_step(i)
     e1.record()
     barrier()
-    e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1) / e2e_steps, dist, "cuda")
 
     if rank != 0:
         if dist is not None:
@@ -271,7 +284,7 @@ def run_ours(args, rank, world, local_rank):
 
     ops_step = sum(layer_ops(M, s) for s in specs)
     ms_per_step = total_ms / args.steps
-    tops = world * ops_step / (ms_per_step * 1e-3) / 1e12
+    tops = whole_job_value(world, ops_step, ms_per_step)
     gemm_ops = sum(layer_ops(M, s) for s in specs)
     gemm_avg_ms = gemm_ms.mean(axis=0)                    # per layer
     gemm_tops = gemm_ops / (gemm_avg_ms.sum() * 1e-3) / 1e12

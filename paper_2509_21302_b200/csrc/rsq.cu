@@ -198,10 +198,6 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
     float *Tm = reinterpret_cast<float *>(stage + 2 * G::STAGE_BYTES);
     float *red = Tm + K;                                       // cross-warp maxima (T = 64 only)
 
-    float m[T];                                                // multipliers of elements T k + t
-#pragma unroll
-    for (int k = 0; k < T; ++k) m[k] = __ldg(mul + T * k + t);
-
     // staging copy: 16-byte piece cg = t + T j belongs to thread cg / CH, piece cg % CH of its T values
     uint32_t cp_dst[CH];
 #pragma unroll
@@ -230,6 +226,9 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
         for (int j = 0; j < CH; ++j) cp_async16(stage + cp_dst[j], src + 16 * (t + T * j));
     }
     cp_async_commit();
+    float m[T];                                                // multipliers of elements T k + t (loaded behind the first row's copies)
+#pragma unroll
+    for (int k = 0; k < T; ++k) m[k] = __ldg(mul + T * k + t);
     int buf = 0;
     for (; row < M; row += stride, buf ^= 1) {
         const long long next = row + stride;
