@@ -49,11 +49,7 @@ struct Cfg {
     static constexpr int US = (CG == 1) ? 2 : 4;           // operand stages (decouple converters and MMA)
     // Converter warps form GROUPS independent groups; group g converts K-blocks g, g + GROUPS, ...  so the
     // fixed costs of a stage (draining the stores, the proxy fence, barrier round trips) overlap.
-#ifdef QVGGT_GROUPS
-    static constexpr int GROUPS = QVGGT_GROUPS;
-#else
     static constexpr int GROUPS = (CG == 1) ? 2 : 4;
-#endif
     static constexpr int GROUP_WARPS = CONV_WARPS / GROUPS;
     static constexpr int GROUP_THREADS = GROUP_WARPS * 32;
     static constexpr int CHUNKS = ROWS * 4 / GROUP_THREADS;   // 16-byte packed pieces per thread per stage
@@ -428,9 +424,6 @@ cudaError_t qvggt_launch_gemm(const qvggt_weights *w, const unsigned char *Xq, c
     if (M == 0) return cudaSuccess;
     if (group == 128) return qvggt_launch_gemm_grouped(w, Xq, a_scale, M, Y, ldy, acc_debug, st);
     if (group != 0) return cudaErrorNotSupported;
-#ifdef QVGGT_GEMM_CG1
-    return acc_debug ? launch<1, true>(w, Xq, a_scale, M, Y, ldy, acc_debug, st) : launch<1, false>(w, Xq, a_scale, M, Y, ldy, acc_debug, st);
-#else
+    // the single-CTA configuration (CG = 1) measured 10-35 % slower on every VGGT shape: the pair halves the weight traffic
     return acc_debug ? launch<2, true>(w, Xq, a_scale, M, Y, ldy, acc_debug, st) : launch<2, false>(w, Xq, a_scale, M, Y, ldy, acc_debug, st);
-#endif
 }
