@@ -65,6 +65,7 @@ typedef enum {
  *   bias_bf16 [N] bf16 or NULL (no bias)
  *   smooth_c  [K] fp32, finite and > 0
  *   sign_v    [K] int8 of +1/-1, or NULL (all +1)
+ *   flags     0, or QVGGT_PREP_C8 to keep an extra int8 [N, K] copy of the codes for the *_c8 entry points
  *   out       receives a new handle (device memory is allocated here, on the current device);
  *             release it with qvggt_free_weights.  The handle is bound to that device.
  * Work is enqueued on the stream; the inputs may be released once the stream has passed this call.
@@ -99,6 +100,24 @@ int qvggt_rotate_smooth_quantize(const qvggt_weights_t *w, const void *X_bf16, l
 int qvggt_w4a4_linear(const qvggt_weights_t *w, const unsigned char *Xq, const float *a_scale, int M,
                       int group, void *Y_bf16, long long ldy, int *acc_debug, void *cuda_stream);
 
+/*
+ * The same two steps on codes held one per byte ("8-bit containers").  tcgen05 has no 4-bit integer
+ * kind, so the tensor core multiplies int8 whatever the storage format; when the producers write one
+ * code per byte, the tiles go from global memory straight into the tensor core's operand stages and
+ * the GEMM spends nothing on unpacking.  Codes, scales, integer sums and outputs are those of the
+ * packed entry points, bit for bit; only the layout of Xq differs.  The handle must have been
+ * prepared with QVGGT_PREP_C8 in `flags` (which adds an int8 [N, K] copy of Wq to the handle: 1 byte
+ * per weight on top of the packed 0.5), otherwise QVGGT_ERR_UNSUPPORTED.  Per-token scales only.
+ *   Xq8      int8 [M, K], one code per byte in [-7, 7], natural element order, 16-byte aligned
+ *   a_scale  fp32 [M]
+ *   Y_bf16, ldy, acc_debug (int32 [M, N]) as for qvggt_w4a4_linear with group 0
+ */
+#define QVGGT_PREP_C8 1
+int qvggt_rotate_smooth_quantize_c8(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M,
+                                    signed char *Xq8, float *a_scale, void *cuda_stream);
+int qvggt_w4a4_linear_c8(const qvggt_weights_t *w, const signed char *Xq8, const float *a_scale, int M,
+                         void *Y_bf16, long long ldy, int *acc_debug, void *cuda_stream);
+
 /* Frees the handle and its device memory (synchronises the device first).  NULL is allowed. */
 void qvggt_free_weights(qvggt_weights_t *w);
 
@@ -109,6 +128,9 @@ void qvggt_free_weights(qvggt_weights_t *w);
  */
 int qvggt_weights_view(const qvggt_weights_t *w, const unsigned char **Wq, const float **w_scale,
                        const float **amul, const void **bias_bf16, int *N, int *K);
+
+/* Device pointer to the int8 [N, K] copy of the codes (NULL if the handle was prepared without QVGGT_PREP_C8). */
+int qvggt_weights_view_c8(const qvggt_weights_t *w, const signed char **Wq8);
 
 /*
  * Synchronises `cuda_stream`, then reads the handle's device status word into *code (HOST pointer):

@@ -20,7 +20,9 @@ _STATUS_NAMES = {0: "QVGGT_OK", -1: "QVGGT_ERR_NULL", -2: "QVGGT_ERR_SHAPE", -3:
 
 EXPORTS = ("qvggt_prepare_weights", "qvggt_rotate_smooth_quantize", "qvggt_w4a4_linear", "qvggt_free_weights",
            "qvggt_weights_view", "qvggt_device_status", "qvggt_calibrate_smooth", "qvggt_status_string",
-           "qvggt_quantize_weights_static")
+           "qvggt_quantize_weights_static", "qvggt_rotate_smooth_quantize_c8", "qvggt_w4a4_linear_c8",
+           "qvggt_weights_view_c8")
+PREP_C8 = 1   # QVGGT_PREP_C8: keep an int8 [N, K] copy of the weight codes for the *_c8 entry points
 
 
 class QvggtError(RuntimeError):
@@ -46,6 +48,9 @@ def lib() -> ctypes.CDLL:
         L.qvggt_prepare_weights.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, ctypes.POINTER(vp)]
         L.qvggt_rotate_smooth_quantize.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp]
         L.qvggt_w4a4_linear.argtypes = [vp, vp, vp, i32, i32, vp, i64, vp, vp]
+        L.qvggt_rotate_smooth_quantize_c8.argtypes = [vp, vp, i64, i32, vp, vp, vp]
+        L.qvggt_w4a4_linear_c8.argtypes = [vp, vp, vp, i32, vp, i64, vp, vp]
+        L.qvggt_weights_view_c8.argtypes = [vp, ctypes.POINTER(vp)]
         L.qvggt_free_weights.argtypes = [vp]
         L.qvggt_free_weights.restype = None
         L.qvggt_weights_view.argtypes = [vp] + [ctypes.POINTER(vp)] * 4 + [ctypes.POINTER(i32)] * 2
@@ -108,6 +113,14 @@ class Weights:
                     amul=wrap(ptrs[2], 4 * K, torch.float32, (K,)),
                     bias=wrap(ptrs[3], 2 * N, torch.bfloat16, (N,)))
 
+    def view_c8(self) -> torch.Tensor | None:
+        """Copy of the int8 [N, K] codes (None if prepared without c8=True)."""
+        p = ctypes.c_void_p()
+        _check(lib().qvggt_weights_view_c8(self.handle, ctypes.byref(p)), "qvggt_weights_view_c8")
+        if not p.value:
+            return None
+        return _from_device_ptr(p.value, self.N * self.K, torch.uint8, (self.N, self.K)).view(torch.int8)
+
     def device_status(self) -> int:
         code = ctypes.c_int(0)
         st = lib().qvggt_device_status(self.handle, _stream(), ctypes.byref(code))
@@ -144,8 +157,9 @@ def _from_device_ptr(ptr: int, nbytes: int, dtype: torch.dtype, shape) -> torch.
 
 
 def prepare_weights(W: torch.Tensor, bias: torch.Tensor | None, smooth_c: torch.Tensor,
-                    sign_v: torch.Tensor | None = None) -> Weights:
-    """W [N,K] bf16, bias [N] bf16 or None, smooth_c [K] fp32, sign_v [K] int8 (+1/-1) or None."""
+                    sign_v: torch.Tensor | None = None, c8: bool = False) -> Weights:
+    """W [N,K] bf16, bias [N] bf16 or None, smooth_c [K] fp32, sign_v [K] int8 (+1/-1) or None.
+    c8: also keep the codes one per byte, as the *_c8 entry points need them."""
     assert W.dim() == 2 and W.element_size() == 2 and W.is_contiguous()
     N, K = W.shape
     assert smooth_c.dtype == torch.float32 and smooth_c.numel() == K and smooth_c.is_contiguous()
@@ -154,7 +168,7 @@ def prepare_weights(W: torch.Tensor, bias: torch.Tensor | None, smooth_c: torch.
     if sign_v is not None:
         assert sign_v.dtype == torch.int8 and sign_v.numel() == K and sign_v.is_contiguous()
     h = ctypes.c_void_p()
-    _check(lib().qvggt_prepare_weights(_ptr(W), _ptr(bias), _ptr(smooth_c), _ptr(sign_v), N, K, 0, _stream(),
+    _check(lib().qvggt_prepare_weights(_ptr(W), _ptr(bias), _ptr(smooth_c), _ptr(sign_v), N, K, PREP_C8 if c8 else 0, _stream(),
                                        ctypes.byref(h)), "qvggt_prepare_weights")
     return Weights(h.value, N, K)
 
@@ -188,6 +202,39 @@ def w4a4_linear(w: Weights, Xq: torch.Tensor, a_scale: torch.Tensor, group: int 
         assert acc_debug.dtype == torch.int32 and acc_debug.is_contiguous()
     _check(lib().qvggt_w4a4_linear(w.handle, _ptr(Xq), _ptr(a_scale), M, group, _ptr(Y), ldy, _ptr(acc_debug), _stream()),
            "qvggt_w4a4_linear")
+    return Y
+
+
+def rotate_smooth_quantize_c8(w: Weights, X: torch.Tensor, Xq8: torch.Tensor | None = None,
+                              a_scale: torch.Tensor | None = None):
+    """X [M,K] bf16 (row stride may exceed K) -> (Xq8 [M,K] int8, one code per byte; a_scale fp32 [M])."""
+    assert X.dim() == 2 and X.element_size() == 2 and X.stride(1) == 1 and X.shape[1] == w.K
+    M = X.shape[0]
+    if Xq8 is None:
+        Xq8 = torch.empty((M, w.K), dtype=torch.int8, device=X.device)
+    if a_scale is None:
+        a_scale = torch.empty((M,), dtype=torch.float32, device=X.device)
+    assert Xq8.dtype == torch.int8 and Xq8.is_contiguous() and a_scale.dtype == torch.float32
+    ldx = X.stride(0) if M > 1 else w.K
+    _check(lib().qvggt_rotate_smooth_quantize_c8(w.handle, _ptr(X), ldx, M, _ptr(Xq8), _ptr(a_scale), _stream()),
+           "qvggt_rotate_smooth_quantize_c8")
+    return Xq8, a_scale
+
+
+def w4a4_linear_c8(w: Weights, Xq8: torch.Tensor, a_scale: torch.Tensor, Y: torch.Tensor | None = None,
+                   acc_debug: torch.Tensor | None = None) -> torch.Tensor:
+    """-> Y [M,N] bf16 from codes held one per byte.  acc_debug: optional int32 [M,N] receiving the integer sums."""
+    M = Xq8.shape[0]
+    assert Xq8.dtype == torch.int8 and Xq8.is_contiguous() and Xq8.shape[1] == w.K
+    assert a_scale.dtype == torch.float32 and a_scale.is_contiguous()
+    if Y is None:
+        Y = torch.empty((M, w.N), dtype=torch.bfloat16, device=Xq8.device)
+    assert Y.element_size() == 2 and Y.stride(1) == 1 and Y.shape == (M, w.N)
+    ldy = Y.stride(0) if M > 1 else w.N
+    if acc_debug is not None:
+        assert acc_debug.dtype == torch.int32 and acc_debug.is_contiguous()
+    _check(lib().qvggt_w4a4_linear_c8(w.handle, _ptr(Xq8), _ptr(a_scale), M, _ptr(Y), ldy, _ptr(acc_debug), _stream()),
+           "qvggt_w4a4_linear_c8")
     return Y
 
 

@@ -21,6 +21,7 @@ void release(qvggt_weights *w)
 {
     if (!w) return;
     cudaFree(w->Wq);
+    cudaFree(w->Wq8);
     cudaFree(w->w_scale);
     cudaFree(w->amul);
     cudaFree(w->bias);
@@ -35,7 +36,7 @@ extern "C" {
 int qvggt_prepare_weights(const void *W_bf16, const void *bias_bf16, const float *smooth_c, const signed char *sign_v,
                           int N, int K, int flags, void *cuda_stream, qvggt_weights_t **out)
 {
-    (void)flags;
+    if (flags & ~QVGGT_PREP_C8) return QVGGT_ERR_UNSUPPORTED;
     if (!out) return QVGGT_ERR_NULL;
     *out = nullptr;
     if (!W_bf16 || !smooth_c) return QVGGT_ERR_NULL;
@@ -48,7 +49,7 @@ int qvggt_prepare_weights(const void *W_bf16, const void *bias_bf16, const float
     if (!w) return QVGGT_ERR_NOMEM;
     w->N = N;
     w->K = K;
-    w->Wq = nullptr; w->w_scale = nullptr; w->amul = nullptr; w->bias = nullptr; w->status = nullptr;
+    w->Wq = nullptr; w->Wq8 = nullptr; w->w_scale = nullptr; w->amul = nullptr; w->bias = nullptr; w->status = nullptr;
     cudaGetDevice(&w->device);
     float *wmul = nullptr;
     bool ok = cudaMalloc(&w->Wq, (size_t)N * K / 2) == cudaSuccess &&
@@ -56,7 +57,8 @@ int qvggt_prepare_weights(const void *W_bf16, const void *bias_bf16, const float
               cudaMalloc(&w->amul, sizeof(float) * K) == cudaSuccess &&
               cudaMalloc(&w->status, sizeof(int)) == cudaSuccess &&
               cudaMallocAsync(&wmul, sizeof(float) * K, st) == cudaSuccess &&
-              (!bias_bf16 || cudaMalloc(&w->bias, sizeof(uint16_t) * N) == cudaSuccess);
+              (!bias_bf16 || cudaMalloc(&w->bias, sizeof(uint16_t) * N) == cudaSuccess) &&
+              (!(flags & QVGGT_PREP_C8) || cudaMalloc(&w->Wq8, (size_t)N * K) == cudaSuccess);
     if (!ok) {
         cudaGetLastError();
         if (wmul) cudaFreeAsync(wmul, st);
@@ -68,6 +70,7 @@ int qvggt_prepare_weights(const void *W_bf16, const void *bias_bf16, const float
         e = cudaMemcpyAsync(w->bias, bias_bf16, sizeof(uint16_t) * N, cudaMemcpyDeviceToDevice, st);
     if (e == cudaSuccess) e = qvggt_launch_multipliers(smooth_c, sign_v, K, w->amul, wmul, st);
     if (e == cudaSuccess) e = qvggt_launch_rsq(W_bf16, K, N, K, wmul, 0, w->Wq, w->w_scale, st);
+    if (e == cudaSuccess && w->Wq8) e = qvggt_launch_rsq_c8(W_bf16, K, N, K, wmul, w->Wq8, w->w_scale, st);
     // wmul is scratch: stream-ordered release so that the call stays asynchronous
     if (cudaFreeAsync(wmul, st) != cudaSuccess) cudaGetLastError();
     if (e != cudaSuccess) {
@@ -110,6 +113,36 @@ int qvggt_w4a4_linear(const qvggt_weights_t *w, const unsigned char *Xq, const f
     return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
 }
 
+int qvggt_rotate_smooth_quantize_c8(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M, signed char *Xq8,
+                                    float *a_scale, void *cuda_stream)
+{
+    if (!w) return QVGGT_ERR_NULL;
+    if (M < 0) return QVGGT_ERR_SHAPE;
+    if (M == 0) return QVGGT_OK;
+    if (!X_bf16 || !Xq8 || !a_scale) return QVGGT_ERR_NULL;
+    if (ldx < w->K) return QVGGT_ERR_SHAPE;
+    if (ldx % 8 != 0 || !aligned16(X_bf16) || !aligned16(Xq8) || (reinterpret_cast<uintptr_t>(a_scale) & 3u)) return QVGGT_ERR_ALIGN;
+    cudaError_t e = qvggt_launch_rsq_c8(X_bf16, ldx, M, w->K, w->amul, Xq8, a_scale, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
+}
+
+int qvggt_w4a4_linear_c8(const qvggt_weights_t *w, const signed char *Xq8, const float *a_scale, int M, void *Y_bf16,
+                         long long ldy, int *acc_debug, void *cuda_stream)
+{
+    if (!w) return QVGGT_ERR_NULL;
+    if (M < 0) return QVGGT_ERR_SHAPE;
+    if (!w->Wq8) return QVGGT_ERR_UNSUPPORTED;
+    if (M == 0) return QVGGT_OK;
+    if (!Xq8 || !a_scale || !Y_bf16) return QVGGT_ERR_NULL;
+    if (ldy < w->N) return QVGGT_ERR_SHAPE;
+    if (ldy % 8 != 0 || !aligned16(Xq8) || !aligned16(Y_bf16) || (acc_debug && !aligned16(acc_debug)) ||
+        (reinterpret_cast<uintptr_t>(a_scale) & 3u))
+        return QVGGT_ERR_ALIGN;
+    cudaError_t e = qvggt_launch_gemm_c8(w, Xq8, a_scale, M, Y_bf16, ldy, acc_debug, static_cast<cudaStream_t>(cuda_stream));
+    if (e == cudaErrorNotSupported) return QVGGT_ERR_UNSUPPORTED;
+    return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
+}
+
 void qvggt_free_weights(qvggt_weights_t *w)
 {
     if (!w) return;
@@ -131,6 +164,13 @@ int qvggt_weights_view(const qvggt_weights_t *w, const unsigned char **Wq, const
     if (bias_bf16) *bias_bf16 = w->bias;
     if (N) *N = w->N;
     if (K) *K = w->K;
+    return QVGGT_OK;
+}
+
+int qvggt_weights_view_c8(const qvggt_weights_t *w, const signed char **Wq8)
+{
+    if (!w || !Wq8) return QVGGT_ERR_NULL;
+    *Wq8 = w->Wq8;
     return QVGGT_OK;
 }
 

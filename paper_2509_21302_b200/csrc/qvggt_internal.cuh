@@ -9,6 +9,7 @@ struct qvggt_weights {
     int N, K;
     int device;
     unsigned char *Wq;   // [N, K/2] packed int4
+    signed char *Wq8;    // [N, K] one code per byte, or nullptr (prepared without QVGGT_PREP_C8)
     float *w_scale;      // [N]
     float *amul;         // [K]
     uint16_t *bias;      // [N] bf16 bits, or nullptr
@@ -31,6 +32,8 @@ cudaError_t qvggt_launch_multipliers(const float *c, const signed char *v, int K
                                      cudaStream_t st);
 cudaError_t qvggt_launch_rsq(const void *X, long long ldx, int M, int K, const float *mul, int group,
                              unsigned char *Xq, float *scales, cudaStream_t st);
+cudaError_t qvggt_launch_rsq_c8(const void *X, long long ldx, int M, int K, const float *mul, signed char *Xq8,
+                                float *scales, cudaStream_t st);
 cudaError_t qvggt_launch_colmax(const void *X, int M, int K, float *colmax, cudaStream_t st);
 cudaError_t qvggt_launch_smooth_finalize(const float *ax, const float *aw, int K, float alpha, float lo, float hi,
                                          float *c, cudaStream_t st);
@@ -43,3 +46,7 @@ cudaError_t qvggt_launch_gemm(const qvggt_weights *w, const unsigned char *Xq, c
 cudaError_t qvggt_launch_gemm_grouped(const qvggt_weights *w, const unsigned char *Xq, const float *a_scale, int M, void *Y,
                                       long long ldy, int *acc_debug, cudaStream_t st);
 
+
+// gemm_c8.cu (codes in 8-bit containers: TMA feeds the tensor core directly)
+cudaError_t qvggt_launch_gemm_c8(const qvggt_weights *w, const signed char *Xq8, const float *a_scale, int M, void *Y,
+                                 long long ldy, int *acc_debug, cudaStream_t st);

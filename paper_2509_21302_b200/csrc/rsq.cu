@@ -183,7 +183,8 @@ __device__ __forceinline__ void stages_in_registers(float (&v)[N])
             if (!(k & h)) bfly2(v[k], v[k + 1], v[k + h], v[k + 1 + h]);
 }
 
-template <int LOGT, int GROUP>
+// C8: one code per byte (int8, natural element order, row pitch K) instead of two per byte.
+template <int LOGT, int GROUP, bool C8 = false>
 __global__ void __launch_bounds__(SqGeom<LOGT>::CTA_THREADS, LOGT == 5 ? 4 : 3)
 rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float *__restrict__ mul,
               unsigned char *__restrict__ Xq, float *__restrict__ scales)
@@ -289,6 +290,28 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
 #pragma unroll
             for (int g = 0; g < NG; ++g) am[g] = fmaxf(red[g], red[NG + g]);
         }
+        if constexpr (C8) {
+            static_assert(!C8 || GROUP == 0, "byte output is built for per-token scales");
+            am[0] = fmaxf(am[0], 1e-8f);
+            const float inv = __fdiv_rn(7.0f, am[0]);
+            const uint64_t inv2 = ptx::f32x2_pack(inv, inv), magic2 = ptx::f32x2_pack(12582912.0f, 12582912.0f);
+            // byte exchange between the 4 lanes that share (t / 4): a 4 x 4 byte transpose in two steps
+            const uint32_t sel0 = (lane & 1) ? 0x3715u : 0x6240u, sel1 = (lane & 2) ? 0x3276u : 0x5410u;
+#pragma unroll
+            for (int kk = 0; kk < T / 4; ++kk) {
+                // exact product + 1.5*2^23, rounded once (half-to-even): the low mantissa byte is the int8 code
+                float f0, f1, f2, f3;
+                ptx::f32x2_unpack(ptx::f32x2_fma(ptx::f32x2_pack(v[4 * kk], v[4 * kk + 1]), inv2, magic2), f0, f1);
+                ptx::f32x2_unpack(ptx::f32x2_fma(ptx::f32x2_pack(v[4 * kk + 2], v[4 * kk + 3]), inv2, magic2), f2, f3);
+                // byte n = code of element T (4 kk + n) + t
+                uint32_t x = __byte_perm(__byte_perm(__float_as_uint(f0), __float_as_uint(f1), 0x0040),
+                                         __byte_perm(__float_as_uint(f2), __float_as_uint(f3), 0x0040), 0x5410);
+                x = __byte_perm(x, __shfl_xor_sync(0xFFFFFFFFu, x, 1), sel0);
+                x = __byte_perm(x, __shfl_xor_sync(0xFFFFFFFFu, x, 2), sel1);
+                // now byte n = code of element T (4 kk + e) + 4 (t / 4) + n, e = t mod 4: one whole output word
+                *reinterpret_cast<uint32_t *>(Xq + row * K + T * (4 * kk + (t & 3)) + 4 * (t >> 2)) = x;
+            }
+        } else {
         uint32_t word[T / 8];
 #pragma unroll
         for (int g = 0; g < NG; ++g) {
@@ -317,6 +340,7 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
                 x = (x & nb_keep[i]) | __shfl_xor_sync(0xFFFFFFFFu, send, 1 << i);
             }
             *reinterpret_cast<uint32_t *>(Xq + row * (K / 2) + 4 * ((T / 8) * (8 * kk + (t & 7)) + (t >> 3))) = x;
+        }
         }
         if (t == 0) {
 #pragma unroll
@@ -395,6 +419,28 @@ cudaError_t qvggt_launch_multipliers(const float *c, const signed char *v, int K
                                      cudaStream_t st)
 {
     multipliers_kernel<<<(K + 255) / 256, 256, 0, st>>>(c, v, K, amul, wmul);
+    return cudaGetLastError();
+}
+
+cudaError_t qvggt_launch_rsq_c8(const void *X, long long ldx, int M, int K, const float *mul, signed char *Xq8,
+                                float *scales, cudaStream_t st)
+{
+    if (M == 0) return cudaSuccess;
+    const uint16_t *x = static_cast<const uint16_t *>(X);
+    unsigned char *out = reinterpret_cast<unsigned char *>(Xq8);
+    static bool configured = false;       // per process
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(rsq_sq_kernel<6, 0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SqGeom<6>::SMEM);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    if (K == 1024) {
+        using G = SqGeom<5>;
+        rsq_sq_kernel<5, 0, true><<<rsq_grid(M, G::ROWS, 4), G::CTA_THREADS, G::SMEM, st>>>(x, ldx, M, mul, out, scales);
+    } else {
+        using G = SqGeom<6>;
+        rsq_sq_kernel<6, 0, true><<<rsq_grid(M, G::ROWS, 3), G::CTA_THREADS, G::SMEM, st>>>(x, ldx, M, mul, out, scales);
+    }
     return cudaGetLastError();
 }
 

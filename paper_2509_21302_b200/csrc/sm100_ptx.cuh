@@ -346,6 +346,16 @@ __device__ __forceinline__ void tma_load_2d(const void *tmap, uint32_t bar, uint
                  : "memory");
 }
 
+// Same load issued inside a CTA pair: the data lands in THIS CTA's shared memory, while the completion may be
+// signalled on an mbarrier of either CTA of the pair (`bar_cluster` is a shared::cluster address, see map_to_cta),
+// so that one barrier of the leader collects the bytes of both halves of an operand stage.
+__device__ __forceinline__ void tma_load_2d_pair(const void *tmap, uint32_t bar_cluster, uint32_t smem_dst, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(smem_dst),
+                 "l"(tmap), "r"(x), "r"(y), "r"(bar_cluster)
+                 : "memory");
+}
+
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
