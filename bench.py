@@ -43,12 +43,33 @@ def layer_ops(M, spec):
     return 2.0 * M * spec.N * spec.K
 
 
-def gemm_bytes(M, spec):
-    return M * spec.K / 2 + 4 * M + spec.N * spec.K / 2 + 6 * spec.N + 2.0 * M * spec.N
+def gemm_bytes(M, spec, code_bytes=0.5):
+    return M * spec.K * code_bytes + 4 * M + spec.N * spec.K * code_bytes + 6 * spec.N + 2.0 * M * spec.N
 
 
-def rsq_bytes(M, K):
-    return M * (2 * K + K / 2 + 4)
+def rsq_bytes(M, K, code_bytes=0.5):
+    return M * (2 * K + K * code_bytes + 4)
+
+
+class Path:
+    """The two storage formats of the codes between the quantize kernel and the GEMM: `packed` (two codes per
+    byte) and `c8` (one code per byte, TMA-fed GEMM without an unpacking stage).  Same codes, scales and outputs."""
+
+    def __init__(self, q, torch, fmt: str):
+        self.fmt = fmt
+        self.code_bytes = 1.0 if fmt == "c8" else 0.5
+        if fmt == "c8":
+            self.prepare = lambda W, b, c: q.prepare_weights(W, b, c, None, c8=True)
+            self.rsq = lambda h, x, xq, a: q.rotate_smooth_quantize_c8(h, x, xq, a)
+            self.gemm = lambda h, xq, a, y: q.w4a4_linear_c8(h, xq, a, y)
+            self.new_xq = lambda M, K: torch.empty((M, K), dtype=torch.int8, device="cuda")
+            self.gemm_kernel, self.rsq_kernel = "gemm_c8_kernel", "rsq_sq_kernel<.., c8>"
+        else:
+            self.prepare = lambda W, b, c: q.prepare_weights(W, b, c, None)
+            self.rsq = lambda h, x, xq, a: q.rotate_smooth_quantize(h, x, 0, xq, a)
+            self.gemm = lambda h, xq, a, y: q.w4a4_linear(h, xq, a, 0, y)
+            self.new_xq = lambda M, K: torch.empty((M, K // 2), dtype=torch.uint8, device="cuda")
+            self.gemm_kernel, self.rsq_kernel = "gemm_w4a4_kernel", "rsq_sq_kernel"
 
 
 def rank_row0(rank: int, rows_per_rank: int) -> int:
@@ -192,6 +213,8 @@ def run_ours(args, rank, world, local_rank):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     q.build()
+    path = Path(q, torch, args.format)
+    cb = path.code_bytes
     peaks = load_peaks()
     M = FRAMES * workload.TOKENS_PER_FRAME
     specs = workload.block_specs(0, 0)
@@ -205,11 +228,11 @@ def run_ours(args, rank, world, local_rank):
     for s in specs:
         W = dev_bf16(s.weight())
         c = q.calibrate_smooth(dev_bf16(s.x_calib()), W)
-        h = q.prepare_weights(W, dev_bf16(s.bias()), c, None)
+        h = path.prepare(W, dev_bf16(s.bias()), c)
         host_x = torch.from_numpy(s.x_rows(row0, M).view(np.int16)).pin_memory()
         xs = [host_x.cuda().view(torch.bfloat16) for _ in range(NBUF)]
         layers.append(dict(spec=s, h=h, host_x=host_x, x=xs,
-                           xq=[torch.empty((M, s.K // 2), dtype=torch.uint8, device="cuda") for _ in range(NBUF)],
+                           xq=[path.new_xq(M, s.K) for _ in range(NBUF)],
                            a=[torch.empty((M,), dtype=torch.float32, device="cuda") for _ in range(NBUF)],
                            y=[torch.empty((M, s.N), dtype=torch.bfloat16, device="cuda") for _ in range(NBUF)],
                            host_y=torch.empty((M, s.N), dtype=torch.bfloat16).pin_memory()))
@@ -220,10 +243,10 @@ def run_ours(args, rank, world, local_rank):
         for li, L in enumerate(layers):
             if ev is not None:
                 ev[li][0].record()
-            q.rotate_smooth_quantize(L["h"], L["x"][b], 0, L["xq"][b], L["a"][b])
+            path.rsq(L["h"], L["x"][b], L["xq"][b], L["a"][b])
             if ev is not None:
                 ev[li][1].record()
-            q.w4a4_linear(L["h"], L["xq"][b], L["a"][b], 0, L["y"][b])
+            path.gemm(L["h"], L["xq"][b], L["a"][b], L["y"][b])
             if ev is not None:
                 ev[li][2].record()
 
@@ -262,8 +285,8 @@ def run_ours(args, rank, world, local_rank):
         b = i % NBUF
         for L in layers:
             L["x"][b].view(torch.int16).copy_(L["host_x"], non_blocking=True)
-            q.rotate_smooth_quantize(L["h"], L["x"][b], 0, L["xq"][b], L["a"][b])
-            q.w4a4_linear(L["h"], L["xq"][b], L["a"][b], 0, L["y"][b])
+            path.rsq(L["h"], L["x"][b], L["xq"][b], L["a"][b])
+            path.gemm(L["h"], L["xq"][b], L["a"][b], L["y"][b])
             L["host_y"].copy_(L["y"][b], non_blocking=True)
 
     e2e_steps = max(2, min(args.steps, 5))
@@ -291,7 +314,7 @@ def run_ours(args, rank, world, local_rank):
     int8_peak = peaks["bf16_tflops"] * NOMINAL_INT8_OVER_BF16
     int8_peak_sus = peaks["bf16_tflops_sustained"] * NOMINAL_INT8_OVER_BF16
     rsq_avg_ms = rsq_ms.mean(axis=0)
-    rsq_b = sum(rsq_bytes(M, s.K) for s in specs)
+    rsq_b = sum(rsq_bytes(M, s.K, cb) for s in specs)
     rsq_gbs = rsq_b / (rsq_avg_ms.sum() * 1e-3) / 1e9
     # DRAM bytes per launch from the committed ncu summary (None once a kernel has changed since the capture).
     # The quantize kernel was captured at M = 137400; its traffic grows with the rows, so it is scaled per row.
@@ -300,6 +323,7 @@ def run_ours(args, rank, world, local_rank):
     if os.path.exists(tpath):
         with open(tpath) as f:
             tj = json.load(f)
+        tj = tj.get(path.fmt, {})
         traffic = tj.get("gemm_bytes_per_launch_avg")
         per_row = tj.get("rsq_bytes_per_row")
         if per_row:
@@ -307,11 +331,11 @@ def run_ours(args, rank, world, local_rank):
     per_layer = {}
     for li, s in enumerate(specs):
         t_g, t_r = gemm_avg_ms[li] * 1e-3, rsq_avg_ms[li] * 1e-3
-        bound = max(layer_ops(M, s) / (int8_peak * 1e12), gemm_bytes(M, s) / (peaks["hbm_gbs"] * 1e9))
+        bound = max(layer_ops(M, s) / (int8_peak * 1e12), gemm_bytes(M, s, cb) / (peaks["hbm_gbs"] * 1e9))
         per_layer[s.name] = {"gemm_us": round(t_g * 1e6, 2), "gemm_tops": round(layer_ops(M, s) / t_g / 1e12, 1),
                              "gemm_roofline_frac": round(bound / t_g, 4),
-                             "rsq_us": round(t_r * 1e6, 2), "rsq_gbs": round(rsq_bytes(M, s.K) / t_r / 1e9, 1),
-                             "rsq_hbm_frac": round(rsq_bytes(M, s.K) / t_r / 1e9 / peaks["hbm_gbs"], 4)}
+                             "rsq_us": round(t_r * 1e6, 2), "rsq_gbs": round(rsq_bytes(M, s.K, cb) / t_r / 1e9, 1),
+                             "rsq_hbm_frac": round(rsq_bytes(M, s.K, cb) / t_r / 1e9 / peaks["hbm_gbs"], 4)}
     out = {
         "metric": "w4a4_linear_tops", "value": tops, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -319,17 +343,18 @@ def run_ours(args, rank, world, local_rank):
         "tokens_per_s": world * M / (ms_per_step * 1e-3),
         "config": {"workload": "aggregator block, 4 linears (qkv/proj/fc1/fc2), 8 frames M=10992 per GPU (BASELINE configs[1])",
                    "l2": f"step working set ~400 MB > 126 MB L2; {NBUF} buffer sets alternated per step",
-                   "timed": "rotate-smooth-quantize + W4A4 GEMM/epilogue per linear; weight prep offline"},
+                   "timed": "rotate-smooth-quantize + W4A4 GEMM/epilogue per linear; weight prep offline",
+                   "code_format": "int4 codes one per byte between the kernels (c8)" if path.fmt == "c8" else "int4 codes packed two per byte"},
         "clocks": clocks,
         "gpu_launches": int(2 * len(layers) * args.steps),
         "e2e": {"value": world * ops_step / (e2e_ms * 1e-3) / 1e12, "unit": "TOPS", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": int(sum(M * s.K * 2 for s in specs)),
                 "d2h_bytes_per_step": int(sum(M * s.N * 2 for s in specs))},
-        "roofline": {"kernel": "gemm_w4a4_kernel (4 launches per step)", "bound": "tensor", "achieved": gemm_tops,
+        "roofline": {"kernel": f"{path.gemm_kernel} (4 launches per step)", "bound": "tensor", "achieved": gemm_tops,
                      "peak": int8_peak, "unit": "TOP/s", "frac": gemm_tops / int8_peak,
                      "peak_note": f"int8 dense = {NOMINAL_INT8_OVER_BF16:g} x bf16 burst, of {peaks['source']}",
                      "frac_of_sustained": gemm_tops / int8_peak_sus, "traffic": traffic},
-        "roofline_rsq": {"kernel": "rsq_sq_kernel (4 launches per step)", "bound": "hbm", "achieved": rsq_gbs,
+        "roofline_rsq": {"kernel": f"{path.rsq_kernel} (4 launches per step)", "bound": "hbm", "achieved": rsq_gbs,
                          "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": rsq_gbs / peaks["hbm_gbs"],
                          "peak_note": f"of {peaks['source']}", "traffic": rsq_traffic},
         "per_layer": per_layer,
@@ -349,36 +374,38 @@ def run_rsq_sweep(args):
 
     torch.cuda.set_device(0)
     q.build()
+    path = Path(q, torch, args.format)
     peaks = load_peaks()
     out = {}
     for K in (1024, 4096):
         W = torch.zeros((128, K), dtype=torch.bfloat16, device="cuda")
-        h = q.prepare_weights(W, None, torch.ones(K, device="cuda"), None)
+        h = path.prepare(W, None, torch.ones(K, device="cuda"))
         for frames in (1, 8, 32, 100):
             M = frames * workload.TOKENS_PER_FRAME
             X = torch.from_numpy(workload.sweep_activations(3, K, 0, M).view(np.int16)).cuda().view(torch.bfloat16)
-            xq = torch.empty((M, K // 2), dtype=torch.uint8, device="cuda")
+            xq = path.new_xq(M, K)
             a = torch.empty((M,), dtype=torch.float32, device="cuda")
             flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
             for _ in range(3):
-                q.rotate_smooth_quantize(h, X, 0, xq, a)
+                path.rsq(h, X, xq, a)
             times = []
             for _ in range(max(5, min(args.steps, 30))):
                 flush.zero_()                                     # larger than L2: the next launch starts cold
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record()
-                q.rotate_smooth_quantize(h, X, 0, xq, a)
+                path.rsq(h, X, xq, a)
                 e1.record()
                 torch.cuda.synchronize()
                 times.append(e0.elapsed_time(e1))
             us = float(np.median(times)) * 1e3
-            gbs = rsq_bytes(M, K) / us / 1e3
+            gbs = rsq_bytes(M, K, path.code_bytes) / us / 1e3
             out[f"K{K}_M{M}"] = {"us": round(us, 2), "gbs": round(gbs, 1), "hbm_frac": round(gbs / peaks["hbm_gbs"], 4)}
             del X, xq, a, flush
     best = max(v["gbs"] for v in out.values())
     print(json.dumps({"metric": "rsq_gbs", "value": best, "unit": "GB/s", "n_gpus": 1, "higher_is_better": True,
                       "dtype": "fp32 rotation -> int4", "data": "synthetic",
-                      "config": {"workload": "rotate-smooth-quantize sweep (BASELINE configs[2]); L2 flushed between launches"},
+                      "config": {"workload": "rotate-smooth-quantize sweep (BASELINE configs[2]); L2 flushed between launches",
+                                 "code_format": path.fmt},
                       "roofline": {"bound": "hbm", "achieved": best, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                    "frac": best / peaks["hbm_gbs"], "peak_note": f"of {peaks['source']}", "traffic": None},
                       "sweep": out}))
@@ -394,6 +421,7 @@ def run_stack(args):
 
     torch.cuda.set_device(0)
     q.build()
+    path = Path(q, torch, args.format)
     M, blocks = 32 * workload.TOKENS_PER_FRAME, 48
 
     def dev_bf16(bits):
@@ -407,16 +435,16 @@ def run_stack(args):
         for i, s in enumerate(workload.block_specs(1, blk)):
             W = dev_bf16(s.weight())
             c = q.calibrate_smooth(xcal[i], W)
-            handles.append((i, q.prepare_weights(W, dev_bf16(s.bias()), c, None)))
-    xq = [torch.empty((M, s.K // 2), dtype=torch.uint8, device="cuda") for s in kinds]
+            handles.append((i, path.prepare(W, dev_bf16(s.bias()), c)))
+    xq = [path.new_xq(M, s.K) for s in kinds]
     a = torch.empty((M,), dtype=torch.float32, device="cuda")
     y = [torch.empty((M, s.N), dtype=torch.bfloat16, device="cuda") for s in kinds]
     torch.cuda.synchronize()
 
     def stack():
         for i, h in handles:
-            q.rotate_smooth_quantize(h, xs[i], 0, xq[i], a)
-            q.w4a4_linear(h, xq[i], a, 0, y[i])
+            path.rsq(h, xs[i], xq[i], a)
+            path.gemm(h, xq[i], a, y[i])
 
     for _ in range(2):
         stack()
@@ -437,7 +465,7 @@ def run_stack(args):
                       "dtype": "int4 x int4 -> int32 (fp32 rotation and scales)", "tokens_per_s": M / (ms * 1e-3),
                       "gpu_launches": 2 * len(handles) * reps,
                       "config": {"workload": "48-block linear stack, 32 frames M=43968 (BASELINE configs[3])",
-                                 "l2": "per-layer working set 90-450 MB > 126 MB L2"}}))
+                                 "l2": "per-layer working set 90-450 MB > 126 MB L2", "code_format": path.fmt}}))
 
 
 def main():
@@ -448,6 +476,8 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--ref-rows", type=int, default=512, help="token rows per step of the oracle arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--format", choices=["c8", "packed"], default="c8",
+                    help="storage of the int4 codes between the kernels: c8 = one per byte (default), packed = two per byte")
     ap.add_argument("--workload", choices=["block", "rsq_sweep", "stack"], default="block",
                     help="block = BASELINE configs[1] (the default, the contract line); rsq_sweep = configs[2]")
     args = ap.parse_args()

@@ -1,0 +1,160 @@
+"""GPU parity of the 8-bit-container entry points (one int4 code per byte between the kernels) against the CPU
+oracle: the codes, scales, int32 sums and bf16 outputs must be those of the packed path, i.e. of the oracle --
+int4 codes and int32 sums bit-exact, scales and outputs within one bf16 ulp (bit-equal in practice).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workload
+from _util import assert_bf16_within_one_ulp, dev_bf16, host_bits
+
+pytestmark = pytest.mark.gpu
+
+q = None
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    global q
+    import paper_2509_21302_b200 as pkg
+    pkg.build()
+    q = pkg
+    yield
+    torch.cuda.synchronize()
+
+
+def make_layer(spec, use_signs=False, calib_rows=256):
+    W, b = spec.weight(), spec.bias()
+    c = oracle.smooth_factors(spec.x_calib(calib_rows), W)
+    v = workload.signs_i8(spec.seed, 900 + spec.layer, spec.K) if use_signs else None
+    prep = oracle.prepare_weights(W, c, v)
+    h = q.prepare_weights(dev_bf16(W), dev_bf16(b), torch.from_numpy(c).cuda(),
+                          torch.from_numpy(v).cuda() if v is not None else None, c8=True)
+    return dict(W=W, b=b, prep=prep, h=h)
+
+
+@pytest.mark.parametrize("K,N,signs", [(1024, 128, False), (1024, 1024, True), (4096, 256, True), (4096, 1024, False)])
+def test_prepare_weights_c8_parity(K, N, signs):
+    spec = workload.LinearSpec("w", K, N, workload.DIST_GELU if K == 4096 else workload.DIST_NORMAL, 7, 3)
+    L = make_layer(spec, signs)
+    assert np.array_equal(L["h"].view_c8().cpu().numpy(), L["prep"]["wq"])          # one code per byte
+    assert np.array_equal(L["h"].view()["wq"].cpu().numpy(), L["prep"]["wq_packed"])  # the packed copy is still there
+    assert np.array_equal(L["h"].view()["w_scale"].cpu().numpy(), L["prep"]["w_scale"])
+    assert L["h"].device_status() == 0
+
+
+@pytest.mark.parametrize("K", [1024, 4096])
+@pytest.mark.parametrize("M", [1, 5, 127, 129, 1374])
+def test_rotate_smooth_quantize_c8_parity(K, M):
+    spec = workload.LinearSpec("a", K, 128, workload.DIST_GELU if K == 4096 else workload.DIST_NORMAL, 1, 1)
+    L = make_layer(spec, use_signs=True)
+    X = spec.x_rows(0, M)
+    codes, scales = oracle.rotate_smooth_quantize(X, L["prep"]["amul"], 0)
+    Xq8, a_scale = q.rotate_smooth_quantize_c8(L["h"], dev_bf16(X))
+    assert np.array_equal(Xq8.cpu().numpy(), codes)
+    assert np.array_equal(a_scale.cpu().numpy(), scales)
+
+
+@pytest.mark.parametrize("K", [1024, 4096])
+def test_rotate_smooth_quantize_c8_edge_rows(K):
+    spec = workload.LinearSpec("e", K, 128, workload.DIST_NORMAL, 2, 0)
+    L = make_layer(spec)
+    X = spec.x_rows(0, 8)
+    X[0] = 0                                    # all-zero row -> codes 0, floor scale
+    X[1] = 0
+    X[1, K // 3] = 0x4580                       # single spike
+    X[2] = 0
+    X[2, 0] = 0x7F7F                            # one element at the largest finite bf16
+    X[3] = 0
+    X[3, 0] = 0xFF7F                            # and its negative
+    X[4, :] = 0x3F80                            # all ones: the transform concentrates everything in channel 0
+    X[5, ::2] = 0x3F80
+    X[5, 1::2] = 0xBF80                         # alternating signs
+    codes, scales = oracle.rotate_smooth_quantize(X, L["prep"]["amul"], 0)
+    Xq8, a_scale = q.rotate_smooth_quantize_c8(L["h"], dev_bf16(X))
+    assert np.array_equal(Xq8.cpu().numpy(), codes)
+    assert np.array_equal(a_scale.cpu().numpy(), scales)
+    assert not codes[0].any() and codes.min() >= -7 and codes.max() <= 7
+
+
+def test_c8_strided_input_empty_batch_and_missing_copy():
+    spec = workload.LinearSpec("s", 1024, 128, workload.DIST_NORMAL, 4, 0)
+    L = make_layer(spec)
+    X = spec.x_rows(0, 37)
+    wide = torch.zeros((37, 1024 + 64), dtype=torch.bfloat16, device="cuda")
+    wide[:, :1024] = dev_bf16(X)
+    Xq8, a_scale = q.rotate_smooth_quantize_c8(L["h"], wide[:, :1024])
+    codes, scales = oracle.rotate_smooth_quantize(X, L["prep"]["amul"], 0)
+    assert np.array_equal(Xq8.cpu().numpy(), codes)
+    Ywide = torch.zeros((37, 128 + 8), dtype=torch.bfloat16, device="cuda")
+    q.w4a4_linear_c8(L["h"], Xq8, a_scale, Y=Ywide[:, :128])
+    want = oracle.epilogue(oracle.gemm_i32(codes, L["prep"]["wq"]), scales, L["prep"]["w_scale"], L["b"])
+    assert assert_bf16_within_one_ulp(host_bits(Ywide[:, :128]), want) == 0.0
+    assert not Ywide[:, 128:].any()                                   # nothing written past N
+    e = torch.empty((0, 1024), dtype=torch.bfloat16, device="cuda")
+    Xq0, s0 = q.rotate_smooth_quantize_c8(L["h"], e)
+    assert q.w4a4_linear_c8(L["h"], Xq0, s0).shape == (0, 128)
+    assert L["h"].device_status() == 0
+    # a handle prepared without the one-code-per-byte copy refuses the c8 GEMM
+    plain = q.prepare_weights(dev_bf16(L["W"]), None, torch.ones(1024, device="cuda"), None)
+    assert plain.view_c8() is None
+    with pytest.raises(q.QvggtError) as err:
+        q.w4a4_linear_c8(plain, Xq8, a_scale)
+    assert err.value.status == -4
+
+
+@pytest.mark.parametrize("K,N,M", [(1024, 128, 1), (1024, 256, 127), (1024, 1024, 129), (4096, 256, 300),
+                                   (1024, 384, 257), (4096, 1024, 1374), (1024, 3072, 2500)])
+def test_w4a4_linear_c8_parity(K, N, M):
+    spec = workload.LinearSpec("g", K, N, workload.DIST_GELU if K == 4096 else workload.DIST_NORMAL, 9, 2)
+    L = make_layer(spec, use_signs=(N == 256))
+    X = spec.x_rows(0, M)
+    ref = oracle.w4a4_linear(X, L["prep"], L["b"], 0)
+    Xq8, a_scale = q.rotate_smooth_quantize_c8(L["h"], dev_bf16(X))
+    acc = torch.full((M, N), -123456, dtype=torch.int32, device="cuda")
+    Y = q.w4a4_linear_c8(L["h"], Xq8, a_scale, acc_debug=acc)
+    Y2 = q.w4a4_linear_c8(L["h"], Xq8, a_scale)                         # the production instantiation (no dump)
+    assert L["h"].device_status() == 0
+    assert np.array_equal(Xq8.cpu().numpy(), ref["xq"])
+    assert np.array_equal(acc.cpu().numpy(), ref["acc"])               # int32 sums bit-exact
+    assert assert_bf16_within_one_ulp(host_bits(Y), ref["y"]) == 0.0
+    assert np.array_equal(host_bits(Y2), host_bits(Y))
+
+
+def test_w4a4_linear_c8_extreme_codes():
+    """Codes of magnitude 7 everywhere: the sums reach +-49 K, the largest possible; plus a zero token."""
+    K, N, M = 4096, 128, 130
+    W = np.zeros((N, K), np.uint16)
+    W[np.arange(N), np.arange(N)] = 0x3F80       # row n = e_n: its rotation is row n of H_K, so every code is +-7
+    h = q.prepare_weights(dev_bf16(W), None, torch.ones(K, device="cuda"), None, c8=True)
+    wq = h.view_c8().cpu().numpy()
+    assert np.all(np.abs(wq) == 7)
+    xq = np.ascontiguousarray(np.tile(wq, (2, 1))[:M])                  # token m carries the pattern of channel m % N
+    xq[1] = -xq[1]
+    xq[2] = 0
+    a_np = np.full(M, 0.5, np.float32)
+    acc = torch.zeros((M, N), dtype=torch.int32, device="cuda")
+    Y = q.w4a4_linear_c8(h, torch.from_numpy(xq).cuda(), torch.from_numpy(a_np).cuda(), acc_debug=acc)
+    want_acc = oracle.gemm_i32(xq, wq)
+    assert want_acc[0, 0] == 49 * K and want_acc[1, 1] == -49 * K and not want_acc[2].any()
+    assert np.array_equal(acc.cpu().numpy(), want_acc)
+    want = oracle.epilogue(want_acc, a_np, h.view()["w_scale"].cpu().numpy(), None)
+    assert assert_bf16_within_one_ulp(host_bits(Y), want) == 0.0
+    assert h.device_status() == 0
+
+
+def test_c8_config1_single_frame_proj():
+    spec = workload.LinearSpec("proj", 1024, 1024, workload.DIST_NORMAL, 0, 1)
+    L = make_layer(spec, calib_rows=workload.TOKENS_PER_FRAME)
+    M = workload.TOKENS_PER_FRAME
+    X = spec.x_rows(0, M)
+    ref = oracle.w4a4_linear(X, L["prep"], L["b"], 0)
+    Xq8, a_scale = q.rotate_smooth_quantize_c8(L["h"], dev_bf16(X))
+    acc = torch.zeros((M, 1024), dtype=torch.int32, device="cuda")
+    Y = q.w4a4_linear_c8(L["h"], Xq8, a_scale, acc_debug=acc)
+    assert np.array_equal(Xq8.cpu().numpy(), ref["xq"])
+    assert np.array_equal(a_scale.cpu().numpy(), ref["a_scale"])
+    assert np.array_equal(acc.cpu().numpy(), ref["acc"])
+    assert assert_bf16_within_one_ulp(host_bits(Y), ref["y"]) == 0.0
