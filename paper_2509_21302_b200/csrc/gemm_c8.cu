@@ -143,26 +143,28 @@ gemm_c8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 const float *wsb = s_ws + b * BN + cpart * C::CW;
                 const float *bsb = s_bs + b * BN + cpart * C::CW;
                 constexpr int NCH = C::CW / 32;
-#pragma unroll 1
+                // the warp's whole share of the accumulator goes to registers first, so that tensor memory is
+                // handed back to the MMA thread a few hundred cycles after the tile completed, not after the
+                // conversions and stores of the first chunks
+                uint32_t raw[NCH][32];
+#pragma unroll
+                for (int c = 0; c < NCH; ++c)
+                    ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + b * BN + cpart * C::CW + c * 32, raw[c]);
+                ptx::tmem_ld_wait();
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive_cluster(leader_tempty + 8 * b);
+#pragma unroll
                 for (int c = 0; c < NCH; ++c) {
                     const int col = c * 32;                               // within this warp's columns
-                    uint32_t raw[32];
-                    ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + b * BN + cpart * C::CW + col, raw);
-                    ptx::tmem_ld_wait();
-                    if (c == NCH - 1) {
-                        // last read of this accumulator: hand it back to the MMA thread before the math
-                        ptx::tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive_cluster(leader_tempty + 8 * b);
-                    }
                     if (cols_ok) {
                         uint32_t out[16];
 #pragma unroll
                         for (int j = 0; j < 32; j += 4) {
                             const ulonglong2 w2 = *reinterpret_cast<const ulonglong2 *>(wsb + col + j);
                             const ulonglong2 b2 = *reinterpret_cast<const ulonglong2 *>(bsb + col + j);
-                            uint64_t z01 = ptx::f32x2_pack(static_cast<float>(static_cast<int>(raw[j])), static_cast<float>(static_cast<int>(raw[j + 1])));
-                            uint64_t z23 = ptx::f32x2_pack(static_cast<float>(static_cast<int>(raw[j + 2])), static_cast<float>(static_cast<int>(raw[j + 3])));
+                            uint64_t z01 = ptx::f32x2_pack(static_cast<float>(static_cast<int>(raw[c][j])), static_cast<float>(static_cast<int>(raw[c][j + 1])));
+                            uint64_t z23 = ptx::f32x2_pack(static_cast<float>(static_cast<int>(raw[c][j + 2])), static_cast<float>(static_cast<int>(raw[c][j + 3])));
                             // fl(fl(float(acc) * fl(a_scale * w_scale)) + bias), every operation rounded to nearest.
                             // The additions are scalar intrinsics: a packed multiply feeding a packed add was
                             // observed to be contracted into one fused operation (single rounding).
@@ -187,7 +189,7 @@ gemm_c8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                         if (DUMP && acc_debug && row_ok) {
                             uint4 *dbg = reinterpret_cast<uint4 *>(acc_debug + (long long)gm * N + n0 + col);
 #pragma unroll
-                            for (int q = 0; q < 8; ++q) dbg[q] = make_uint4(raw[4 * q], raw[4 * q + 1], raw[4 * q + 2], raw[4 * q + 3]);
+                            for (int q = 0; q < 8; ++q) dbg[q] = make_uint4(raw[c][4 * q], raw[c][4 * q + 1], raw[c][4 * q + 2], raw[c][4 * q + 3]);
                         }
                         ptx::fence_proxy_async_smem();          // staging writes -> visible to the TMA engine
                         __syncwarp();
