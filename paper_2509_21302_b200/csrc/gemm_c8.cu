@@ -105,6 +105,10 @@ gemm_c8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     ptx::cluster_sync();                     // the leader's barriers exist before the peer's loads signal them
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *s_tmem;
+    // everything above touched only kernel parameters and on-chip state: it may overlap the tail of the previous
+    // kernel in the stream; the operands (and the output buffer) may not be touched before that kernel is done
+    ptx::grid_launch_dependents();
+    ptx::grid_dependency_wait();
 
     if (warp < EPI_WARPS) {
         // ------------------------------------------------------------ epilogue
@@ -280,9 +284,11 @@ cudaError_t launch(const qvggt_weights *w, const signed char *Xq8, const float *
     using C = Cfg<EPI_WARPS>;
     static int max_workers = 0;       // per process; one GPU type per process
     cudaError_t e;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;      // see grid_dependency_wait()
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     if (!max_workers) {
         e = cudaFuncSetAttribute(gemm_c8_kernel<EPI_WARPS, DUMP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::DYN_SMEM);
         if (e != cudaSuccess) return e;
@@ -290,7 +296,7 @@ cudaError_t launch(const qvggt_weights *w, const signed char *Xq8, const float *
         probe.gridDim = dim3(2 * qvggt_sm_count());
         probe.blockDim = dim3(C::THREADS);
         probe.dynamicSmemBytes = C::DYN_SMEM;
-        probe.attrs = &attr;
+        probe.attrs = attr;
         probe.numAttrs = 1;
         int clusters = 0;
         e = cudaOccupancyMaxActiveClusters(&clusters, gemm_c8_kernel<EPI_WARPS, DUMP>, &probe);
@@ -311,8 +317,8 @@ cudaError_t launch(const qvggt_weights *w, const signed char *Xq8, const float *
     cfg.blockDim = dim3(C::THREADS);
     cfg.dynamicSmemBytes = C::DYN_SMEM;
     cfg.stream = st;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, gemm_c8_kernel<EPI_WARPS, DUMP>, map_x, map_w, map_y, a_scale, (const float *)w->w_scale,
                               (const uint16_t *)w->bias, acc_debug, M, N, K, w->status);
 }

@@ -221,6 +221,10 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
 
     const long long stride = (long long)gridDim.x * G::ROWS;
     long long row = (long long)blockIdx.x * G::ROWS + slot;
+    // the blocks may have become resident before the previous kernel in the stream finished (programmatic
+    // dependent launch): no global memory is touched before that kernel is done
+    ptx::grid_launch_dependents();
+    ptx::grid_dependency_wait();
     if (row < M) {
         const unsigned char *src = reinterpret_cast<const unsigned char *>(X + row * ldx);
 #pragma unroll
@@ -422,26 +426,43 @@ cudaError_t qvggt_launch_multipliers(const float *c, const signed char *v, int K
     return cudaGetLastError();
 }
 
+namespace {
+
+// Launch with programmatic stream serialization allowed: the blocks may become resident while the previous
+// kernel of the stream drains (they wait in grid_dependency_wait() before touching global memory).
+template <int LOGT, int GROUP, bool C8>
+cudaError_t launch_sq(const uint16_t *x, long long ldx, int M, const float *mul, unsigned char *out, float *scales,
+                      cudaStream_t st)
+{
+    using G = SqGeom<LOGT>;
+    static bool configured = false;       // per process and instantiation
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(rsq_sq_kernel<LOGT, GROUP, C8>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(rsq_grid(M, G::ROWS, LOGT == 5 ? 4 : 3));
+    cfg.blockDim = dim3(G::CTA_THREADS);
+    cfg.dynamicSmemBytes = G::SMEM;
+    cfg.stream = st;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, rsq_sq_kernel<LOGT, GROUP, C8>, x, ldx, M, mul, out, scales);
+}
+
+}  // namespace
+
 cudaError_t qvggt_launch_rsq_c8(const void *X, long long ldx, int M, int K, const float *mul, signed char *Xq8,
                                 float *scales, cudaStream_t st)
 {
     if (M == 0) return cudaSuccess;
     const uint16_t *x = static_cast<const uint16_t *>(X);
     unsigned char *out = reinterpret_cast<unsigned char *>(Xq8);
-    static bool configured = false;       // per process
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(rsq_sq_kernel<6, 0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SqGeom<6>::SMEM);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
-    if (K == 1024) {
-        using G = SqGeom<5>;
-        rsq_sq_kernel<5, 0, true><<<rsq_grid(M, G::ROWS, 4), G::CTA_THREADS, G::SMEM, st>>>(x, ldx, M, mul, out, scales);
-    } else {
-        using G = SqGeom<6>;
-        rsq_sq_kernel<6, 0, true><<<rsq_grid(M, G::ROWS, 3), G::CTA_THREADS, G::SMEM, st>>>(x, ldx, M, mul, out, scales);
-    }
-    return cudaGetLastError();
+    return K == 1024 ? launch_sq<5, 0, true>(x, ldx, M, mul, out, scales, st) : launch_sq<6, 0, true>(x, ldx, M, mul, out, scales, st);
 }
 
 cudaError_t qvggt_launch_rsq(const void *X, long long ldx, int M, int K, const float *mul, int group,
@@ -449,25 +470,9 @@ cudaError_t qvggt_launch_rsq(const void *X, long long ldx, int M, int K, const f
 {
     if (M == 0) return cudaSuccess;
     const uint16_t *x = static_cast<const uint16_t *>(X);
-    static bool configured = false;       // per process
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(rsq_sq_kernel<6, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SqGeom<6>::SMEM);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(rsq_sq_kernel<6, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, SqGeom<6>::SMEM);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
-    if (K == 1024) {
-        using G = SqGeom<5>;
-        const int grid = rsq_grid(M, G::ROWS, 4);
-        if (group == 128) rsq_sq_kernel<5, 128><<<grid, G::CTA_THREADS, G::SMEM, st>>>(x, ldx, M, mul, Xq, scales);
-        else rsq_sq_kernel<5, 0><<<grid, G::CTA_THREADS, G::SMEM, st>>>(x, ldx, M, mul, Xq, scales);
-    } else {
-        using G = SqGeom<6>;
-        const int grid = rsq_grid(M, G::ROWS, 3);
-        if (group == 128) rsq_sq_kernel<6, 128><<<grid, G::CTA_THREADS, G::SMEM, st>>>(x, ldx, M, mul, Xq, scales);
-        else rsq_sq_kernel<6, 0><<<grid, G::CTA_THREADS, G::SMEM, st>>>(x, ldx, M, mul, Xq, scales);
-    }
-    return cudaGetLastError();
+    if (K == 1024)
+        return group == 128 ? launch_sq<5, 128, false>(x, ldx, M, mul, Xq, scales, st) : launch_sq<5, 0, false>(x, ldx, M, mul, Xq, scales, st);
+    return group == 128 ? launch_sq<6, 128, false>(x, ldx, M, mul, Xq, scales, st) : launch_sq<6, 0, false>(x, ldx, M, mul, Xq, scales, st);
 }
 
 cudaError_t qvggt_launch_colmax(const void *X, int M, int K, float *colmax, cudaStream_t st)

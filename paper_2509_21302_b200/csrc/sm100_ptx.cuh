@@ -366,6 +366,15 @@ __device__ __forceinline__ void prefetch_tensormap(const void *tmap)
     asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// A kernel launched with the programmatic-stream-serialization attribute may become resident while its
+// predecessor in the stream is still running.  grid_dependency_wait() returns once every prerequisite grid has
+// completed and its memory is visible: nothing a predecessor may have written is read, and nothing is written,
+// before it.  (Without the attribute it returns at once.)  grid_launch_dependents() lets the successor's blocks
+// start their own preamble as soon as every block of this grid has called it.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------- packed fp32 pairs (one issue slot for two IEEE operations)
 __device__ __forceinline__ float2 mul_f32x2(float2 a, float2 b)
 {
