@@ -43,6 +43,7 @@ def _L():
             "orc_fwht_f64": [vp, i32],
             "orc_multipliers": [vp, vp, i32, vp, vp],
             "orc_rotate_smooth_quantize": [vp, i64, i64, i32, vp, i32, vp, vp],
+            "orc_rotate_smooth_quantize_bits": [vp, i64, i64, i32, vp, i32, i32, vp, vp],
             "orc_pack_int4": [vp, i64, i32, vp],
             "orc_unpack_int4": [vp, i64, i32, vp],
             "orc_gemm_i32": [vp, vp, i64, i32, i32, i32, vp],
@@ -102,16 +103,21 @@ def multipliers(c: np.ndarray, v: np.ndarray | None = None):
     return amul, wmul
 
 
-def rotate_smooth_quantize(X: np.ndarray, mul: np.ndarray, group: int = 0):
-    """X bf16 bits [M, K] -> (codes int8 [M, K], scales fp32 [M] or [M, K/group])."""
-    assert X.dtype == np.uint16 and X.ndim == 2 and X.strides[1] == 2
+def rotate_smooth_quantize(X: np.ndarray, mul: np.ndarray, group: int = 0, bits: int = 4):
+    """X bf16 bits [M, K] -> (codes int8 [M, K], scales fp32 [M] or [M, K/group]).
+    bits: N of Eq. "quantization" (4 = the W4A4 setting, 8 = the paper's W8A8 setting)."""
+    assert X.dtype == np.uint16 and X.ndim == 2 and X.strides[1] == 2 and 2 <= bits <= 8
     M, K = X.shape
     mul = _c(mul, np.float32)
     G = K // group if group else 1
     codes = np.empty((M, K), np.int8)
     scales = np.empty((M, G), np.float32)
-    _L().orc_rotate_smooth_quantize(X.ctypes.data, X.strides[0] // 2, M, K, mul.ctypes.data, group,
-                                    codes.ctypes.data, scales.ctypes.data)
+    if bits == 4:
+        _L().orc_rotate_smooth_quantize(X.ctypes.data, X.strides[0] // 2, M, K, mul.ctypes.data, group,
+                                        codes.ctypes.data, scales.ctypes.data)
+    else:
+        _L().orc_rotate_smooth_quantize_bits(X.ctypes.data, X.strides[0] // 2, M, K, mul.ctypes.data, group, bits,
+                                             codes.ctypes.data, scales.ctypes.data)
     return codes, (scales if group else scales.reshape(M))
 
 
@@ -200,20 +206,20 @@ def bf16_to_f32(bits: np.ndarray) -> np.ndarray:
     return (np.asarray(bits).astype(np.uint32) << 16).view(np.float32)
 
 
-def prepare_weights(W: np.ndarray, c: np.ndarray, v: np.ndarray | None = None):
-    """Offline weight path: fold H and diag(c) into W, quantize per output channel.
+def prepare_weights(W: np.ndarray, c: np.ndarray, v: np.ndarray | None = None, bits: int = 4):
+    """Offline weight path: fold H and diag(c) into W, quantize per output channel (N = bits).
 
-    -> dict(wq codes int8 [N, K], wq_packed uint8 [N, K/2], w_scale fp32 [N], amul fp32 [K], wmul fp32 [K])
+    -> dict(wq codes int8 [N, K], wq_packed uint8 [N, K/2] (bits = 4 only), w_scale fp32 [N], amul fp32 [K], wmul fp32 [K])
     """
     amul, wmul = multipliers(c, v)
-    wq, w_scale = rotate_smooth_quantize(W, wmul, 0)
-    return dict(wq=wq, wq_packed=pack_int4(wq), w_scale=w_scale, amul=amul, wmul=wmul)
+    wq, w_scale = rotate_smooth_quantize(W, wmul, 0, bits)
+    return dict(wq=wq, wq_packed=pack_int4(wq) if bits == 4 else None, w_scale=w_scale, amul=amul, wmul=wmul, bits=bits)
 
 
 def w4a4_linear(X: np.ndarray, prepared: dict, bias: np.ndarray | None, group: int = 0, timings: dict | None = None):
     """Online path for activations X (bf16 bits [M, K]) -> dict(xq, a_scale, acc, y)."""
     t0 = time.perf_counter()
-    xq, a_scale = rotate_smooth_quantize(X, prepared["amul"], group)
+    xq, a_scale = rotate_smooth_quantize(X, prepared["amul"], group, prepared.get("bits", 4))
     t1 = time.perf_counter()
     acc = gemm_i32(xq, prepared["wq"], group)
     t2 = time.perf_counter()

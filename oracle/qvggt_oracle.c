@@ -92,22 +92,26 @@ void orc_multipliers(const float *c, const int8_t *v, int K, float *amul, float 
 }
 
 /*
- * Rotate -> smooth -> symmetric 4-bit quantize, row by row (Eq. "quantization" with N = 4:
- * Delta = max|y| / 7, q = clamp(round(y / Delta), -8, 7)).
+ * Rotate -> smooth -> symmetric N-bit quantize, row by row (Eq. "quantization":
+ * Delta = max|y| / (2^(N-1) - 1), q = clamp(round(y / Delta), -2^(N-1), 2^(N-1) - 1)); N = 4 is the
+ * W4A4 setting, N = 8 the paper's W8A8 setting.
  *   X      bf16 bits [M, K], row stride ldx elements
  *   mul    fp32 [K] (amul for activations, wmul for weight rows)
  *   group  scale granularity along K: 0 = one scale per row (the paper's token-wise /
  *          out-channel-wise setting); g > 0 = one scale per g consecutive rotated channels
- *   codes  int8 [M, K], values in [-8, 7] (in fact [-7, 7])
+ *   bits   N (2..8)
+ *   codes  int8 [M, K], values in [-2^(N-1), 2^(N-1) - 1] (in fact never the most negative code)
  *   scales fp32 [M, K/group]
  * Reading of the unspecified points: round() is round-half-to-even; y/Delta is evaluated as the
- * exact product y * fl(7/amax) rounded once to an integer; an all-zero group gets amax = 1e-8.
+ * exact product y * fl(qmax/amax) rounded once to an integer; an all-zero group gets amax = 1e-8.
  */
-void orc_rotate_smooth_quantize(const uint16_t *X, int64_t ldx, int64_t M, int K, const float *mul,
-                                int group, int8_t *codes, float *scales)
+void orc_rotate_smooth_quantize_bits(const uint16_t *X, int64_t ldx, int64_t M, int K, const float *mul,
+                                     int group, int bits, int8_t *codes, float *scales)
 {
     int G = group > 0 ? K / group : 1;
     int glen = group > 0 ? group : K;
+    const float qmax = (float)((1 << (bits - 1)) - 1);
+    const double lo = -(double)(1 << (bits - 1)), hi = (double)qmax;
 #pragma omp parallel
     {
         float *u = (float *)malloc(sizeof(float) * (size_t)K);
@@ -125,20 +129,27 @@ void orc_rotate_smooth_quantize(const uint16_t *X, int64_t ldx, int64_t M, int K
                     if (a > amax) amax = a;
                 }
                 if (amax < 1e-8f) amax = 1e-8f;
-                float scale = amax / 7.0f;
-                float inv = 7.0f / amax;
+                float scale = amax / qmax;
+                float inv = qmax / amax;
                 scales[m * G + g] = scale;
                 int8_t *q = codes + m * K + g * glen;
                 for (int k = 0; k < glen; ++k) {
                     double r = nearbyint((double)y[k] * (double)inv); /* exact product, one rounding */
-                    if (r < -8.0) r = -8.0;
-                    if (r > 7.0) r = 7.0;
+                    if (r < lo) r = lo;
+                    if (r > hi) r = hi;
                     q[k] = (int8_t)r;
                 }
             }
         }
         free(u);
     }
+}
+
+/* The W4A4 setting (N = 4: Delta = max|y| / 7, codes in [-8, 7]). */
+void orc_rotate_smooth_quantize(const uint16_t *X, int64_t ldx, int64_t M, int K, const float *mul,
+                                int group, int8_t *codes, float *scales)
+{
+    orc_rotate_smooth_quantize_bits(X, ldx, M, K, mul, group, 4, codes, scales);
 }
 
 /* Canonical packed layout: byte i of a row = code 2i in bits 0-3, code 2i+1 in bits 4-7 (two's complement). */

@@ -321,7 +321,6 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
         for (int g = 0; g < NG; ++g) {
             am[g] = fmaxf(am[g], 1e-8f);
             const float inv = __fdiv_rn(7.0f, am[g]);
-#pragma unroll
             const uint64_t inv2 = ptx::f32x2_pack(inv, inv), magic2 = ptx::f32x2_pack(12582912.0f, 12582912.0f);
 #pragma unroll
             for (int k = g * GREGS; k < (g + 1) * GREGS; k += 2) {

@@ -172,6 +172,49 @@ def test_quantizer_error_bound_and_range(K, group):
     assert np.all(np.sign(qg[hit]) == np.sign(yg[hit]))
 
 
+@pytest.mark.parametrize("bits", [8, 6, 4])
+def test_nbit_quantizer_error_bound_range_and_independent_rounding(bits):
+    """Eq. "quantization" for general N (N = 8 is the W8A8 setting): Delta = max|x| / (2^(N-1) - 1), error at most
+    Delta / 2, the absolute maximum maps to +-(2^(N-1) - 1), the most negative code never appears; away from ties
+    the codes equal an independent float64 evaluation of round(y / Delta)."""
+    K, qmax = 1024, 2 ** (bits - 1) - 1
+    spec = workload.LinearSpec("t", K, 8, workload.DIST_NORMAL, 23, 0)
+    X = spec.x_rows(0, 12)
+    c = workload.loguniform_f32(23, 5, K, 0.05, 20)
+    amul, _ = oracle.multipliers(c, workload.signs_i8(23, 6, K))
+    codes, scales = oracle.rotate_smooth_quantize(X, amul, 0, bits)
+    y = _rotated_y(X, amul).astype(np.float64)
+    q, s_ = codes.astype(np.float64), scales.astype(np.float64)[:, None]
+    assert np.all(np.abs(y - s_ * q) <= s_ / 2 * (1 + 2.0 ** -20))
+    amax = np.abs(y).max(axis=1, keepdims=True)
+    assert np.array_equal(scales, (amax[:, 0].astype(np.float32) / np.float32(qmax)))
+    assert codes.min() >= -qmax and codes.max() <= qmax
+    hit = np.abs(y) == amax
+    assert np.all(np.abs(q[hit]) == qmax) and np.all(np.sign(q[hit]) == np.sign(y[hit]))
+    t = y * qmax / amax                                    # float64, a different evaluation order
+    clear = np.abs(t - np.floor(t) - 0.5) > 1e-4           # not within 1e-4 of a rounding boundary
+    assert clear.mean() > 0.99
+    assert np.array_equal(q[clear], np.rint(t)[clear])
+    if bits == 4:                                          # the general routine at N = 4 is the W4A4 routine
+        c4, s4 = oracle.rotate_smooth_quantize(X, amul, 0)
+        assert np.array_equal(c4, codes) and np.array_equal(s4, scales)
+
+
+def test_8bit_round_half_to_even_and_extremes():
+    """N = 8 on exactly representable values: a unit vector rotates to all ones, so y equals the multiplier vector;
+    with amax = 127 the factor 127/amax is 1 and y itself is rounded: ties go to the even integer, +-127 stay,
+    nothing reaches -128."""
+    K = 16
+    y = np.array([127.0, -127.0, 0.5, 1.5, 2.5, -0.5, -1.5, -2.5, 126.5, -126.5, 63.5, 64.5, 0.0, 1.0, -100.5, 99.5], np.float32)
+    want = np.array([127, -127, 0, 2, 2, 0, -2, -2, 126, -126, 64, 64, 0, 1, -100, 100], np.int8)
+    X = np.zeros((1, K), np.uint16)
+    X[0, 0] = 0x3F80                                              # 1.0: its transform is the all-ones row of H_16
+    assert np.array_equal(oracle.fwht_f32(workload.bf16_to_f32(X))[0], np.ones(K, np.float32))
+    codes, scales = oracle.rotate_smooth_quantize(X, y, 0, 8)
+    assert scales[0] == np.float32(1.0)
+    assert np.array_equal(codes[0], want)
+
+
 def test_round_half_to_even_on_handbuilt_ties():
     tab = load_table("round_ties.txt")
     y, want = tab[:, 0], tab[:, 1].astype(np.int8)
