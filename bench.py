@@ -57,9 +57,10 @@ class Path:
 
     def __init__(self, q, torch, fmt: str):
         self.fmt = fmt
-        self.code_bytes = 1.0 if fmt == "c8" else 0.5
-        if fmt == "c8":
-            self.prepare = lambda W, b, c: q.prepare_weights(W, b, c, None, c8=True)
+        self.code_bytes = 0.5 if fmt == "packed" else 1.0
+        self.bits = 8 if fmt == "w8a8" else 4
+        if fmt in ("c8", "w8a8"):
+            self.prepare = lambda W, b, c: q.prepare_weights(W, b, c, None, c8=True, bits=self.bits)
             self.rsq = lambda h, x, xq, a: q.rotate_smooth_quantize_c8(h, x, xq, a)
             self.gemm = lambda h, xq, a, y: q.w4a4_linear_c8(h, xq, a, y)
             self.new_xq = lambda M, K: torch.empty((M, K), dtype=torch.int8, device="cuda")
@@ -344,16 +345,18 @@ def run_ours(args, rank, world, local_rank):
                              "rsq_us": round(t_r * 1e6, 2), "rsq_gbs": round(rsq_bytes(M, s.K, cb) / t_r / 1e9, 1),
                              "rsq_hbm_frac": round(rsq_bytes(M, s.K, cb) / t_r / 1e9 / peaks["hbm_gbs"], 4)}
     out = {
-        "metric": "w4a4_linear_tops", "value": tops, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
+        "metric": "w4a4_linear_tops" if path.bits == 4 else "w8a8_linear_tops", "value": tops, "unit": "TOPS", "n_gpus": world,
+        "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "int4 x int4 -> int32 (fp32 rotation and scales)", "data": "synthetic",
+        "vs_baseline": None, "dtype": f"int{path.bits} x int{path.bits} -> int32 (fp32 rotation and scales)", "data": "synthetic",
         "tokens_per_s": world * M / (ms_per_step * 1e-3),
         "config": {"workload": "aggregator block, 4 linears (qkv/proj/fc1/fc2), 8 frames M=10992 per GPU (BASELINE configs[1])",
                    "l2": f"step working set ~400 MB > 126 MB L2; {NBUF} buffer sets alternated per step",
                    "timed": "rotate-smooth-quantize + W4A4 GEMM/epilogue per linear; weight prep offline; one event pair "
                             "around the K steps; the per-kernel durations behind roofline / per_layer come from a second pass "
                             "of the same steps with an event after every launch",
-                   "code_format": "int4 codes one per byte between the kernels (c8)" if path.fmt == "c8" else "int4 codes packed two per byte"},
+                   "code_format": {"c8": "int4 codes one per byte between the kernels (c8)", "packed": "int4 codes packed two per byte",
+                                   "w8a8": "W8A8: int8 codes (Eq. quantization with N = 8), one per byte"}[path.fmt]},
         "clocks": clocks,
         "gpu_launches": int(2 * len(layers) * args.steps),
         "e2e": {"value": world * ops_step / (e2e_ms * 1e-3) / 1e12, "unit": "TOPS", "ms_per_step": e2e_ms,
@@ -485,8 +488,9 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--ref-rows", type=int, default=512, help="token rows per step of the oracle arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--format", choices=["c8", "packed"], default="c8",
-                    help="storage of the int4 codes between the kernels: c8 = one per byte (default), packed = two per byte")
+    ap.add_argument("--format", choices=["c8", "packed", "w8a8"], default="c8",
+                    help="storage of the int4 codes between the kernels: c8 = one per byte (default), packed = two per byte; "
+                         "w8a8 = the paper's 8-bit setting through the same kernels (not the headline metric)")
     ap.add_argument("--workload", choices=["block", "rsq_sweep", "stack"], default="block",
                     help="block = BASELINE configs[1] (the default, the contract line); rsq_sweep = configs[2]")
     args = ap.parse_args()

@@ -65,7 +65,8 @@ typedef enum {
  *   bias_bf16 [N] bf16 or NULL (no bias)
  *   smooth_c  [K] fp32, finite and > 0
  *   sign_v    [K] int8 of +1/-1, or NULL (all +1)
- *   flags     0, or QVGGT_PREP_C8 to keep an extra int8 [N, K] copy of the codes for the *_c8 entry points
+ *   flags     0, QVGGT_PREP_C8 to keep an extra int8 [N, K] copy of the codes for the *_c8 entry points, or
+ *             QVGGT_PREP_W8A8 for 8-bit codes (see the *_c8 entry points)
  *   out       receives a new handle (device memory is allocated here, on the current device);
  *             release it with qvggt_free_weights.  The handle is bound to that device.
  * Work is enqueued on the stream; the inputs may be released once the stream has passed this call.
@@ -111,8 +112,15 @@ int qvggt_w4a4_linear(const qvggt_weights_t *w, const unsigned char *Xq, const f
  *   Xq8      int8 [M, K], one code per byte in [-7, 7], natural element order, 16-byte aligned
  *   a_scale  fp32 [M]
  *   Y_bf16, ldy, acc_debug (int32 [M, N]) as for qvggt_w4a4_linear with group 0
+ *
+ * W8A8 (the paper's other setting, Eq. "quantization" with N = 8: Delta = max|x| / 127, codes in [-127, 127]) uses the
+ * same two calls: a handle prepared with QVGGT_PREP_W8A8 holds 8-bit weight codes (one per byte only: there is no
+ * packed copy, and the packed entry points refuse it with QVGGT_ERR_UNSUPPORTED), qvggt_rotate_smooth_quantize_c8
+ * then quantizes the activations to 8 bits, and qvggt_w4a4_linear_c8 multiplies them: the integer sums stay below
+ * 2^31 (127^2 * 4096), the epilogue is the same.
  */
 #define QVGGT_PREP_C8 1
+#define QVGGT_PREP_W8A8 2
 int qvggt_rotate_smooth_quantize_c8(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M,
                                     signed char *Xq8, float *a_scale, void *cuda_stream);
 int qvggt_w4a4_linear_c8(const qvggt_weights_t *w, const signed char *Xq8, const float *a_scale, int M,
@@ -129,8 +137,9 @@ void qvggt_free_weights(qvggt_weights_t *w);
 int qvggt_weights_view(const qvggt_weights_t *w, const unsigned char **Wq, const float **w_scale,
                        const float **amul, const void **bias_bf16, int *N, int *K);
 
-/* Device pointer to the int8 [N, K] copy of the codes (NULL if the handle was prepared without QVGGT_PREP_C8). */
-int qvggt_weights_view_c8(const qvggt_weights_t *w, const signed char **Wq8);
+/* Device pointer to the int8 [N, K] copy of the codes (NULL if the handle was prepared without QVGGT_PREP_C8 or
+ * QVGGT_PREP_W8A8) and, if `bits` is not NULL, the handle's code width (4 or 8). */
+int qvggt_weights_view_c8(const qvggt_weights_t *w, const signed char **Wq8, int *bits);
 
 /*
  * Synchronises `cuda_stream`, then reads the handle's device status word into *code (HOST pointer):

@@ -23,6 +23,7 @@ EXPORTS = ("qvggt_prepare_weights", "qvggt_rotate_smooth_quantize", "qvggt_w4a4_
            "qvggt_quantize_weights_static", "qvggt_rotate_smooth_quantize_c8", "qvggt_w4a4_linear_c8",
            "qvggt_weights_view_c8")
 PREP_C8 = 1   # QVGGT_PREP_C8: keep an int8 [N, K] copy of the weight codes for the *_c8 entry points
+PREP_W8A8 = 2  # QVGGT_PREP_W8A8: 8-bit codes (one per byte only)
 
 
 class QvggtError(RuntimeError):
@@ -50,7 +51,7 @@ def lib() -> ctypes.CDLL:
         L.qvggt_w4a4_linear.argtypes = [vp, vp, vp, i32, i32, vp, i64, vp, vp]
         L.qvggt_rotate_smooth_quantize_c8.argtypes = [vp, vp, i64, i32, vp, vp, vp]
         L.qvggt_w4a4_linear_c8.argtypes = [vp, vp, vp, i32, vp, i64, vp, vp]
-        L.qvggt_weights_view_c8.argtypes = [vp, ctypes.POINTER(vp)]
+        L.qvggt_weights_view_c8.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(i32)]
         L.qvggt_free_weights.argtypes = [vp]
         L.qvggt_free_weights.restype = None
         L.qvggt_weights_view.argtypes = [vp] + [ctypes.POINTER(vp)] * 4 + [ctypes.POINTER(i32)] * 2
@@ -115,8 +116,9 @@ class Weights:
 
     def view_c8(self) -> torch.Tensor | None:
         """Copy of the int8 [N, K] codes (None if prepared without c8=True)."""
-        p = ctypes.c_void_p()
-        _check(lib().qvggt_weights_view_c8(self.handle, ctypes.byref(p)), "qvggt_weights_view_c8")
+        p, bits = ctypes.c_void_p(), ctypes.c_int()
+        _check(lib().qvggt_weights_view_c8(self.handle, ctypes.byref(p), ctypes.byref(bits)), "qvggt_weights_view_c8")
+        self.bits = bits.value
         if not p.value:
             return None
         return _from_device_ptr(p.value, self.N * self.K, torch.uint8, (self.N, self.K)).view(torch.int8)
@@ -157,9 +159,11 @@ def _from_device_ptr(ptr: int, nbytes: int, dtype: torch.dtype, shape) -> torch.
 
 
 def prepare_weights(W: torch.Tensor, bias: torch.Tensor | None, smooth_c: torch.Tensor,
-                    sign_v: torch.Tensor | None = None, c8: bool = False) -> Weights:
+                    sign_v: torch.Tensor | None = None, c8: bool = False, bits: int = 4) -> Weights:
     """W [N,K] bf16, bias [N] bf16 or None, smooth_c [K] fp32, sign_v [K] int8 (+1/-1) or None.
-    c8: also keep the codes one per byte, as the *_c8 entry points need them."""
+    c8: also keep the codes one per byte, as the *_c8 entry points need them.
+    bits: 4 (W4A4) or 8 (W8A8: one code per byte only; use the *_c8 entry points)."""
+    assert bits in (4, 8)
     assert W.dim() == 2 and W.element_size() == 2 and W.is_contiguous()
     N, K = W.shape
     assert smooth_c.dtype == torch.float32 and smooth_c.numel() == K and smooth_c.is_contiguous()
@@ -168,7 +172,7 @@ def prepare_weights(W: torch.Tensor, bias: torch.Tensor | None, smooth_c: torch.
     if sign_v is not None:
         assert sign_v.dtype == torch.int8 and sign_v.numel() == K and sign_v.is_contiguous()
     h = ctypes.c_void_p()
-    _check(lib().qvggt_prepare_weights(_ptr(W), _ptr(bias), _ptr(smooth_c), _ptr(sign_v), N, K, PREP_C8 if c8 else 0, _stream(),
+    _check(lib().qvggt_prepare_weights(_ptr(W), _ptr(bias), _ptr(smooth_c), _ptr(sign_v), N, K, PREP_W8A8 if bits == 8 else (PREP_C8 if c8 else 0), _stream(),
                                        ctypes.byref(h)), "qvggt_prepare_weights")
     return Weights(h.value, N, K)
 

@@ -36,7 +36,9 @@ extern "C" {
 int qvggt_prepare_weights(const void *W_bf16, const void *bias_bf16, const float *smooth_c, const signed char *sign_v,
                           int N, int K, int flags, void *cuda_stream, qvggt_weights_t **out)
 {
-    if (flags & ~QVGGT_PREP_C8) return QVGGT_ERR_UNSUPPORTED;
+    if (flags & ~(QVGGT_PREP_C8 | QVGGT_PREP_W8A8)) return QVGGT_ERR_UNSUPPORTED;
+    const bool w8 = (flags & QVGGT_PREP_W8A8) != 0;       // 8-bit codes exist one per byte only
+    const bool c8 = w8 || (flags & QVGGT_PREP_C8) != 0;
     if (!out) return QVGGT_ERR_NULL;
     *out = nullptr;
     if (!W_bf16 || !smooth_c) return QVGGT_ERR_NULL;
@@ -49,16 +51,17 @@ int qvggt_prepare_weights(const void *W_bf16, const void *bias_bf16, const float
     if (!w) return QVGGT_ERR_NOMEM;
     w->N = N;
     w->K = K;
+    w->bits = w8 ? 8 : 4;
     w->Wq = nullptr; w->Wq8 = nullptr; w->w_scale = nullptr; w->amul = nullptr; w->bias = nullptr; w->status = nullptr;
     cudaGetDevice(&w->device);
     float *wmul = nullptr;
-    bool ok = cudaMalloc(&w->Wq, (size_t)N * K / 2) == cudaSuccess &&
+    bool ok = (w8 || cudaMalloc(&w->Wq, (size_t)N * K / 2) == cudaSuccess) &&
               cudaMalloc(&w->w_scale, sizeof(float) * N) == cudaSuccess &&
               cudaMalloc(&w->amul, sizeof(float) * K) == cudaSuccess &&
               cudaMalloc(&w->status, sizeof(int)) == cudaSuccess &&
               cudaMallocAsync(&wmul, sizeof(float) * K, st) == cudaSuccess &&
               (!bias_bf16 || cudaMalloc(&w->bias, sizeof(uint16_t) * N) == cudaSuccess) &&
-              (!(flags & QVGGT_PREP_C8) || cudaMalloc(&w->Wq8, (size_t)N * K) == cudaSuccess);
+              (!c8 || cudaMalloc(&w->Wq8, (size_t)N * K) == cudaSuccess);
     if (!ok) {
         cudaGetLastError();
         if (wmul) cudaFreeAsync(wmul, st);
@@ -69,8 +72,8 @@ int qvggt_prepare_weights(const void *W_bf16, const void *bias_bf16, const float
     if (e == cudaSuccess && bias_bf16)
         e = cudaMemcpyAsync(w->bias, bias_bf16, sizeof(uint16_t) * N, cudaMemcpyDeviceToDevice, st);
     if (e == cudaSuccess) e = qvggt_launch_multipliers(smooth_c, sign_v, K, w->amul, wmul, st);
-    if (e == cudaSuccess) e = qvggt_launch_rsq(W_bf16, K, N, K, wmul, 0, w->Wq, w->w_scale, st);
-    if (e == cudaSuccess && w->Wq8) e = qvggt_launch_rsq_c8(W_bf16, K, N, K, wmul, w->Wq8, w->w_scale, st);
+    if (e == cudaSuccess && w->Wq) e = qvggt_launch_rsq(W_bf16, K, N, K, wmul, 0, w->Wq, w->w_scale, st);
+    if (e == cudaSuccess && w->Wq8) e = qvggt_launch_rsq_c8(W_bf16, K, N, K, wmul, w->bits, w->Wq8, w->w_scale, st);
     // wmul is scratch: stream-ordered release so that the call stays asynchronous
     if (cudaFreeAsync(wmul, st) != cudaSuccess) cudaGetLastError();
     if (e != cudaSuccess) {
@@ -87,7 +90,7 @@ int qvggt_rotate_smooth_quantize(const qvggt_weights_t *w, const void *X_bf16, l
 {
     if (!w) return QVGGT_ERR_NULL;
     if (M < 0) return QVGGT_ERR_SHAPE;
-    if (group != 0 && group != 128) return QVGGT_ERR_UNSUPPORTED;
+    if ((group != 0 && group != 128) || w->bits != 4) return QVGGT_ERR_UNSUPPORTED;
     if (M == 0) return QVGGT_OK;
     if (!X_bf16 || !Xq || !a_scale) return QVGGT_ERR_NULL;
     if (ldx < w->K) return QVGGT_ERR_SHAPE;
@@ -101,7 +104,7 @@ int qvggt_w4a4_linear(const qvggt_weights_t *w, const unsigned char *Xq, const f
 {
     if (!w) return QVGGT_ERR_NULL;
     if (M < 0) return QVGGT_ERR_SHAPE;
-    if (group != 0 && group != 128) return QVGGT_ERR_UNSUPPORTED;
+    if ((group != 0 && group != 128) || w->bits != 4) return QVGGT_ERR_UNSUPPORTED;
     if (M == 0) return QVGGT_OK;
     if (!Xq || !a_scale || !Y_bf16) return QVGGT_ERR_NULL;
     if (ldy < w->N) return QVGGT_ERR_SHAPE;
@@ -122,7 +125,7 @@ int qvggt_rotate_smooth_quantize_c8(const qvggt_weights_t *w, const void *X_bf16
     if (!X_bf16 || !Xq8 || !a_scale) return QVGGT_ERR_NULL;
     if (ldx < w->K) return QVGGT_ERR_SHAPE;
     if (ldx % 8 != 0 || !aligned16(X_bf16) || !aligned16(Xq8) || (reinterpret_cast<uintptr_t>(a_scale) & 3u)) return QVGGT_ERR_ALIGN;
-    cudaError_t e = qvggt_launch_rsq_c8(X_bf16, ldx, M, w->K, w->amul, Xq8, a_scale, static_cast<cudaStream_t>(cuda_stream));
+    cudaError_t e = qvggt_launch_rsq_c8(X_bf16, ldx, M, w->K, w->amul, w->bits, Xq8, a_scale, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
 }
 
@@ -167,10 +170,11 @@ int qvggt_weights_view(const qvggt_weights_t *w, const unsigned char **Wq, const
     return QVGGT_OK;
 }
 
-int qvggt_weights_view_c8(const qvggt_weights_t *w, const signed char **Wq8)
+int qvggt_weights_view_c8(const qvggt_weights_t *w, const signed char **Wq8, int *bits)
 {
     if (!w || !Wq8) return QVGGT_ERR_NULL;
     *Wq8 = w->Wq8;
+    if (bits) *bits = w->bits;
     return QVGGT_OK;
 }
 

@@ -8,7 +8,8 @@
 struct qvggt_weights {
     int N, K;
     int device;
-    unsigned char *Wq;   // [N, K/2] packed int4
+    int bits;            // 4 (W4A4) or 8 (W8A8: codes one per byte only)
+    unsigned char *Wq;   // [N, K/2] packed int4 (nullptr when bits == 8)
     signed char *Wq8;    // [N, K] one code per byte, or nullptr (prepared without QVGGT_PREP_C8)
     float *w_scale;      // [N]
     float *amul;         // [K]
@@ -32,7 +33,7 @@ cudaError_t qvggt_launch_multipliers(const float *c, const signed char *v, int K
                                      cudaStream_t st);
 cudaError_t qvggt_launch_rsq(const void *X, long long ldx, int M, int K, const float *mul, int group,
                              unsigned char *Xq, float *scales, cudaStream_t st);
-cudaError_t qvggt_launch_rsq_c8(const void *X, long long ldx, int M, int K, const float *mul, signed char *Xq8,
+cudaError_t qvggt_launch_rsq_c8(const void *X, long long ldx, int M, int K, const float *mul, int bits, signed char *Xq8,
                                 float *scales, cudaStream_t st);
 cudaError_t qvggt_launch_colmax(const void *X, int M, int K, float *colmax, cudaStream_t st);
 cudaError_t qvggt_launch_smooth_finalize(const float *ax, const float *aw, int K, float alpha, float lo, float hi,

@@ -184,7 +184,8 @@ __device__ __forceinline__ void stages_in_registers(float (&v)[N])
 }
 
 // C8: one code per byte (int8, natural element order, row pitch K) instead of two per byte.
-template <int LOGT, int GROUP, bool C8 = false>
+// QMAX: largest code magnitude, 2^(N-1) - 1 of Eq. "quantization": 7 (N = 4) or, with C8 only, 127 (N = 8).
+template <int LOGT, int GROUP, bool C8 = false, int QMAX = 7>
 __global__ void __launch_bounds__(SqGeom<LOGT>::CTA_THREADS, LOGT == 5 ? 4 : 3)
 rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float *__restrict__ mul,
               unsigned char *__restrict__ Xq, float *__restrict__ scales)
@@ -296,8 +297,9 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
         }
         if constexpr (C8) {
             static_assert(!C8 || GROUP == 0, "byte output is built for per-token scales");
+            static_assert(QMAX == 7 || QMAX == 127, "4-bit or 8-bit codes");
             am[0] = fmaxf(am[0], 1e-8f);
-            const float inv = __fdiv_rn(7.0f, am[0]);
+            const float inv = __fdiv_rn(static_cast<float>(QMAX), am[0]);
             const uint64_t inv2 = ptx::f32x2_pack(inv, inv), magic2 = ptx::f32x2_pack(12582912.0f, 12582912.0f);
             // byte exchange between the 4 lanes that share (t / 4): a 4 x 4 byte transpose in two steps
             const uint32_t sel0 = (lane & 1) ? 0x3715u : 0x6240u, sel1 = (lane & 2) ? 0x3276u : 0x5410u;
@@ -316,11 +318,12 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
                 *reinterpret_cast<uint32_t *>(Xq + row * K + T * (4 * kk + (t & 3)) + 4 * (t >> 2)) = x;
             }
         } else {
+        static_assert(C8 || QMAX == 7, "two codes per byte hold 4-bit codes only");
         uint32_t word[T / 8];
 #pragma unroll
         for (int g = 0; g < NG; ++g) {
             am[g] = fmaxf(am[g], 1e-8f);
-            const float inv = __fdiv_rn(7.0f, am[g]);
+            const float inv = __fdiv_rn(static_cast<float>(QMAX), am[g]);
             const uint64_t inv2 = ptx::f32x2_pack(inv, inv), magic2 = ptx::f32x2_pack(12582912.0f, 12582912.0f);
 #pragma unroll
             for (int k = g * GREGS; k < (g + 1) * GREGS; k += 2) {
@@ -347,7 +350,7 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
         }
         if (t == 0) {
 #pragma unroll
-            for (int g = 0; g < NG; ++g) scales[row * NG + g] = __fdiv_rn(am[g], 7.0f);
+            for (int g = 0; g < NG; ++g) scales[row * NG + g] = __fdiv_rn(am[g], static_cast<float>(QMAX));
         }
     }
 }
@@ -429,14 +432,14 @@ namespace {
 
 // Launch with programmatic stream serialization allowed: the blocks may become resident while the previous
 // kernel of the stream drains (they wait in grid_dependency_wait() before touching global memory).
-template <int LOGT, int GROUP, bool C8>
+template <int LOGT, int GROUP, bool C8, int QMAX = 7>
 cudaError_t launch_sq(const uint16_t *x, long long ldx, int M, const float *mul, unsigned char *out, float *scales,
                       cudaStream_t st)
 {
     using G = SqGeom<LOGT>;
     static bool configured = false;       // per process and instantiation
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(rsq_sq_kernel<LOGT, GROUP, C8>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM);
+        cudaError_t e = cudaFuncSetAttribute(rsq_sq_kernel<LOGT, GROUP, C8, QMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM);
         if (e != cudaSuccess) return e;
         configured = true;
     }
@@ -450,17 +453,19 @@ cudaError_t launch_sq(const uint16_t *x, long long ldx, int M, const float *mul,
     cfg.stream = st;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, rsq_sq_kernel<LOGT, GROUP, C8>, x, ldx, M, mul, out, scales);
+    return cudaLaunchKernelEx(&cfg, rsq_sq_kernel<LOGT, GROUP, C8, QMAX>, x, ldx, M, mul, out, scales);
 }
 
 }  // namespace
 
-cudaError_t qvggt_launch_rsq_c8(const void *X, long long ldx, int M, int K, const float *mul, signed char *Xq8,
+cudaError_t qvggt_launch_rsq_c8(const void *X, long long ldx, int M, int K, const float *mul, int bits, signed char *Xq8,
                                 float *scales, cudaStream_t st)
 {
     if (M == 0) return cudaSuccess;
     const uint16_t *x = static_cast<const uint16_t *>(X);
     unsigned char *out = reinterpret_cast<unsigned char *>(Xq8);
+    if (bits == 8)
+        return K == 1024 ? launch_sq<5, 0, true, 127>(x, ldx, M, mul, out, scales, st) : launch_sq<6, 0, true, 127>(x, ldx, M, mul, out, scales, st);
     return K == 1024 ? launch_sq<5, 0, true>(x, ldx, M, mul, out, scales, st) : launch_sq<6, 0, true>(x, ldx, M, mul, out, scales, st);
 }
 
