@@ -29,6 +29,9 @@
  *     integer partial sums are rescaled per group in the epilogue).
  *   - All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = default
  *     stream); no call synchronises the device except where stated.
+ *     The quantize and *_c8 GEMM kernels are launched with programmatic stream serialization allowed:
+ *     their blocks may become resident while the previous kernel of the stream drains, but they touch
+ *     no global memory before that kernel has completed, so stream order is what the caller sees.
  *   - Return value: QVGGT_OK or a negative qvggt_status_t.  Arguments are validated on the host
  *     before anything is launched; nothing throws or exits.
  *   - Device-side waits are bounded.  If one expires the kernel records a code in the handle's
