@@ -167,14 +167,16 @@ __device__ __forceinline__ void group_sync(int slot)
 
 // In-register stages over n values: the first joins neighbours (scalar: packing it costs more register
 // moves than it saves), the others pair (k, k + 1).
-template <int N>
+template <int N, bool FIRST = true>
 __device__ __forceinline__ void stages_in_registers(float (&v)[N])
 {
+    if (FIRST) {
 #pragma unroll
-    for (int k = 0; k < N; k += 2) {
-        const float a = v[k], b = v[k + 1];
-        v[k] = __fadd_rn(a, b);
-        v[k + 1] = __fsub_rn(a, b);
+        for (int k = 0; k < N; k += 2) {
+            const float a = v[k], b = v[k + 1];
+            v[k] = __fadd_rn(a, b);
+            v[k + 1] = __fsub_rn(a, b);
+        }
     }
 #pragma unroll
     for (int h = 2; h < N; h <<= 1)
@@ -255,12 +257,17 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
                 const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    v[8 * c + 2 * j] = __uint_as_float(w[j] << 16);
-                    v[8 * c + 2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+                    // a 32-bit word holds elements 2i (low half) and 2i + 1 of the row: the first stage joins exactly
+                    // these two, and the mixed-precision add takes the bf16 half as it is (its conversion is exact,
+                    // so this is fl(float(lo) + float(hi)) and fl(float(lo) - float(hi)), one rounding each)
+                    const float hi = __uint_as_float(w[j] & 0xFFFF0000u);
+                    const unsigned short lo = static_cast<unsigned short>(w[j]);
+                    asm("add.rn.f32.bf16 %0, %1, %2;" : "=f"(v[8 * c + 2 * j]) : "h"(lo), "f"(hi));
+                    asm("sub.rn.f32.bf16 %0, %1, %2;" : "=f"(v[8 * c + 2 * j + 1]) : "h"(lo), "f"(hi));
                 }
             }
         }
-        stages_in_registers<T>(v);          // strides 1 .. T/2
+        stages_in_registers<T, false>(v);   // strides 2 .. T/2 (stride 1 was taken with the conversion)
 #pragma unroll
         for (int j = 0; j < T; ++j) Tm[j * T + ((((t >> 2) ^ (j & 7)) << 2) | (t & 3))] = v[j];
         group_sync<T>(slot);
@@ -281,7 +288,8 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
         for (int g = 0; g < NG; ++g) {
             float a = fmaxf(fabsf(v[g * GREGS]), fabsf(v[g * GREGS + 1]));
 #pragma unroll
-            for (int k = 2; k < GREGS; k += 2) a = fmaxf(fmaxf(a, fabsf(v[g * GREGS + k])), fabsf(v[g * GREGS + k + 1]));
+            for (int k = 2; k < GREGS; k += 2)     // max(|a|, |x|, |y|) in one instruction
+                asm("max.abs.f32 %0, %1, %2, %3;" : "=f"(a) : "f"(a), "f"(v[g * GREGS + k]), "f"(v[g * GREGS + k + 1]));
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, o));
             am[g] = a;
