@@ -44,6 +44,7 @@ def _L():
             "orc_multipliers": [vp, vp, i32, vp, vp],
             "orc_rotate_smooth_quantize": [vp, i64, i64, i32, vp, i32, vp, vp],
             "orc_rotate_smooth_quantize_bits": [vp, i64, i64, i32, vp, i32, i32, vp, vp],
+            "orc_rotate_smooth_quantize_static": [vp, i64, i64, i32, vp, ctypes.c_float, i32, vp],
             "orc_pack_int4": [vp, i64, i32, vp],
             "orc_unpack_int4": [vp, i64, i32, vp],
             "orc_gemm_i32": [vp, vp, i64, i32, i32, i32, vp],
@@ -119,6 +120,18 @@ def rotate_smooth_quantize(X: np.ndarray, mul: np.ndarray, group: int = 0, bits:
         _L().orc_rotate_smooth_quantize_bits(X.ctypes.data, X.strides[0] // 2, M, K, mul.ctypes.data, group, bits,
                                              codes.ctypes.data, scales.ctypes.data)
     return codes, (scales if group else scales.reshape(M))
+
+
+def rotate_smooth_quantize_static(X: np.ndarray, mul: np.ndarray, delta: float, bits: int = 4) -> np.ndarray:
+    """Static tensor-wise quantizer (Tab. "granularity"): X bf16 bits [M, K], one given step size -> codes int8 [M, K]
+    (clamped to [-2^(bits-1), 2^(bits-1) - 1])."""
+    assert X.dtype == np.uint16 and X.ndim == 2 and X.strides[1] == 2 and 2 <= bits <= 8 and delta > 0
+    M, K = X.shape
+    mul = _c(mul, np.float32)
+    codes = np.empty((M, K), np.int8)
+    _L().orc_rotate_smooth_quantize_static(X.ctypes.data, X.strides[0] // 2, M, K, mul.ctypes.data, np.float32(delta), bits,
+                                           codes.ctypes.data)
+    return codes
 
 
 def pack_int4(codes: np.ndarray) -> np.ndarray:

@@ -145,6 +145,38 @@ void orc_rotate_smooth_quantize_bits(const uint16_t *X, int64_t ldx, int64_t M, 
     }
 }
 
+/*
+ * Static tensor-wise activation quantizer (the other arm of the paper's granularity ablation, Tab. "granularity":
+ * one step size Delta for the whole tensor, fixed offline, instead of one per token computed from the data).
+ * Eq. "quantization" with a given Delta: q = clamp(round(y / Delta), -2^(N-1), 2^(N-1) - 1), where the clamp now
+ * matters.  Same readings as above: round-half-to-even; y / Delta is the exact product y * fl(1 / Delta) rounded once.
+ *   delta  the step size (> 0);  codes int8 [M, K]
+ */
+void orc_rotate_smooth_quantize_static(const uint16_t *X, int64_t ldx, int64_t M, int K, const float *mul, float delta,
+                                       int bits, int8_t *codes)
+{
+    const double lo = -(double)(1 << (bits - 1)), hi = (double)((1 << (bits - 1)) - 1);
+    const float inv = 1.0f / delta;
+#pragma omp parallel
+    {
+        float *u = (float *)malloc(sizeof(float) * (size_t)K);
+#pragma omp for schedule(static)
+        for (int64_t m = 0; m < M; ++m) {
+            const uint16_t *x = X + m * ldx;
+            for (int k = 0; k < K; ++k) u[k] = orc_bf16_to_f32(x[k]);
+            orc_fwht_f32(u, K);
+            for (int k = 0; k < K; ++k) {
+                float y = u[k] * mul[k];
+                double r = nearbyint((double)y * (double)inv); /* exact product, one rounding */
+                if (r < lo) r = lo;
+                if (r > hi) r = hi;
+                codes[m * K + k] = (int8_t)r;
+            }
+        }
+        free(u);
+    }
+}
+
 /* The W4A4 setting (N = 4: Delta = max|y| / 7, codes in [-8, 7]). */
 void orc_rotate_smooth_quantize(const uint16_t *X, int64_t ldx, int64_t M, int K, const float *mul,
                                 int group, int8_t *codes, float *scales)

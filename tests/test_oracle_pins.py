@@ -215,6 +215,41 @@ def test_8bit_round_half_to_even_and_extremes():
     assert np.array_equal(codes[0], want)
 
 
+@pytest.mark.parametrize("bits", [4, 8])
+def test_static_quantizer_power_of_two_step_against_float64(bits):
+    """Static tensor-wise quantizer (Tab. "granularity"): with Delta a power of two, y / Delta is exact in any
+    precision, so the codes must equal clamp(rint(y / Delta)) computed independently in float64; both ends of the
+    clamp are reached (outlier channels and special-token rows)."""
+    K = 1024
+    spec = workload.LinearSpec("t", K, 8, workload.DIST_NORMAL, 29, 0)
+    X = spec.x_rows(0, 12)
+    amul, _ = oracle.multipliers(workload.loguniform_f32(29, 5, K, 0.05, 20), workload.signs_i8(29, 6, K))
+    y = _rotated_y(X, amul).astype(np.float64)
+    delta = 2.0 ** np.floor(np.log2(np.median(np.abs(y)) / 2))
+    codes = oracle.rotate_smooth_quantize_static(X, amul, float(delta), bits)
+    lo, hi = -(2 ** (bits - 1)), 2 ** (bits - 1) - 1
+    want = np.clip(np.rint(y / delta), lo, hi)
+    assert np.array_equal(codes.astype(np.float64), want)
+    assert codes.min() == lo and codes.max() == hi                 # the clamp is exercised on both sides
+    inside = (want > lo) & (want < hi)
+    assert np.all(np.abs(y - delta * want)[inside] <= delta / 2)     # |x - Delta q| <= Delta / 2 where nothing was clamped
+
+
+def test_static_quantizer_ties_and_saturation_by_hand():
+    """Delta = 1 on hand-picked values (a unit vector rotates to all ones, so y equals the multiplier vector)."""
+    K = 16
+    y = np.array([0.5, 1.5, 2.5, -0.5, 7.49, 7.5, 7.51, 8.5, 100.0, -8.5, -9.0, -100.0, 1e30, -1e30, 6.5, -7.5], np.float32)
+    want = np.array([0, 2, 2, 0, 7, 7, 7, 7, 7, -8, -8, -8, 7, -8, 6, -8], np.int8)
+    X = np.zeros((1, K), np.uint16)
+    X[0, 0] = 0x3F80
+    assert np.array_equal(oracle.rotate_smooth_quantize_static(X, y, 1.0, 4)[0], want)
+    # a step that is not a power of two: the factor is fl(1/3); 4.5 * fl(1/3) = 1.5000000447 rounds up to 2
+    y3 = np.array([3.0, 4.5, -4.5, 1.5, 21.0, 22.5, -24.0, -25.5] * 2, np.float32)
+    want3 = np.array([1, 2, -2, 1, 7, 7, -8, -8] * 2, np.int8)
+    assert float(np.float32(1.0) / np.float32(3.0)) > 1.0 / 3.0    # fl(1/3) lies above 1/3
+    assert np.array_equal(oracle.rotate_smooth_quantize_static(X, y3, 3.0, 4)[0], want3)
+
+
 def test_round_half_to_even_on_handbuilt_ties():
     tab = load_table("round_ties.txt")
     y, want = tab[:, 0], tab[:, 1].astype(np.int8)
