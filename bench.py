@@ -438,6 +438,19 @@ def run_rsq_sweep(args):
             us = float(np.median(times)) * 1e3
             gbs = rsq_bytes(M, K, path.code_bytes) / us / 1e3
             out[f"K{K}_M{M}"] = {"us": round(us, 2), "gbs": round(gbs, 1), "hbm_frac": round(gbs / peaks["hbm_gbs"], 4)}
+            if path.fmt != "packed":
+                # the granularity ablation's other arm: static tensor-wise step size (no absolute maximum per token)
+                delta = a.median().reshape(1).contiguous()
+                times = []
+                for _ in range(max(5, min(args.steps, 30))):
+                    flush.zero_()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    q.rotate_smooth_quantize_static_c8(h, X, delta, xq, a)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    times.append(e0.elapsed_time(e1))
+                out[f"K{K}_M{M}"]["static_tensorwise_us"] = round(float(np.median(times)) * 1e3, 2)
             del X, xq, a, flush
     best = max(v["gbs"] for v in out.values())
     print(json.dumps({"metric": "rsq_gbs", "value": best, "unit": "GB/s", "n_gpus": 1, "higher_is_better": True,

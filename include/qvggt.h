@@ -129,6 +129,17 @@ int qvggt_rotate_smooth_quantize_c8(const qvggt_weights_t *w, const void *X_bf16
 int qvggt_w4a4_linear_c8(const qvggt_weights_t *w, const signed char *Xq8, const float *a_scale, int M,
                          void *Y_bf16, long long ldy, int *acc_debug, void *cuda_stream);
 
+/*
+ * Static tensor-wise activation quantizer: the other arm of the paper's granularity ablation (Tab. "granularity",
+ * dynamic token-wise against static tensor-wise).  One step size for the whole tensor, fixed offline, instead of
+ * one per token from the token's absolute maximum:  Xq8 = clamp(round(y * fl(1 / delta)), -2^(N-1), 2^(N-1) - 1)
+ * (Eq. "quantization" with its clamp active; N = the handle's code width), a_scale[m] = delta for every m, so that
+ * qvggt_w4a4_linear_c8 follows unchanged.
+ *   delta    DEVICE pointer to one fp32 step size (> 0, finite); read by the kernel, not by the host
+ */
+int qvggt_rotate_smooth_quantize_static_c8(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M,
+                                           const float *delta, signed char *Xq8, float *a_scale, void *cuda_stream);
+
 /* Frees the handle and its device memory (synchronises the device first).  NULL is allowed. */
 void qvggt_free_weights(qvggt_weights_t *w);
 

@@ -187,11 +187,15 @@ __device__ __forceinline__ void stages_in_registers(float (&v)[N])
 
 // C8: one code per byte (int8, natural element order, row pitch K) instead of two per byte.
 // QMAX: largest code magnitude, 2^(N-1) - 1 of Eq. "quantization": 7 (N = 4) or, with C8 only, 127 (N = 8).
-template <int LOGT, int GROUP, bool C8 = false, int QMAX = 7>
+// STATIC (C8 only): one given step size *static_delta for the whole tensor (the static tensor-wise arm of the
+// granularity ablation) instead of one per row from the row's absolute maximum; the clamp of Eq. "quantization"
+// to [-QMAX - 1, QMAX] is then active, and every row's scale is written as that step size.
+template <int LOGT, int GROUP, bool C8 = false, int QMAX = 7, bool STATIC = false>
 __global__ void __launch_bounds__(SqGeom<LOGT>::CTA_THREADS, LOGT == 5 ? 4 : 3)
 rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float *__restrict__ mul,
-              unsigned char *__restrict__ Xq, float *__restrict__ scales)
+              unsigned char *__restrict__ Xq, float *__restrict__ scales, const float *__restrict__ static_delta)
 {
+    static_assert(!STATIC || (C8 && GROUP == 0), "the static step size is built for one code per byte");
     using G = SqGeom<LOGT>;
     constexpr int T = G::T, K = G::K, CH = G::CH;
     constexpr int NG = (GROUP == 128) ? K / 128 : 1;           // scale groups per row
@@ -234,6 +238,7 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
         for (int j = 0; j < CH; ++j) cp_async16(stage + cp_dst[j], src + 16 * (t + T * j));
     }
     cp_async_commit();
+    const float delta = STATIC ? __ldg(static_delta) : 0.0f;
     float m[T];                                                // multipliers of elements T k + t (loaded behind the first row's copies)
 #pragma unroll
     for (int k = 0; k < T; ++k) m[k] = __ldg(mul + T * k + t);
@@ -285,7 +290,7 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
         // absolute maxima: one per row, or one per 128 consecutive elements (GREGS registers of every thread)
         float am[NG];
 #pragma unroll
-        for (int g = 0; g < NG; ++g) {
+        for (int g = 0; g < (STATIC ? 0 : NG); ++g) {
             float a = fmaxf(fabsf(v[g * GREGS]), fabsf(v[g * GREGS + 1]));
 #pragma unroll
             for (int k = 2; k < GREGS; k += 2)     // max(|a|, |x|, |y|) in one instruction
@@ -294,7 +299,7 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
             for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, o));
             am[g] = a;
         }
-        if (T == 64) {
+        if (T == 64 && !STATIC) {
             if (lane == 0) {
 #pragma unroll
                 for (int g = 0; g < NG; ++g) red[(t >> 5) * NG + g] = am[g];
@@ -306,8 +311,14 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
         if constexpr (C8) {
             static_assert(!C8 || GROUP == 0, "byte output is built for per-token scales");
             static_assert(QMAX == 7 || QMAX == 127, "4-bit or 8-bit codes");
-            am[0] = fmaxf(am[0], 1e-8f);
-            const float inv = __fdiv_rn(static_cast<float>(QMAX), am[0]);
+            float inv;
+            if (STATIC) {
+                inv = __fdiv_rn(1.0f, delta);
+                am[0] = __fmul_rn(delta, static_cast<float>(QMAX));     // the scale written below is am / QMAX = delta
+            } else {
+                am[0] = fmaxf(am[0], 1e-8f);
+                inv = __fdiv_rn(static_cast<float>(QMAX), am[0]);
+            }
             const uint64_t inv2 = ptx::f32x2_pack(inv, inv), magic2 = ptx::f32x2_pack(12582912.0f, 12582912.0f);
             // byte exchange between the 4 lanes that share (t / 4): a 4 x 4 byte transpose in two steps
             const uint32_t sel0 = (lane & 1) ? 0x3715u : 0x6240u, sel1 = (lane & 2) ? 0x3276u : 0x5410u;
@@ -317,6 +328,14 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
                 float f0, f1, f2, f3;
                 ptx::f32x2_unpack(ptx::f32x2_fma(ptx::f32x2_pack(v[4 * kk], v[4 * kk + 1]), inv2, magic2), f0, f1);
                 ptx::f32x2_unpack(ptx::f32x2_fma(ptx::f32x2_pack(v[4 * kk + 2], v[4 * kk + 3]), inv2, magic2), f2, f3);
+                if (STATIC) {
+                    // The clamp of Eq. "quantization", taken on the sum with the magic number: inside +-2^22 that sum is
+                    // 1.5 * 2^23 + q exactly; beyond, the fused operation still returns the correctly rounded (huge) sum,
+                    // which the clamp saturates all the same.  The low mantissa byte stays the two's-complement code.
+                    constexpr float lo = 12582912.0f - (QMAX + 1), hi = 12582912.0f + QMAX;
+                    f0 = fminf(fmaxf(f0, lo), hi); f1 = fminf(fmaxf(f1, lo), hi);
+                    f2 = fminf(fmaxf(f2, lo), hi); f3 = fminf(fmaxf(f3, lo), hi);
+                }
                 // byte n = code of element T (4 kk + n) + t
                 uint32_t x = __byte_perm(__byte_perm(__float_as_uint(f0), __float_as_uint(f1), 0x0040),
                                          __byte_perm(__float_as_uint(f2), __float_as_uint(f3), 0x0040), 0x5410);
@@ -358,7 +377,7 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
         }
         if (t == 0) {
 #pragma unroll
-            for (int g = 0; g < NG; ++g) scales[row * NG + g] = __fdiv_rn(am[g], static_cast<float>(QMAX));
+            for (int g = 0; g < NG; ++g) scales[row * NG + g] = STATIC ? delta : __fdiv_rn(am[g], static_cast<float>(QMAX));
         }
     }
 }
@@ -440,14 +459,14 @@ namespace {
 
 // Launch with programmatic stream serialization allowed: the blocks may become resident while the previous
 // kernel of the stream drains (they wait in grid_dependency_wait() before touching global memory).
-template <int LOGT, int GROUP, bool C8, int QMAX = 7>
+template <int LOGT, int GROUP, bool C8, int QMAX = 7, bool STATIC = false>
 cudaError_t launch_sq(const uint16_t *x, long long ldx, int M, const float *mul, unsigned char *out, float *scales,
-                      cudaStream_t st)
+                      cudaStream_t st, const float *static_delta = nullptr)
 {
     using G = SqGeom<LOGT>;
     static bool configured = false;       // per process and instantiation
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(rsq_sq_kernel<LOGT, GROUP, C8, QMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM);
+        cudaError_t e = cudaFuncSetAttribute(rsq_sq_kernel<LOGT, GROUP, C8, QMAX, STATIC>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM);
         if (e != cudaSuccess) return e;
         configured = true;
     }
@@ -461,7 +480,7 @@ cudaError_t launch_sq(const uint16_t *x, long long ldx, int M, const float *mul,
     cfg.stream = st;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, rsq_sq_kernel<LOGT, GROUP, C8, QMAX>, x, ldx, M, mul, out, scales);
+    return cudaLaunchKernelEx(&cfg, rsq_sq_kernel<LOGT, GROUP, C8, QMAX, STATIC>, x, ldx, M, mul, out, scales, static_delta);
 }
 
 }  // namespace
@@ -475,6 +494,19 @@ cudaError_t qvggt_launch_rsq_c8(const void *X, long long ldx, int M, int K, cons
     if (bits == 8)
         return K == 1024 ? launch_sq<5, 0, true, 127>(x, ldx, M, mul, out, scales, st) : launch_sq<6, 0, true, 127>(x, ldx, M, mul, out, scales, st);
     return K == 1024 ? launch_sq<5, 0, true>(x, ldx, M, mul, out, scales, st) : launch_sq<6, 0, true>(x, ldx, M, mul, out, scales, st);
+}
+
+cudaError_t qvggt_launch_rsq_static_c8(const void *X, long long ldx, int M, int K, const float *mul, int bits, const float *delta,
+                                       signed char *Xq8, float *scales, cudaStream_t st)
+{
+    if (M == 0) return cudaSuccess;
+    const uint16_t *x = static_cast<const uint16_t *>(X);
+    unsigned char *out = reinterpret_cast<unsigned char *>(Xq8);
+    if (bits == 8)
+        return K == 1024 ? launch_sq<5, 0, true, 127, true>(x, ldx, M, mul, out, scales, st, delta)
+                         : launch_sq<6, 0, true, 127, true>(x, ldx, M, mul, out, scales, st, delta);
+    return K == 1024 ? launch_sq<5, 0, true, 7, true>(x, ldx, M, mul, out, scales, st, delta)
+                     : launch_sq<6, 0, true, 7, true>(x, ldx, M, mul, out, scales, st, delta);
 }
 
 cudaError_t qvggt_launch_rsq(const void *X, long long ldx, int M, int K, const float *mul, int group,
