@@ -158,3 +158,28 @@ def test_c8_config1_single_frame_proj():
     assert np.array_equal(a_scale.cpu().numpy(), ref["a_scale"])
     assert np.array_equal(acc.cpu().numpy(), ref["acc"])
     assert assert_bf16_within_one_ulp(host_bits(Y), ref["y"]) == 0.0
+
+
+def test_c8_chained_launches_are_deterministic():
+    """The quantize kernel and the GEMM chained 60 times on one stream (consecutive kernels overlap through
+    programmatic dependent launch: each one's blocks may become resident while its predecessor drains): every
+    repetition must reproduce the oracle-checked first result bit for bit."""
+    spec = workload.LinearSpec("d", 1024, 1024, workload.DIST_NORMAL, 13, 1)
+    L = make_layer(spec)
+    M = 4 * workload.TOKENS_PER_FRAME
+    X = spec.x_rows(0, M)
+    rows = np.arange(0, M, 97)
+    Xd = dev_bf16(X)
+    Xq8, a_scale = q.rotate_smooth_quantize_c8(L["h"], Xd)
+    Y0 = q.w4a4_linear_c8(L["h"], Xq8, a_scale).clone()
+    codes, scales = oracle.rotate_smooth_quantize(np.ascontiguousarray(X[rows]), L["prep"]["amul"], 0)
+    want = oracle.epilogue(oracle.gemm_i32(codes, L["prep"]["wq"]), scales, L["prep"]["w_scale"], L["b"])
+    assert assert_bf16_within_one_ulp(host_bits(Y0[torch.from_numpy(rows).cuda()]), want) == 0.0
+    q0, a0 = Xq8.clone(), a_scale.clone()
+    Y = torch.empty_like(Y0)
+    for i in range(60):
+        q.rotate_smooth_quantize_c8(L["h"], Xd, Xq8, a_scale)
+        q.w4a4_linear_c8(L["h"], Xq8, a_scale, Y)
+        if i % 6 == 5:
+            assert torch.equal(Y.view(torch.int16), Y0.view(torch.int16)) and torch.equal(Xq8, q0) and torch.equal(a_scale, a0), i
+    assert L["h"].device_status() == 0
