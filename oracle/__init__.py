@@ -45,6 +45,7 @@ def _L():
             "orc_rotate_smooth_quantize": [vp, i64, i64, i32, vp, i32, vp, vp],
             "orc_rotate_smooth_quantize_bits": [vp, i64, i64, i32, vp, i32, i32, vp, vp],
             "orc_rotate_smooth_quantize_static": [vp, i64, i64, i32, vp, ctypes.c_float, i32, vp],
+            "orc_layernorm": [vp, i64, i64, i32, vp, vp, ctypes.c_float, vp],
             "orc_pack_int4": [vp, i64, i32, vp],
             "orc_unpack_int4": [vp, i64, i32, vp],
             "orc_gemm_i32": [vp, vp, i64, i32, i32, i32, vp],
@@ -120,6 +121,17 @@ def rotate_smooth_quantize(X: np.ndarray, mul: np.ndarray, group: int = 0, bits:
         _L().orc_rotate_smooth_quantize_bits(X.ctypes.data, X.strides[0] // 2, M, K, mul.ctypes.data, group, bits,
                                              codes.ctypes.data, scales.ctypes.data)
     return codes, (scales if group else scales.reshape(M))
+
+
+def layernorm(X: np.ndarray, gamma: np.ndarray, beta: np.ndarray, eps: float = 1e-5) -> np.ndarray:
+    """LayerNorm over the K channels of every token row, fp32 with pairwise-summed statistics -> bf16 bits [M, K]."""
+    assert X.dtype == np.uint16 and X.ndim == 2 and X.strides[1] == 2
+    M, K = X.shape
+    assert K & (K - 1) == 0
+    gamma, beta = _c(gamma, np.float32), _c(beta, np.float32)
+    out = np.empty((M, K), np.uint16)
+    _L().orc_layernorm(X.ctypes.data, X.strides[0] // 2, M, K, gamma.ctypes.data, beta.ctypes.data, np.float32(eps), out.ctypes.data)
+    return out
 
 
 def rotate_smooth_quantize_static(X: np.ndarray, mul: np.ndarray, delta: float, bits: int = 4) -> np.ndarray:

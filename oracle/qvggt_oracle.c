@@ -69,6 +69,55 @@ void orc_fwht_f64(double *u, int K)
 }
 
 /* K^{-1/2}: an exact power of two when log2 K is even (K = 1024, 4096). */
+/*
+ * LayerNorm in front of the rotation (Sec. 3.2 places the quantized linear behind a normalization layer; the
+ * upstream-fusion row fuses the two).  The paper does not say how the statistics are summed, so this build fixes it:
+ * plain pairwise summation (the sum of n terms is fl(sum of the first half + sum of the second half), recursively),
+ * everything in fp32, one rounding per operation:
+ *   mean = pairwise(x) / K;  d_k = fl(x_k - mean);  var = pairwise(fl(d_k * d_k)) / K      (K a power of two: exact divisions)
+ *   rstd = fl(1 / fl(sqrt(fl(var + eps))))
+ *   out_k = bf16( fl( fl(fl(d_k * rstd) * gamma_k) + beta_k ) )                               (round to nearest even)
+ *   X bf16 bits [M, K] (row stride ldx), gamma / beta fp32 [K], out bf16 bits [M, K] contiguous
+ */
+static float orc_pairwise(const float *a, int n)
+{
+    if (n == 1) return a[0];
+    float lo = orc_pairwise(a, n / 2), hi = orc_pairwise(a + n / 2, n / 2);
+    return lo + hi;
+}
+
+void orc_layernorm(const uint16_t *X, int64_t ldx, int64_t M, int K, const float *gamma, const float *beta, float eps,
+                   uint16_t *out)
+{
+    const float invK = 1.0f / (float)K;
+#pragma omp parallel
+    {
+        float *x = (float *)malloc(sizeof(float) * (size_t)K);
+        float *d = (float *)malloc(sizeof(float) * (size_t)K);
+#pragma omp for schedule(static)
+        for (int64_t m = 0; m < M; ++m) {
+            for (int k = 0; k < K; ++k) x[k] = orc_bf16_to_f32(X[m * ldx + k]);
+            float mean = orc_pairwise(x, K) * invK;
+            for (int k = 0; k < K; ++k) {
+                d[k] = x[k] - mean;
+                x[k] = d[k] * d[k];
+            }
+            float var = orc_pairwise(x, K) * invK;
+            float t = var + eps;
+            t = sqrtf(t);
+            float rstd = 1.0f / t;
+            for (int k = 0; k < K; ++k) {
+                float n = d[k] * rstd;
+                n = n * gamma[k];
+                n = n + beta[k];
+                out[m * K + k] = orc_f32_to_bf16(n);
+            }
+        }
+        free(x);
+        free(d);
+    }
+}
+
 static float orc_norm(int K)
 {
     return (float)(1.0 / sqrt((double)K));

@@ -250,6 +250,69 @@ def test_static_quantizer_ties_and_saturation_by_hand():
     assert np.array_equal(oracle.rotate_smooth_quantize_static(X, y3, 3.0, 4)[0], want3)
 
 
+@pytest.mark.parametrize("K", [1024, 4096])
+def test_layernorm_against_float64_and_special_rows(K):
+    """LayerNorm of the upstream-fusion row: within fp32 rounding of a float64 LayerNorm (numpy, a different
+    summation) on heavy-tailed rows, so a wrong statistic, a dropped eps, gamma or beta would show; exact on rows
+    whose arithmetic is exact (constant row -> beta; a +-a row with gamma = a power of two)."""
+    spec = workload.LinearSpec("t", K, 8, workload.DIST_NORMAL, 37, 0)
+    X = spec.x_rows(0, 9)
+    rng = np.random.default_rng(K)
+    gamma = rng.uniform(0.5, 2.0, K).astype(np.float32)
+    beta = rng.normal(0, 0.3, K).astype(np.float32)
+    eps = 1e-5
+    got = workload.bf16_to_f32(oracle.layernorm(X, gamma, beta, eps)).astype(np.float64)
+    x = workload.bf16_to_f32(X).astype(np.float64)
+    mu = x.mean(axis=1, keepdims=True)
+    var = ((x - mu) ** 2).mean(axis=1, keepdims=True)
+    want = (x - mu) / np.sqrt(var + eps) * gamma + beta
+    assert np.all(np.abs(got - want) <= 2.0 ** -8 * np.abs(want) + 1e-5 * (np.abs(x - mu) / np.sqrt(var + eps) + 1))
+    # constant row: d = 0 exactly, so the output is bf16(beta) whatever gamma is
+    Xc = np.full((1, K), 0x4049, np.uint16)
+    assert np.array_equal(oracle.layernorm(Xc, gamma, beta, eps), f32_round_to_bf16_bits(beta)[None, :])
+    # +-2 alternating: mean 0, var 4, rstd = fl(1/sqrt(4 + eps)); output = bf16(fl(fl(+-2 * rstd) * 4) + 0)
+    Xa = np.tile(np.array([0x4000, 0xC000], np.uint16), K // 2)[None, :]
+    rstd = np.float32(1.0) / np.sqrt(np.float32(4.0) + np.float32(eps), dtype=np.float32)
+    val = np.float32(np.float32(2.0) * rstd) * np.float32(4.0)
+    out = oracle.layernorm(Xa, np.full(K, 4.0, np.float32), np.zeros(K, np.float32), eps)
+    assert np.array_equal(out[0, 0::2], np.full(K // 2, f32_round_to_bf16_bits(np.array([val]))[0]))
+    assert np.array_equal(out[0, 1::2], np.full(K // 2, f32_round_to_bf16_bits(np.array([-val]))[0]))
+
+
+def test_layernorm_pairwise_order_is_the_stated_tree():
+    """The statistic is summed pairwise (halves, recursively), not left to right: a row on which the two orders
+    give different fp32 sums must follow the tree."""
+    K = 1024
+    x = np.zeros(K, np.float32)
+    x[0] = 2.0 ** 24                 # left to right, every later 1.0 is absorbed by 2^24; pairwise keeps them
+    x[1:] = 1.0
+    X = (x.view(np.uint32) >> 16).astype(np.uint16)[None, :]
+
+    def pairwise(a):
+        a = a.astype(np.float32)
+        while a.size > 1:
+            a = (a[0::2] + a[1::2]).astype(np.float32)
+        return a[0]
+
+    seq = np.float32(0)
+    for v in x:
+        seq = np.float32(seq + v)
+    assert pairwise(x) != seq
+    mean = np.float32(pairwise(x) * np.float32(1.0 / K))
+    d = (x - mean).astype(np.float32)
+    var = np.float32(pairwise((d * d).astype(np.float32)) * np.float32(1.0 / K))
+    rstd = np.float32(1.0) / np.sqrt(np.float32(var + np.float32(1e-5)), dtype=np.float32)
+    want = f32_round_to_bf16_bits((d * rstd).astype(np.float32))
+    got = oracle.layernorm(X, np.ones(K, np.float32), np.zeros(K, np.float32), 1e-5)[0]
+    assert np.array_equal(got, want)
+
+
+def f32_round_to_bf16_bits(a):
+    """Round-to-nearest-even fp32 -> bf16 bits, written out independently of the oracle."""
+    u = np.asarray(a, np.float32).view(np.uint32).astype(np.uint64)
+    return (((u + 0x7FFF + ((u >> 16) & 1)) >> 16) & 0xFFFF).astype(np.uint16)
+
+
 def test_round_half_to_even_on_handbuilt_ties():
     tab = load_table("round_ties.txt")
     y, want = tab[:, 0], tab[:, 1].astype(np.int8)
