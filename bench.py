@@ -481,6 +481,29 @@ def run_rsq_sweep(args):
                     torch.cuda.synchronize()
                     times.append(e0.elapsed_time(e1))
                 out[f"K{K}_M{M}"]["static_tensorwise_us"] = round(float(np.median(times)) * 1e3, 2)
+                # upstream fusion: LayerNorm + quantize as two kernels against the fused kernel (same results, bit for bit)
+                gamma = torch.rand(K, device="cuda") + 0.5
+                beta = torch.randn(K, device="cuda") * 0.1
+                ln_out = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+
+                def two_kernels():
+                    q.layernorm(X, gamma, beta, 1e-5, ln_out)
+                    path.rsq(h, ln_out, xq, a)
+
+                for name, fn in (("ln_then_quantize_us", two_kernels),
+                                 ("ln_fused_us", lambda: q.layernorm_rotate_smooth_quantize_c8(h, X, gamma, beta, 1e-5, xq, a))):
+                    fn()
+                    times = []
+                    for _ in range(max(5, min(args.steps, 30))):
+                        flush.zero_()
+                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        e0.record()
+                        fn()
+                        e1.record()
+                        torch.cuda.synchronize()
+                        times.append(e0.elapsed_time(e1))
+                    out[f"K{K}_M{M}"][name] = round(float(np.median(times)) * 1e3, 2)
+                del ln_out
             del X, xq, a, flush
     best = max(v["gbs"] for v in out.values())
     print(json.dumps({"metric": "rsq_gbs", "value": best, "unit": "GB/s", "n_gpus": 1, "higher_is_better": True,

@@ -140,6 +140,24 @@ int qvggt_w4a4_linear_c8(const qvggt_weights_t *w, const signed char *Xq8, const
 int qvggt_rotate_smooth_quantize_static_c8(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M,
                                            const float *delta, signed char *Xq8, float *a_scale, void *cuda_stream);
 
+/*
+ * Upstream fusion (Sec. 3.2 places the quantized linears of a block behind its normalization layers): LayerNorm over
+ * the K channels of every token, then the activation path of qvggt_rotate_smooth_quantize_c8, in one pass over X --
+ * the normalized activations never go to memory.  The result is, bit for bit, that of qvggt_layernorm followed by
+ * qvggt_rotate_smooth_quantize_c8.  LayerNorm in fp32, one rounding per operation, statistics summed pairwise
+ * (the sum of n terms is fl(sum of the first half + sum of the second half), recursively):
+ *   mean = sum(x) / K;  d = x - mean;  var = sum(d * d) / K;  rstd = 1 / sqrt(var + eps)
+ *   ln[k] = bf16( (d[k] * rstd) * gamma[k] + beta[k] )
+ *   gamma, beta  fp32 [K], 16-byte aligned;  other arguments as for qvggt_rotate_smooth_quantize_c8
+ */
+int qvggt_layernorm_rotate_smooth_quantize_c8(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M,
+                                              const float *gamma, const float *beta, float eps, signed char *Xq8,
+                                              float *a_scale, void *cuda_stream);
+
+/* The same LayerNorm alone (the unfused arm): Y_bf16 [M, K] contiguous bf16.  K must be 1024 or 4096. */
+int qvggt_layernorm(const void *X_bf16, long long ldx, int M, int K, const float *gamma, const float *beta, float eps,
+                    void *Y_bf16, void *cuda_stream);
+
 /* Frees the handle and its device memory (synchronises the device first).  NULL is allowed. */
 void qvggt_free_weights(qvggt_weights_t *w);
 

@@ -21,7 +21,8 @@ _STATUS_NAMES = {0: "QVGGT_OK", -1: "QVGGT_ERR_NULL", -2: "QVGGT_ERR_SHAPE", -3:
 EXPORTS = ("qvggt_prepare_weights", "qvggt_rotate_smooth_quantize", "qvggt_w4a4_linear", "qvggt_free_weights",
            "qvggt_weights_view", "qvggt_device_status", "qvggt_calibrate_smooth", "qvggt_status_string",
            "qvggt_quantize_weights_static", "qvggt_rotate_smooth_quantize_c8", "qvggt_w4a4_linear_c8",
-           "qvggt_weights_view_c8", "qvggt_rotate_smooth_quantize_static_c8")
+           "qvggt_weights_view_c8", "qvggt_rotate_smooth_quantize_static_c8",
+           "qvggt_layernorm_rotate_smooth_quantize_c8", "qvggt_layernorm")
 PREP_C8 = 1   # QVGGT_PREP_C8: keep an int8 [N, K] copy of the weight codes for the *_c8 entry points
 PREP_W8A8 = 2  # QVGGT_PREP_W8A8: 8-bit codes (one per byte only)
 
@@ -52,6 +53,8 @@ def lib() -> ctypes.CDLL:
         L.qvggt_rotate_smooth_quantize_c8.argtypes = [vp, vp, i64, i32, vp, vp, vp]
         L.qvggt_w4a4_linear_c8.argtypes = [vp, vp, vp, i32, vp, i64, vp, vp]
         L.qvggt_rotate_smooth_quantize_static_c8.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp]
+        L.qvggt_layernorm_rotate_smooth_quantize_c8.argtypes = [vp, vp, i64, i32, vp, vp, f32, vp, vp, vp]
+        L.qvggt_layernorm.argtypes = [vp, i64, i32, i32, vp, vp, f32, vp, vp]
         L.qvggt_weights_view_c8.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(i32)]
         L.qvggt_free_weights.argtypes = [vp]
         L.qvggt_free_weights.restype = None
@@ -240,6 +243,35 @@ def rotate_smooth_quantize_static_c8(w: Weights, X: torch.Tensor, delta: torch.T
     _check(lib().qvggt_rotate_smooth_quantize_static_c8(w.handle, _ptr(X), ldx, M, _ptr(delta), _ptr(Xq8), _ptr(a_scale),
                                                         _stream()), "qvggt_rotate_smooth_quantize_static_c8")
     return Xq8, a_scale
+
+
+def layernorm_rotate_smooth_quantize_c8(w: Weights, X: torch.Tensor, gamma: torch.Tensor, beta: torch.Tensor, eps: float = 1e-5,
+                                        Xq8: torch.Tensor | None = None, a_scale: torch.Tensor | None = None):
+    """LayerNorm (gamma, beta fp32 [K]) fused in front of rotate_smooth_quantize_c8 -> (Xq8 [M,K] int8, a_scale [M])."""
+    assert X.dim() == 2 and X.element_size() == 2 and X.stride(1) == 1 and X.shape[1] == w.K
+    assert gamma.dtype == torch.float32 and beta.dtype == torch.float32 and gamma.numel() == w.K and beta.numel() == w.K
+    M = X.shape[0]
+    if Xq8 is None:
+        Xq8 = torch.empty((M, w.K), dtype=torch.int8, device=X.device)
+    if a_scale is None:
+        a_scale = torch.empty((M,), dtype=torch.float32, device=X.device)
+    ldx = X.stride(0) if M > 1 else w.K
+    _check(lib().qvggt_layernorm_rotate_smooth_quantize_c8(w.handle, _ptr(X), ldx, M, _ptr(gamma), _ptr(beta), eps, _ptr(Xq8),
+                                                           _ptr(a_scale), _stream()), "qvggt_layernorm_rotate_smooth_quantize_c8")
+    return Xq8, a_scale
+
+
+def layernorm(X: torch.Tensor, gamma: torch.Tensor, beta: torch.Tensor, eps: float = 1e-5, Y: torch.Tensor | None = None):
+    """The same LayerNorm alone: X [M,K] bf16 -> Y [M,K] bf16 (K = 1024 or 4096)."""
+    assert X.dim() == 2 and X.element_size() == 2 and X.stride(1) == 1
+    M, K = X.shape
+    assert gamma.dtype == torch.float32 and beta.dtype == torch.float32 and gamma.numel() == K and beta.numel() == K
+    if Y is None:
+        Y = torch.empty((M, K), dtype=torch.bfloat16, device=X.device)
+    assert Y.is_contiguous() and Y.element_size() == 2
+    ldx = X.stride(0) if M > 1 else K
+    _check(lib().qvggt_layernorm(_ptr(X), ldx, M, K, _ptr(gamma), _ptr(beta), eps, _ptr(Y), _stream()), "qvggt_layernorm")
+    return Y
 
 
 def w4a4_linear_c8(w: Weights, Xq8: torch.Tensor, a_scale: torch.Tensor, Y: torch.Tensor | None = None,

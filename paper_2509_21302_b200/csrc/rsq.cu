@@ -185,17 +185,43 @@ __device__ __forceinline__ void stages_in_registers(float (&v)[N])
             if (!(k & h)) bfly2(v[k], v[k + 1], v[k + h], v[k + 1 + h]);
 }
 
+// Pairwise sum of N registers: adjacent pairs, recursively (the tree of the LayerNorm statistics).
+template <int N>
+__device__ __forceinline__ float tree_sum(const float (&a)[N])
+{
+    if constexpr (N == 1) {
+        return a[0];
+    } else {
+        float b[N / 2];
+#pragma unroll
+        for (int i = 0; i < N / 2; ++i) b[i] = __fadd_rn(a[2 * i], a[2 * i + 1]);
+        return tree_sum<N / 2>(b);
+    }
+}
+
+// Parameters of the LayerNorm that may run in front of the rotation (gamma == nullptr: none).
+struct LnArgs {
+    const float *gamma, *beta;   // fp32 [K]
+    float eps;
+    uint16_t *out;               // LN == 2 only: bf16 [M, K], the normalized rows (nothing else is computed)
+};
+
 // C8: one code per byte (int8, natural element order, row pitch K) instead of two per byte.
 // QMAX: largest code magnitude, 2^(N-1) - 1 of Eq. "quantization": 7 (N = 4) or, with C8 only, 127 (N = 8).
 // STATIC (C8 only): one given step size *static_delta for the whole tensor (the static tensor-wise arm of the
 // granularity ablation) instead of one per row from the row's absolute maximum; the clamp of Eq. "quantization"
 // to [-QMAX - 1, QMAX] is then active, and every row's scale is written as that step size.
-template <int LOGT, int GROUP, bool C8 = false, int QMAX = 7, bool STATIC = false>
+// LN: 1 = every row goes through LayerNorm first (fp32, statistics summed pairwise: in-thread tree over the thread's
+// T contiguous elements, then the xor-shuffle tree over the row's threads -- together the halves-recursion over the
+// row), its output rounded to bf16 as a separate normalization kernel would store it; 2 = only that, written out.
+template <int LOGT, int GROUP, bool C8 = false, int QMAX = 7, bool STATIC = false, int LN = 0>
 __global__ void __launch_bounds__(SqGeom<LOGT>::CTA_THREADS, LOGT == 5 ? 4 : 3)
 rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float *__restrict__ mul,
-              unsigned char *__restrict__ Xq, float *__restrict__ scales, const float *__restrict__ static_delta)
+              unsigned char *__restrict__ Xq, float *__restrict__ scales, const float *__restrict__ static_delta,
+              const LnArgs ln)
 {
     static_assert(!STATIC || (C8 && GROUP == 0), "the static step size is built for one code per byte");
+    static_assert(LN == 0 || (C8 && GROUP == 0 && !STATIC), "the fused LayerNorm is built for the dynamic one-code-per-byte path");
     using G = SqGeom<LOGT>;
     constexpr int T = G::T, K = G::K, CH = G::CH;
     constexpr int NG = (GROUP == 128) ? K / 128 : 1;           // scale groups per row
@@ -239,6 +265,18 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
     }
     cp_async_commit();
     const float delta = STATIC ? __ldg(static_delta) : 0.0f;
+    // LayerNorm parameters (T = 32): one copy per CTA in shared memory behind the row slots, as 16-byte pieces ordered
+    // [piece][thread], so that thread t reads its T contiguous gammas with conflict-free 16-byte loads
+    constexpr bool LN_SMEM = (LN != 0) && (LOGT == 5);
+    float4 *g_sm = reinterpret_cast<float4 *>(dsm + G::SMEM), *b_sm = g_sm + K / 4;
+    if constexpr (LN_SMEM) {
+        for (int i = threadIdx.x; i < K / 4; i += G::CTA_THREADS) {
+            const int dst = (i % (T / 4)) * T + i / (T / 4);
+            g_sm[dst] = __ldg(reinterpret_cast<const float4 *>(ln.gamma) + i);
+            b_sm[dst] = __ldg(reinterpret_cast<const float4 *>(ln.beta) + i);
+        }
+        __syncthreads();
+    }
     float m[T];                                                // multipliers of elements T k + t (loaded behind the first row's copies)
 #pragma unroll
     for (int k = 0; k < T; ++k) m[k] = __ldg(mul + T * k + t);
@@ -262,6 +300,11 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
                 const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
+                    if (LN) {                               // plain conversion: the normalization comes first
+                        v[8 * c + 2 * j] = __uint_as_float(w[j] << 16);
+                        v[8 * c + 2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+                        continue;
+                    }
                     // a 32-bit word holds elements 2i (low half) and 2i + 1 of the row: the first stage joins exactly
                     // these two, and the mixed-precision add takes the bf16 half as it is (its conversion is exact,
                     // so this is fl(float(lo) + float(hi)) and fl(float(lo) - float(hi)), one rounding each)
@@ -272,7 +315,63 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
                 }
             }
         }
-        stages_in_registers<T, false>(v);   // strides 2 .. T/2 (stride 1 was taken with the conversion)
+        if constexpr (LN != 0) {
+            // row sum over the tree: registers, lanes, and (T = 64) the two warps of the row
+            auto row_sum = [&](float part, int word) {
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) part = __fadd_rn(part, __shfl_xor_sync(0xFFFFFFFFu, part, o));
+                if (T == 64) {
+                    if (lane == 0) red[word + (t >> 5)] = part;
+                    group_sync<T>(slot);
+                    part = __fadd_rn(red[word], red[word + 1]);
+                }
+                return part;
+            };
+            constexpr float inv_k = 1.0f / K;                      // a power of two: the divisions are exact
+            const float mean = __fmul_rn(row_sum(tree_sum<T>(v), 8), inv_k);
+            // two elements per instruction where no multiply feeds an add (the bias add stays scalar: a packed multiply
+            // in front of a packed add was seen contracted into one fused operation)
+            const uint64_t mean2 = ptx::f32x2_pack(mean, mean);
+            uint64_t d2[T / 2];
+            float sq[T];
+#pragma unroll
+            for (int k = 0; k < T; k += 2) {
+                d2[k / 2] = ptx::f32x2_sub(ptx::f32x2_pack(v[k], v[k + 1]), mean2);
+                ptx::f32x2_unpack(ptx::f32x2_mul(d2[k / 2], d2[k / 2]), sq[k], sq[k + 1]);
+            }
+            const float var = __fmul_rn(row_sum(tree_sum<T>(sq), 10), inv_k);
+            const float rstd = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(var, ln.eps)));
+            const uint64_t rstd2 = ptx::f32x2_pack(rstd, rstd);
+            const float4 *g4 = reinterpret_cast<const float4 *>(ln.gamma + T * t), *b4 = reinterpret_cast<const float4 *>(ln.beta + T * t);
+            uint32_t packed[T / 2];
+#pragma unroll
+            for (int k = 0; k < T; k += 4) {
+                const float4 g = LN_SMEM ? g_sm[(k / 4) * T + t] : __ldg(g4 + k / 4), b = LN_SMEM ? b_sm[(k / 4) * T + t] : __ldg(b4 + k / 4);
+                float n0, n1, n2, n3;
+                ptx::f32x2_unpack(ptx::f32x2_mul(ptx::f32x2_mul(d2[k / 2], rstd2), ptx::f32x2_pack(g.x, g.y)), n0, n1);
+                ptx::f32x2_unpack(ptx::f32x2_mul(ptx::f32x2_mul(d2[k / 2 + 1], rstd2), ptx::f32x2_pack(g.z, g.w)), n2, n3);
+                // bf16 pair, round to nearest even: what a separate normalization kernel would have stored
+                const uint32_t p01 = ptx::pack_bf16x2(__fadd_rn(n0, b.x), __fadd_rn(n1, b.y));
+                const uint32_t p23 = ptx::pack_bf16x2(__fadd_rn(n2, b.z), __fadd_rn(n3, b.w));
+                v[k] = __uint_as_float(p01 << 16);
+                v[k + 1] = __uint_as_float(p01 & 0xFFFF0000u);
+                v[k + 2] = __uint_as_float(p23 << 16);
+                v[k + 3] = __uint_as_float(p23 & 0xFFFF0000u);
+                if (LN == 2) {
+                    packed[k / 2] = p01;
+                    packed[k / 2 + 1] = p23;
+                }
+            }
+            if constexpr (LN == 2) {
+                uint4 *dst = reinterpret_cast<uint4 *>(ln.out + row * K + T * t);
+#pragma unroll
+                for (int k = 0; k < T / 8; ++k) dst[k] = make_uint4(packed[4 * k], packed[4 * k + 1], packed[4 * k + 2], packed[4 * k + 3]);
+                continue;
+            }
+            stages_in_registers<T, true>(v);    // strides 1 .. T/2
+        } else {
+            stages_in_registers<T, false>(v);   // strides 2 .. T/2 (stride 1 was taken with the conversion)
+        }
 #pragma unroll
         for (int j = 0; j < T; ++j) Tm[j * T + ((((t >> 2) ^ (j & 7)) << 2) | (t & 3))] = v[j];
         group_sync<T>(slot);
@@ -459,14 +558,15 @@ namespace {
 
 // Launch with programmatic stream serialization allowed: the blocks may become resident while the previous
 // kernel of the stream drains (they wait in grid_dependency_wait() before touching global memory).
-template <int LOGT, int GROUP, bool C8, int QMAX = 7, bool STATIC = false>
+template <int LOGT, int GROUP, bool C8, int QMAX = 7, bool STATIC = false, int LN = 0>
 cudaError_t launch_sq(const uint16_t *x, long long ldx, int M, const float *mul, unsigned char *out, float *scales,
-                      cudaStream_t st, const float *static_delta = nullptr)
+                      cudaStream_t st, const float *static_delta = nullptr, LnArgs ln = LnArgs{nullptr, nullptr, 0.0f, nullptr})
 {
     using G = SqGeom<LOGT>;
+    constexpr int SMEM = G::SMEM + ((LN != 0 && LOGT == 5) ? 2 * G::K * 4 : 0);   // + the CTA's copy of gamma and beta
     static bool configured = false;       // per process and instantiation
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(rsq_sq_kernel<LOGT, GROUP, C8, QMAX, STATIC>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM);
+        cudaError_t e = cudaFuncSetAttribute(rsq_sq_kernel<LOGT, GROUP, C8, QMAX, STATIC, LN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
         if (e != cudaSuccess) return e;
         configured = true;
     }
@@ -476,11 +576,11 @@ cudaError_t launch_sq(const uint16_t *x, long long ldx, int M, const float *mul,
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(rsq_grid(M, G::ROWS, LOGT == 5 ? 4 : 3));
     cfg.blockDim = dim3(G::CTA_THREADS);
-    cfg.dynamicSmemBytes = G::SMEM;
+    cfg.dynamicSmemBytes = SMEM;
     cfg.stream = st;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, rsq_sq_kernel<LOGT, GROUP, C8, QMAX, STATIC>, x, ldx, M, mul, out, scales, static_delta);
+    return cudaLaunchKernelEx(&cfg, rsq_sq_kernel<LOGT, GROUP, C8, QMAX, STATIC, LN>, x, ldx, M, mul, out, scales, static_delta, ln);
 }
 
 }  // namespace
@@ -507,6 +607,23 @@ cudaError_t qvggt_launch_rsq_static_c8(const void *X, long long ldx, int M, int 
                          : launch_sq<6, 0, true, 127, true>(x, ldx, M, mul, out, scales, st, delta);
     return K == 1024 ? launch_sq<5, 0, true, 7, true>(x, ldx, M, mul, out, scales, st, delta)
                      : launch_sq<6, 0, true, 7, true>(x, ldx, M, mul, out, scales, st, delta);
+}
+
+cudaError_t qvggt_launch_ln_rsq_c8(const void *X, long long ldx, int M, int K, const float *mul, int bits, const float *gamma,
+                                   const float *beta, float eps, signed char *Xq8, float *scales, void *ln_out, cudaStream_t st)
+{
+    if (M == 0) return cudaSuccess;
+    const uint16_t *x = static_cast<const uint16_t *>(X);
+    unsigned char *out = reinterpret_cast<unsigned char *>(Xq8);
+    const LnArgs ln = {gamma, beta, eps, static_cast<uint16_t *>(ln_out)};
+    if (ln_out)       // the normalization alone
+        return K == 1024 ? launch_sq<5, 0, true, 7, false, 2>(x, ldx, M, mul, out, scales, st, nullptr, ln)
+                         : launch_sq<6, 0, true, 7, false, 2>(x, ldx, M, mul, out, scales, st, nullptr, ln);
+    if (bits == 8)
+        return K == 1024 ? launch_sq<5, 0, true, 127, false, 1>(x, ldx, M, mul, out, scales, st, nullptr, ln)
+                         : launch_sq<6, 0, true, 127, false, 1>(x, ldx, M, mul, out, scales, st, nullptr, ln);
+    return K == 1024 ? launch_sq<5, 0, true, 7, false, 1>(x, ldx, M, mul, out, scales, st, nullptr, ln)
+                     : launch_sq<6, 0, true, 7, false, 1>(x, ldx, M, mul, out, scales, st, nullptr, ln);
 }
 
 cudaError_t qvggt_launch_rsq(const void *X, long long ldx, int M, int K, const float *mul, int group,
