@@ -4,7 +4,7 @@
 One "step" = one pass of the whole online hot path over one batch: for each of the four linears of
 one aggregator block (qkv 1024->3072, proj 1024->1024, fc1 1024->4096, fc2 4096->1024) at 8 frames
 (M = 10992 tokens): rotate-smooth-quantize, then W4A4 GEMM + rescale + bias + bf16.  Weight
-preparation is offline and untimed.  Prints ONE JSON line (see the design doc for the fields).
+preparation is offline and untimed.  Prints ONE JSON line.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 """
@@ -399,7 +399,7 @@ def run_ours(args, rank, world, local_rank):
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": f"int{path.bits} x int{path.bits} -> int32 (fp32 rotation and scales)", "data": "synthetic",
         "tokens_per_s": world * M / (ms_per_step * 1e-3),
-        "config": {"workload": "aggregator block, 4 linears (qkv/proj/fc1/fc2), 8 frames M=10992 per GPU (BASELINE configs[1])",
+        "config": {"workload": "aggregator block, 4 linears (qkv/proj/fc1/fc2), 8 frames M=10992 per GPU",
                    "l2": f"step working set ~400 MB > 126 MB L2; {NBUF} buffer sets alternated per step",
                    "timed": "rotate-smooth-quantize + W4A4 GEMM/epilogue per linear; weight prep offline; one event pair "
                             "around the K steps; the per-kernel durations behind roofline / per_layer come from a second pass "
@@ -435,7 +435,7 @@ def run_ours(args, rank, world, local_rank):
 
 
 def run_rsq_sweep(args):
-    """BASELINE configs[2]: rotate-smooth-quantize alone, M = 1374 x {1..100}, K in {1024, 4096}, Student-t(3)
+    """The quantize-kernel sweep: rotate-smooth-quantize alone, M = 1374 x {1..100}, K in {1024, 4096}, Student-t(3)
     entries with 1 % outlier channels; achieved GB/s against the measured copy bandwidth (one JSON line)."""
     import torch
     import paper_2509_21302_b200 as q
@@ -508,7 +508,7 @@ def run_rsq_sweep(args):
     best = max(v["gbs"] for v in out.values())
     print(json.dumps({"metric": "rsq_gbs", "value": best, "unit": "GB/s", "n_gpus": 1, "higher_is_better": True,
                       "dtype": "fp32 rotation -> int4", "data": "synthetic",
-                      "config": {"workload": "rotate-smooth-quantize sweep (BASELINE configs[2]); L2 flushed between launches",
+                      "config": {"workload": "rotate-smooth-quantize sweep, M = 1374 x {1, 8, 32, 100}; L2 flushed between launches",
                                  "code_format": path.fmt},
                       "roofline": {"bound": "hbm", "achieved": best, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                    "frac": best / peaks["hbm_gbs"], "peak_note": f"of {peaks['source']}", "traffic": None},
@@ -516,7 +516,7 @@ def run_rsq_sweep(args):
 
 
 def run_stack(args):
-    """BASELINE configs[3]: the full 48-block linear stack (24 frame + 24 global blocks, 4 linears each) at 32
+    """The full 48-block linear stack (24 frame + 24 global blocks, 4 linears each) at 32
     frames (M = 43968): per-layer seeded weights, bias and smoothing factors; activations of the four layer
     kinds come from the seeded heavy-tailed generator (one tensor per kind, reused by every block: there is no
     data dependence between layers in this benchmark).  Reports end-to-end linear time and tokens/s."""
@@ -568,7 +568,7 @@ def run_stack(args):
                       "steps": reps, "ms_per_step": ms, "higher_is_better": True, "data": "synthetic",
                       "dtype": "int4 x int4 -> int32 (fp32 rotation and scales)", "tokens_per_s": M / (ms * 1e-3),
                       "gpu_launches": 2 * len(handles) * reps,
-                      "config": {"workload": "48-block linear stack, 32 frames M=43968 (BASELINE configs[3])",
+                      "config": {"workload": "48-block linear stack, 32 frames M=43968",
                                  "l2": "per-layer working set 90-450 MB > 126 MB L2", "code_format": path.fmt}}))
 
 
@@ -584,7 +584,8 @@ def main():
                     help="storage of the int4 codes between the kernels: c8 = one per byte (default), packed = two per byte; "
                          "w8a8 = the paper's 8-bit setting through the same kernels (not the headline metric)")
     ap.add_argument("--workload", choices=["block", "rsq_sweep", "stack"], default="block",
-                    help="block = BASELINE configs[1] (the default, the contract line); rsq_sweep = configs[2]")
+                    help="block = one aggregator block at 8 frames (the default line); rsq_sweep = the quantize kernel alone over M; "
+                         "stack = all 48 blocks at 32 frames")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

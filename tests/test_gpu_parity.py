@@ -213,7 +213,7 @@ def test_calibrate_smooth_matches_oracle(K):
     assert np.allclose(got, want, rtol=2e-5, atol=0)
 
 
-# ------------------------------------------------------------------------------ config 1 (benchmark configs[0])
+# ------------------------------------------------------------------------------ the single-frame proj layer (the smallest benchmark configuration)
 def test_config1_single_frame_proj():
     spec = workload.LinearSpec("proj", 1024, 1024, workload.DIST_NORMAL, 0, 1)
     L = make_layer(spec, calib_rows=workload.TOKENS_PER_FRAME)

@@ -1,4 +1,4 @@
-"""The seeded input generator: deterministic, row-addressable, with the structure the design doc states."""
+"""The seeded input generator: deterministic, row-addressable, with the structure of VGGT activations (outlier channels, special-token rows)."""
 import numpy as np
 
 import workload
