@@ -183,3 +183,39 @@ def test_c8_chained_launches_are_deterministic():
         if i % 6 == 5:
             assert torch.equal(Y.view(torch.int16), Y0.view(torch.int16)) and torch.equal(Xq8, q0) and torch.equal(a_scale, a0), i
     assert L["h"].device_status() == 0
+
+
+def test_c8_entry_points_validate_their_arguments():
+    """Bad arguments are refused on the host with the documented status, before anything is launched."""
+    import ctypes
+    from paper_2509_21302_b200 import binding as B
+    L = B.lib()
+    K, N, M = 1024, 128, 16
+    h = q.prepare_weights(dev_bf16(workload.normal_bf16(1, 1, N, K, 0.02)), None, torch.ones(K, device="cuda"), None, c8=True)
+    X = torch.zeros((M, K), dtype=torch.bfloat16, device="cuda")
+    Xq8 = torch.zeros((M, K + 16), dtype=torch.int8, device="cuda")
+    a = torch.zeros(M, dtype=torch.float32, device="cuda")
+    Y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    g = torch.ones(K + 4, dtype=torch.float32, device="cuda")
+    st = torch.cuda.current_stream().cuda_stream
+    hp, xp, qp, ap, yp, gp = h.handle, X.data_ptr(), Xq8.data_ptr(), a.data_ptr(), Y.data_ptr(), g.data_ptr()
+    NULL, SHAPE, ALIGN, UNSUP = -1, -2, -3, -4
+    assert L.qvggt_rotate_smooth_quantize_c8(None, xp, K, M, qp, ap, st) == NULL
+    assert L.qvggt_rotate_smooth_quantize_c8(hp, xp, K, -1, qp, ap, st) == SHAPE
+    assert L.qvggt_rotate_smooth_quantize_c8(hp, xp, K - 8, M, qp, ap, st) == SHAPE          # row stride below K
+    assert L.qvggt_rotate_smooth_quantize_c8(hp, xp, K + 4, M, qp, ap, st) == ALIGN          # row stride not a multiple of 8
+    assert L.qvggt_rotate_smooth_quantize_c8(hp, xp, K, M, qp + 4, ap, st) == ALIGN
+    assert L.qvggt_rotate_smooth_quantize_c8(hp, xp, K, M, None, ap, st) == NULL
+    assert L.qvggt_rotate_smooth_quantize_c8(hp, xp, K, 0, None, None, st) == 0              # M = 0 is a no-op
+    assert L.qvggt_w4a4_linear_c8(hp, qp, ap, M, yp, N - 8, None, st) == SHAPE
+    assert L.qvggt_w4a4_linear_c8(hp, qp, ap, M, yp + 2, N, None, st) == ALIGN
+    assert L.qvggt_w4a4_linear_c8(hp, None, ap, M, yp, N, None, st) == NULL
+    assert L.qvggt_rotate_smooth_quantize_static_c8(hp, xp, K, M, None, qp, ap, st) == NULL  # no step size
+    assert L.qvggt_layernorm_rotate_smooth_quantize_c8(hp, xp, K, M, gp, None, 1e-5, qp, ap, st) == NULL
+    assert L.qvggt_layernorm_rotate_smooth_quantize_c8(hp, xp, K, M, gp + 4, gp, 1e-5, qp, ap, st) == ALIGN
+    assert L.qvggt_layernorm(xp, K, M, 2048, gp, gp, 1e-5, yp, st) == SHAPE                   # K must be 1024 or 4096
+    out = ctypes.c_void_p()
+    assert L.qvggt_prepare_weights(xp, None, gp, None, N, K, 8, st, ctypes.byref(out)) == UNSUP   # unknown flag
+    assert out.value is None
+    torch.cuda.synchronize()
+    assert h.device_status() == 0
