@@ -36,6 +36,9 @@
  *     before anything is launched; nothing throws or exits.
  *   - Device-side waits are bounded.  If one expires the kernel records a code in the handle's
  *     status word and returns; read it with qvggt_device_status().
+ *   - One process may drive several devices: a handle is bound to the device that was current when it was
+ *     prepared, every other call uses the current device, and the library's caches (kernel attributes,
+ *     occupancy, SM count) are kept per device.
  */
 #ifndef QVGGT_H
 #define QVGGT_H
@@ -68,7 +71,8 @@ typedef enum {
  *   bias_bf16 [N] bf16 or NULL (no bias)
  *   smooth_c  [K] fp32, finite and > 0
  *   sign_v    [K] int8 of +1/-1, or NULL (all +1)
- *   flags     0, QVGGT_PREP_C8 to keep an extra int8 [N, K] copy of the codes for the *_c8 entry points, or
+ *   flags     0, QVGGT_PREP_C8 to keep an extra int8 [N, K] copy of the codes for the *_c8 entry points (1.5 bytes
+ *             per weight in all), QVGGT_PREP_C8_ONLY to keep only that copy (1 byte per weight), or
  *             QVGGT_PREP_W8A8 for 8-bit codes (see the *_c8 entry points)
  *   out       receives a new handle (device memory is allocated here, on the current device);
  *             release it with qvggt_free_weights.  The handle is bound to that device.
@@ -124,6 +128,7 @@ int qvggt_w4a4_linear(const qvggt_weights_t *w, const unsigned char *Xq, const f
  */
 #define QVGGT_PREP_C8 1
 #define QVGGT_PREP_W8A8 2
+#define QVGGT_PREP_C8_ONLY 4 /* 4-bit codes one per byte only, no packed copy (1 byte per weight; the packed entry points refuse the handle) */
 int qvggt_rotate_smooth_quantize_c8(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M,
                                     signed char *Xq8, float *a_scale, void *cuda_stream);
 int qvggt_w4a4_linear_c8(const qvggt_weights_t *w, const signed char *Xq8, const float *a_scale, int M,
@@ -157,6 +162,18 @@ int qvggt_layernorm_rotate_smooth_quantize_c8(const qvggt_weights_t *w, const vo
 /* The same LayerNorm alone (the unfused arm): Y_bf16 [M, K] contiguous bf16.  K must be 1024 or 4096. */
 int qvggt_layernorm(const void *X_bf16, long long ldx, int M, int K, const float *gamma, const float *beta, float eps,
                     void *Y_bf16, void *cuda_stream);
+
+/*
+ * Test hook for the bounded device-side waits (the paper has no counterpart).  Launches the GEMM of
+ * qvggt_w4a4_linear_c8 with its TMA producers switched off and every wait limited to wait_limit_cycles
+ * (1000 .. 2e9) SM cycles: no operand ever arrives, the first wait runs out, the kernel records the code of that
+ * wait in the handle's status word, releases its tensor memory and returns -- nothing faults, traps or spins
+ * without bound, and no asynchronous operation is in flight when it leaves.  Y_bf16 is not written.  Afterwards
+ * qvggt_device_status() on this handle reports QVGGT_ERR_DEVICE_TIMEOUT (the status word is sticky: use a fresh
+ * handle for real work).  Arguments as for qvggt_w4a4_linear_c8 (M >= 1).
+ */
+int qvggt_debug_starved_linear_c8(const qvggt_weights_t *w, const signed char *Xq8, const float *a_scale, int M,
+                                  void *Y_bf16, long long ldy, long long wait_limit_cycles, void *cuda_stream);
 
 /* Frees the handle and its device memory (synchronises the device first).  NULL is allowed. */
 void qvggt_free_weights(qvggt_weights_t *w);

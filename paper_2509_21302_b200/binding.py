@@ -22,9 +22,10 @@ EXPORTS = ("qvggt_prepare_weights", "qvggt_rotate_smooth_quantize", "qvggt_w4a4_
            "qvggt_weights_view", "qvggt_device_status", "qvggt_calibrate_smooth", "qvggt_status_string",
            "qvggt_quantize_weights_static", "qvggt_rotate_smooth_quantize_c8", "qvggt_w4a4_linear_c8",
            "qvggt_weights_view_c8", "qvggt_rotate_smooth_quantize_static_c8",
-           "qvggt_layernorm_rotate_smooth_quantize_c8", "qvggt_layernorm")
+           "qvggt_layernorm_rotate_smooth_quantize_c8", "qvggt_layernorm", "qvggt_debug_starved_linear_c8")
 PREP_C8 = 1   # QVGGT_PREP_C8: keep an int8 [N, K] copy of the weight codes for the *_c8 entry points
 PREP_W8A8 = 2  # QVGGT_PREP_W8A8: 8-bit codes (one per byte only)
+PREP_C8_ONLY = 4  # QVGGT_PREP_C8_ONLY: 4-bit codes one per byte only (no packed copy)
 
 
 class QvggtError(RuntimeError):
@@ -55,6 +56,7 @@ def lib() -> ctypes.CDLL:
         L.qvggt_rotate_smooth_quantize_static_c8.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp]
         L.qvggt_layernorm_rotate_smooth_quantize_c8.argtypes = [vp, vp, i64, i32, vp, vp, f32, vp, vp, vp]
         L.qvggt_layernorm.argtypes = [vp, i64, i32, i32, vp, vp, f32, vp, vp]
+        L.qvggt_debug_starved_linear_c8.argtypes = [vp, vp, vp, i32, vp, i64, i64, vp]
         L.qvggt_weights_view_c8.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(i32)]
         L.qvggt_free_weights.argtypes = [vp]
         L.qvggt_free_weights.restype = None
@@ -163,11 +165,11 @@ def _from_device_ptr(ptr: int, nbytes: int, dtype: torch.dtype, shape) -> torch.
 
 
 def prepare_weights(W: torch.Tensor, bias: torch.Tensor | None, smooth_c: torch.Tensor,
-                    sign_v: torch.Tensor | None = None, c8: bool = False, bits: int = 4) -> Weights:
+                    sign_v: torch.Tensor | None = None, c8: bool | str = False, bits: int = 4) -> Weights:
     """W [N,K] bf16, bias [N] bf16 or None, smooth_c [K] fp32, sign_v [K] int8 (+1/-1) or None.
-    c8: also keep the codes one per byte, as the *_c8 entry points need them.
+    c8: True = also keep the codes one per byte, as the *_c8 entry points need them; "only" = keep only that copy.
     bits: 4 (W4A4) or 8 (W8A8: one code per byte only; use the *_c8 entry points)."""
-    assert bits in (4, 8)
+    assert bits in (4, 8) and c8 in (False, True, "only")
     assert W.dim() == 2 and W.element_size() == 2 and W.is_contiguous()
     N, K = W.shape
     assert smooth_c.dtype == torch.float32 and smooth_c.numel() == K and smooth_c.is_contiguous()
@@ -176,7 +178,8 @@ def prepare_weights(W: torch.Tensor, bias: torch.Tensor | None, smooth_c: torch.
     if sign_v is not None:
         assert sign_v.dtype == torch.int8 and sign_v.numel() == K and sign_v.is_contiguous()
     h = ctypes.c_void_p()
-    _check(lib().qvggt_prepare_weights(_ptr(W), _ptr(bias), _ptr(smooth_c), _ptr(sign_v), N, K, PREP_W8A8 if bits == 8 else (PREP_C8 if c8 else 0), _stream(),
+    _check(lib().qvggt_prepare_weights(_ptr(W), _ptr(bias), _ptr(smooth_c), _ptr(sign_v), N, K,
+                                       PREP_W8A8 if bits == 8 else (PREP_C8_ONLY if c8 == "only" else (PREP_C8 if c8 else 0)), _stream(),
                                        ctypes.byref(h)), "qvggt_prepare_weights")
     return Weights(h.value, N, K)
 
@@ -289,6 +292,14 @@ def w4a4_linear_c8(w: Weights, Xq8: torch.Tensor, a_scale: torch.Tensor, Y: torc
     _check(lib().qvggt_w4a4_linear_c8(w.handle, _ptr(Xq8), _ptr(a_scale), M, _ptr(Y), ldy, _ptr(acc_debug), _stream()),
            "qvggt_w4a4_linear_c8")
     return Y
+
+
+def debug_starved_linear_c8(w: Weights, Xq8: torch.Tensor, a_scale: torch.Tensor, Y: torch.Tensor, wait_limit_cycles: int) -> int:
+    """Test hook: the GEMM launch with its loads switched off and short wait limits; returns the C status of the launch
+    (the expired wait shows in w.device_status())."""
+    M = Xq8.shape[0]
+    return lib().qvggt_debug_starved_linear_c8(w.handle, _ptr(Xq8), _ptr(a_scale), M, _ptr(Y), Y.stride(0) if M > 1 else w.N,
+                                               wait_limit_cycles, _stream())
 
 
 def calibrate_smooth(X_calib: torch.Tensor, W: torch.Tensor, alpha: float = 0.5, lo: float = 1e-2,

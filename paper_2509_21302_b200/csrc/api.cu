@@ -36,9 +36,10 @@ extern "C" {
 int qvggt_prepare_weights(const void *W_bf16, const void *bias_bf16, const float *smooth_c, const signed char *sign_v,
                           int N, int K, int flags, void *cuda_stream, qvggt_weights_t **out)
 {
-    if (flags & ~(QVGGT_PREP_C8 | QVGGT_PREP_W8A8)) return QVGGT_ERR_UNSUPPORTED;
+    if (flags & ~(QVGGT_PREP_C8 | QVGGT_PREP_W8A8 | QVGGT_PREP_C8_ONLY)) return QVGGT_ERR_UNSUPPORTED;
     const bool w8 = (flags & QVGGT_PREP_W8A8) != 0;       // 8-bit codes exist one per byte only
-    const bool c8 = w8 || (flags & QVGGT_PREP_C8) != 0;
+    const bool c8 = w8 || (flags & (QVGGT_PREP_C8 | QVGGT_PREP_C8_ONLY)) != 0;
+    const bool packed = !w8 && !(flags & QVGGT_PREP_C8_ONLY);
     if (!out) return QVGGT_ERR_NULL;
     *out = nullptr;
     if (!W_bf16 || !smooth_c) return QVGGT_ERR_NULL;
@@ -55,7 +56,7 @@ int qvggt_prepare_weights(const void *W_bf16, const void *bias_bf16, const float
     w->Wq = nullptr; w->Wq8 = nullptr; w->w_scale = nullptr; w->amul = nullptr; w->bias = nullptr; w->status = nullptr;
     cudaGetDevice(&w->device);
     float *wmul = nullptr;
-    bool ok = (w8 || cudaMalloc(&w->Wq, (size_t)N * K / 2) == cudaSuccess) &&
+    bool ok = (!packed || cudaMalloc(&w->Wq, (size_t)N * K / 2) == cudaSuccess) &&
               cudaMalloc(&w->w_scale, sizeof(float) * N) == cudaSuccess &&
               cudaMalloc(&w->amul, sizeof(float) * K) == cudaSuccess &&
               cudaMalloc(&w->status, sizeof(int)) == cudaSuccess &&
@@ -104,7 +105,7 @@ int qvggt_w4a4_linear(const qvggt_weights_t *w, const unsigned char *Xq, const f
 {
     if (!w) return QVGGT_ERR_NULL;
     if (M < 0) return QVGGT_ERR_SHAPE;
-    if ((group != 0 && group != 128) || w->bits != 4) return QVGGT_ERR_UNSUPPORTED;
+    if ((group != 0 && group != 128) || w->bits != 4 || !w->Wq) return QVGGT_ERR_UNSUPPORTED;
     if (M == 0) return QVGGT_OK;
     if (!Xq || !a_scale || !Y_bf16) return QVGGT_ERR_NULL;
     if (ldy < w->N) return QVGGT_ERR_SHAPE;
@@ -171,7 +172,7 @@ int qvggt_layernorm(const void *X_bf16, long long ldx, int M, int K, const float
     if (ldx < K) return QVGGT_ERR_SHAPE;
     if (ldx % 8 != 0 || !aligned16(X_bf16) || !aligned16(Y_bf16) || !aligned16(gamma) || !aligned16(beta)) return QVGGT_ERR_ALIGN;
     if (!device_is_sm100()) return QVGGT_ERR_UNSUPPORTED;
-    cudaError_t e = qvggt_launch_ln_rsq_c8(X_bf16, ldx, M, K, gamma, 4, gamma, beta, eps, nullptr, nullptr, Y_bf16,
+    cudaError_t e = qvggt_launch_ln_rsq_c8(X_bf16, ldx, M, K, nullptr, 4, gamma, beta, eps, nullptr, nullptr, Y_bf16,
                                            static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
 }
@@ -193,15 +194,28 @@ int qvggt_w4a4_linear_c8(const qvggt_weights_t *w, const signed char *Xq8, const
     return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
 }
 
+int qvggt_debug_starved_linear_c8(const qvggt_weights_t *w, const signed char *Xq8, const float *a_scale, int M, void *Y_bf16,
+                                  long long ldy, long long wait_limit_cycles, void *cuda_stream)
+{
+    if (!w) return QVGGT_ERR_NULL;
+    if (!w->Wq8) return QVGGT_ERR_UNSUPPORTED;
+    if (M < 1 || ldy < w->N || wait_limit_cycles < 1000 || wait_limit_cycles > 2000000000LL) return QVGGT_ERR_SHAPE;
+    if (!Xq8 || !a_scale || !Y_bf16) return QVGGT_ERR_NULL;
+    if (ldy % 8 != 0 || !aligned16(Xq8) || !aligned16(Y_bf16) || (reinterpret_cast<uintptr_t>(a_scale) & 3u)) return QVGGT_ERR_ALIGN;
+    cudaError_t e = qvggt_launch_gemm_c8_starved(w, Xq8, a_scale, M, Y_bf16, ldy, wait_limit_cycles, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
+}
+
 void qvggt_free_weights(qvggt_weights_t *w)
 {
     if (!w) return;
     int cur = 0;
     cudaGetDevice(&cur);
-    if (cur != w->device) cudaSetDevice(w->device);
+    const int owner = w->device;
+    if (cur != owner) cudaSetDevice(owner);
     cudaDeviceSynchronize();
     release(w);
-    if (cur != w->device) cudaSetDevice(cur);
+    if (cur != owner) cudaSetDevice(cur);
 }
 
 int qvggt_weights_view(const qvggt_weights_t *w, const unsigned char **Wq, const float **w_scale, const float **amul,

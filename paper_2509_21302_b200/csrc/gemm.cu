@@ -9,9 +9,10 @@
 // land in separate 16-byte chunks; the same permutation of K is applied to both operands, so the
 // dot product is unchanged.
 //
-// Persistent and warp-specialised.  A "worker" is one CTA (CG = 1: tile 128 tokens x 256 channels)
-// or a pair of CTAs on neighbouring SMs (CG = 2: tile 256 x 256, each CTA stages 128 token rows and
-// 128 weight rows, one thread of the leader CTA issues tcgen05.mma.cta_group::2 for both).
+// Persistent and warp-specialised.  A "worker" is a pair of CTAs on neighbouring SMs (tile 256 x 256, each
+// CTA stages 128 token rows and 128 weight rows, one thread of the leader CTA issues tcgen05.mma.cta_group::2
+// for both; a single-CTA configuration measured 10-35 % slower on every VGGT shape: the pair halves the
+// weight traffic).
 //   warps 0-7    epilogue: TMEM -> registers -> scale, bias, bf16 -> swizzled staging -> TMA store
 //   warps 8-15   converters: packed stage -> registers -> int8 operand stage
 //   warp  16     one thread issues tcgen05.mma and the commits that release stages / publish accumulators
@@ -21,11 +22,14 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include "gemm_common.cuh"
 #include "qvggt_internal.cuh"
 #include "sm100_ptx.cuh"
 #include "tensor_map.cuh"
 
 namespace {
+
+using gemmc::STG_BYTES;
 
 constexpr int BM = 128;            // token rows per CTA (TMEM lanes)
 constexpr int BN = 256;            // output channels per tile
@@ -37,19 +41,19 @@ constexpr int MMA_WARP = EPI_WARPS + CONV_WARPS;
 constexpr int TMA_WARP = MMA_WARP + 1;
 constexpr int THREADS = (TMA_WARP + 1) * 32;
 constexpr int ACC_BUFS = 2;        // TMEM accumulators: the epilogue of tile i overlaps the MMAs of tile i+1
-constexpr int STG_BYTES = 32 * 64;    // per epilogue warp: 32 rows x 32 bf16, 64-byte swizzled
 
-template <int CG>
-struct Cfg {
+constexpr int CG = 2;               // CTAs per worker
+
+struct C {
     static constexpr int B_ROWS = BN / CG;                 // weight rows staged by one CTA
     static constexpr int ROWS = BM + B_ROWS;
     static constexpr int PK_STAGE = ROWS * (BK / 2);       // packed codes
     static constexpr int UP_STAGE = ROWS * BK;             // int8 operands
     static constexpr int PS = 4;                           // packed stages (cover the L2 latency)
-    static constexpr int US = (CG == 1) ? 2 : 4;           // operand stages (decouple converters and MMA)
+    static constexpr int US = 4;                           // operand stages (decouple converters and MMA)
     // Converter warps form GROUPS independent groups; group g converts K-blocks g, g + GROUPS, ...  so the
     // fixed costs of a stage (draining the stores, the proxy fence, barrier round trips) overlap.
-    static constexpr int GROUPS = (CG == 1) ? 2 : 4;
+    static constexpr int GROUPS = 4;
     static constexpr int GROUP_WARPS = CONV_WARPS / GROUPS;
     static constexpr int GROUP_THREADS = GROUP_WARPS * 32;
     static constexpr int CHUNKS = ROWS * 4 / GROUP_THREADS;   // 16-byte packed pieces per thread per stage
@@ -71,14 +75,13 @@ struct Cfg {
 
 // DUMP: also write the int32 sums to acc_debug (a separate instantiation keeps that code, and the registers it
 // pins, out of the production kernel)
-template <int CG, bool DUMP>
+template <bool DUMP>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                  const __grid_constant__ CUtensorMap map_y, const float *__restrict__ a_scale,
                  const float *__restrict__ w_scale, const uint16_t *__restrict__ bias, int *__restrict__ acc_debug,
                  int M, int N, int K, int *status)
 {
-    using C = Cfg<CG>;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = ptx::smem_addr(smem);
@@ -93,7 +96,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     volatile int *s_flags = reinterpret_cast<volatile int *>(smem + C::OFF_FLAGS);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t rank = (CG == 2) ? ptx::cluster_ctarank() : 0u;     // 0 = leader of the pair
+    const uint32_t rank = ptx::cluster_ctarank();                       // 0 = leader of the pair
     const int worker = blockIdx.x / CG, workers = gridDim.x / CG;
     const int KB = K / BK;
     const int n_tiles = (N + BN - 1) / BN;
@@ -116,10 +119,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         *s_abort = 0;
         ptx::fence_mbar_init();
     }
-    if (warp == MMA_WARP) {
-        if (CG == 2) { ptx::tmem_alloc_pair(ptx::smem_addr(s_tmem), C::TMEM_COLS); ptx::tmem_relinquish_pair(); }
-        else         { ptx::tmem_alloc(ptx::smem_addr(s_tmem), C::TMEM_COLS);      ptx::tmem_relinquish(); }
-    }
+    if (warp == MMA_WARP) { ptx::tmem_alloc_pair(ptx::smem_addr(s_tmem), C::TMEM_COLS); ptx::tmem_relinquish_pair(); }
     if (warp == TMA_WARP && lane == 0) {
         ptx::prefetch_tensormap(&map_x);
         ptx::prefetch_tensormap(&map_w);
@@ -127,7 +127,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (CG == 2) ptx::cluster_sync();        // the peer's barriers exist before anything arrives on them remotely
+    ptx::cluster_sync();                     // the peer's barriers exist before anything arrives on them remotely
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *s_tmem;
 
@@ -138,7 +138,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         const uint32_t stg_addr = sbase + C::OFF_STG + warp * STG_BYTES;
         float *s_ws = reinterpret_cast<float *>(smem + C::OFF_CH);          // [2][BN] per-channel scale of the tile
         float *s_bs = s_ws + ACC_BUFS * BN;                                   // [2][BN] bias as fp32
-        const uint32_t leader_tempty = (CG == 2) ? ptx::map_to_cta(bar_tempty, 0) : bar_tempty;
+        const uint32_t leader_tempty = ptx::map_to_cta(bar_tempty, 0);
         bool alive = true;
         uint32_t toggle = 0;
         for (int t = 0; t < my_tiles; ++t) {
@@ -152,12 +152,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             const bool cols_ok = n0 < N;                       // N is a multiple of 128: a half tile is all in or all out
             // per-channel scale and bias of the tile -> shared memory; buffer b was last read two tiles ago,
             // and every epilogue warp has passed the group barrier of the tile in between since then
-            {
-                const int e = threadIdx.x;                     // 0..255: one channel each
-                const bool ch_ok = nt0 + e < N;
-                s_ws[b * BN + e] = ch_ok ? __ldg(w_scale + nt0 + e) : 0.0f;
-                s_bs[b * BN + e] = (ch_ok && bias) ? __uint_as_float(static_cast<uint32_t>(__ldg(bias + nt0 + e)) << 16) : 0.0f;
-            }
+            gemmc::load_channel_params(s_ws + b * BN, s_bs + b * BN, w_scale, bias, nt0, N, threadIdx.x);   // 256 threads, one channel each
             // a_scale / 256: exact (power of two), cancels the factor 256 carried by the raw accumulator
             const float as = row_ok ? __fmul_rn(__ldg(a_scale + gm), 0.00390625f) : 0.0f;
             const uint64_t as2 = ptx::f32x2_pack(as, as);
@@ -178,53 +173,15 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                         // last read of this accumulator: hand it back to the MMA thread before the math
                         ptx::tc_fence_before_sync();
                         __syncwarp();
-                        if (lane == 0) {
-                            if (CG == 2) ptx::mbar_arrive_cluster(leader_tempty + 8 * b);
-                            else ptx::mbar_arrive(bar_tempty + 8 * b);
-                        }
+                        if (lane == 0) ptx::mbar_arrive_cluster(leader_tempty + 8 * b);
                     }
                     if (cols_ok) {
                         uint32_t out[16];
-#pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            const ulonglong2 w2 = *reinterpret_cast<const ulonglong2 *>(wsb + col + j);
-                            const ulonglong2 b2 = *reinterpret_cast<const ulonglong2 *>(bsb + col + j);
-                            uint64_t z01 = ptx::f32x2_pack(static_cast<float>(static_cast<int>(raw[j])), static_cast<float>(static_cast<int>(raw[j + 1])));
-                            uint64_t z23 = ptx::f32x2_pack(static_cast<float>(static_cast<int>(raw[j + 2])), static_cast<float>(static_cast<int>(raw[j + 3])));
-                            // fl(fl(float(acc) * fl(a_scale * w_scale)) + bias), every operation rounded to nearest.
-                            // The additions are scalar intrinsics: a packed multiply feeding a packed add was
-                            // observed to be contracted into one fused operation (single rounding).
-                            z01 = ptx::f32x2_mul(z01, ptx::f32x2_mul(as2, w2.x));
-                            z23 = ptx::f32x2_mul(z23, ptx::f32x2_mul(as2, w2.y));
-                            float y0, y1, y2, y3, c0, c1, c2, c3;
-                            ptx::f32x2_unpack(z01, y0, y1);
-                            ptx::f32x2_unpack(z23, y2, y3);
-                            ptx::f32x2_unpack(b2.x, c0, c1);
-                            ptx::f32x2_unpack(b2.y, c2, c3);
-                            out[j >> 1] = ptx::pack_bf16x2(__fadd_rn(y0, c0), __fadd_rn(y1, c1));
-                            out[(j >> 1) + 1] = ptx::pack_bf16x2(__fadd_rn(y2, c2), __fadd_rn(y3, c3));
-                        }
-                        // the previous TMA store has finished reading the staging buffer
-                        if (lane == 0) ptx::tma_store_wait_read<0>();
-                        __syncwarp();
-                        // row `lane` of the staging tile (64-byte rows, 64-byte swizzle): 16-byte chunk q XOR ((lane / 2) mod 4)
-#pragma unroll
-                        for (int q = 0; q < 4; ++q)
-                            *reinterpret_cast<uint4 *>(stg + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4)) =
-                                make_uint4(out[4 * q], out[4 * q + 1], out[4 * q + 2], out[4 * q + 3]);
-                        if (DUMP && acc_debug && row_ok) {
-                            uint4 *dbg = reinterpret_cast<uint4 *>(acc_debug + (long long)gm * N + n0 + col);
-#pragma unroll
-                            for (int q = 0; q < 8; ++q)
-                                dbg[q] = make_uint4(static_cast<int>(raw[4 * q]) >> 8, static_cast<int>(raw[4 * q + 1]) >> 8,
-                                                    static_cast<int>(raw[4 * q + 2]) >> 8, static_cast<int>(raw[4 * q + 3]) >> 8);
-                        }
-                        ptx::fence_proxy_async_smem();          // staging writes -> visible to the TMA engine
-                        __syncwarp();
-                        if (lane == 0 && m0 < M) {
-                            ptx::tma_store_2d(&map_y, stg_addr, n0 + col, m0);   // rows >= M are clipped by the tensor map
-                            ptx::tma_store_commit();
-                        }
+                        gemmc::scale_bias_bf16_x32(raw, as2, wsb + col, bsb + col, out);
+                        gemmc::stage_row_32(stg, out, lane);
+                        // the raw sums carry a factor 256 (codes in the high half-byte)
+                        if (DUMP && acc_debug && row_ok) gemmc::dump_acc_x32<8>(acc_debug + (long long)gm * N + n0 + col, raw);
+                        gemmc::store_staged_32x32(&map_y, stg_addr, n0 + col, m0, m0 < M, lane);
                     }
                 }
             }
@@ -232,63 +189,9 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         if (lane == 0) ptx::tma_store_wait_all();
     } else if (warp < MMA_WARP) {
         // ------------------------------------------------------------ converters
-        const int cw = warp - CONV_WARP0;
-        const int group = cw / C::GROUP_WARPS;
-        const int gt = (cw % C::GROUP_WARPS) * 32 + lane;                // thread within the group
-        const int row = gt >> 2, piece = gt & 3;                         // piece i of this thread: row + (GROUP_THREADS/4) i
-        constexpr int SRC_STEP = C::GROUP_THREADS * 16;                  // bytes between a thread's consecutive packed pieces
-        constexpr int DST_STEP = (C::GROUP_THREADS / 4) * 128;
-        const uint32_t src_off = gt * 16;
-        const uint32_t dst_off = row * 128 + (((2 * piece) ^ (row & 7)) << 4);   // even codes
-        const uint32_t dst_hi_off = dst_off ^ 16;                                // odd codes: the neighbouring 16-byte chunk
-        const uint32_t leader_ufull = (CG == 2) ? ptx::map_to_cta(bar_ufull, 0) : bar_ufull;
-        const int total_kb = my_tiles * KB;
-        bool alive = true;
-        uint32_t toggle = 0;
-        for (int it = group; it < total_kb && alive; it += C::GROUPS) {
-            const int ps = it % C::PS, us = it % C::US;
-            alive = ptx::mbar_wait_group(bar_pfull + 8 * ps, (it / C::PS) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_PACKED, gt == 0,
-                                         2 + group, C::GROUP_THREADS, s_flags + 2 + 2 * group, toggle, 20);
-            if (!alive) break;
-            // the whole share of the stage goes to registers first, so the packed stage is handed back
-            // to the TMA producer before the (longer) conversion starts
-            const unsigned char *src = smem + C::OFF_PK + ps * C::PK_STAGE + src_off;
-            uint4 pk[C::CHUNKS];
-#pragma unroll
-            for (int i = 0; i < C::CHUNKS; ++i) pk[i] = *reinterpret_cast<const uint4 *>(src + SRC_STEP * i);
-            // consume one value of every load: the loads have completed before the stage is released
-            uint32_t seen = 0;
-#pragma unroll
-            for (int i = 0; i < C::CHUNKS; ++i) seen |= pk[i].x;
-            // a real (if never taken) use of every loaded value: the loads must have returned before
-            // this branch resolves, hence before the arrival below lets the TMA overwrite the stage
-            if (seen == 0x9E3779B9u) s_flags[1 + 2 * CONV_WARPS] = 1;
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(bar_pempty + 8 * ps);
-            if (it >= C::US) {
-                alive = ptx::mbar_wait_group(bar_uempty + 8 * us, ((it / C::US) - 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_EMPTY,
-                                             gt == 0, 2 + group, C::GROUP_THREADS, s_flags + 2 + 2 * group, toggle, 20);
-                if (!alive) break;
-            }
-            unsigned char *dst = smem + C::OFF_UP + us * C::UP_STAGE;
-#pragma unroll
-            for (int i = 0; i < C::CHUNKS; ++i) {
-                const uint4 w = pk[i];
-                uint4 lo, hi;
-                lo.x = (w.x << 4) & 0xF0F0F0F0u; hi.x = w.x & 0xF0F0F0F0u;
-                lo.y = (w.y << 4) & 0xF0F0F0F0u; hi.y = w.y & 0xF0F0F0F0u;
-                lo.z = (w.z << 4) & 0xF0F0F0F0u; hi.z = w.z & 0xF0F0F0F0u;
-                lo.w = (w.w << 4) & 0xF0F0F0F0u; hi.w = w.w & 0xF0F0F0F0u;
-                *reinterpret_cast<uint4 *>(dst + dst_off + DST_STEP * i) = lo;
-                *reinterpret_cast<uint4 *>(dst + dst_hi_off + DST_STEP * i) = hi;
-            }
-            ptx::fence_proxy_async_smem();      // my generic-proxy writes -> visible to the tensor core's async proxy
-            __syncwarp();                        // orders the whole warp's reads and writes before the two arrivals
-            if (lane == 0) {
-                if (CG == 2) ptx::mbar_arrive_cluster(leader_ufull + 8 * us);
-                else ptx::mbar_arrive(bar_ufull + 8 * us);
-            }
-        }
+        gemmc::convert_packed_stages<C, true>(smem, warp - CONV_WARP0, lane, my_tiles * KB, bar_pfull, bar_pempty, bar_uempty,
+                                              ptx::map_to_cta(bar_ufull, 0), s_abort, status, s_flags + 2,
+                                              s_flags + 1 + 2 * CONV_WARPS, QVGGT_DEV_TIMEOUT_PACKED, QVGGT_DEV_TIMEOUT_EMPTY);
     } else if (warp == MMA_WARP) {
         // ------------------------------------------------------------ MMA issuer (one thread of the leader CTA)
         if (lane == 0 && rank == 0) {
@@ -309,22 +212,11 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     if (!alive) break;
                     ptx::tc_fence_after_sync();
                     const uint32_t a_addr = sbase + C::OFF_UP + us * C::UP_STAGE;
-                    const uint64_t a_desc = ptx::smem_desc_k_sw128(a_addr);
-                    const uint64_t b_desc = ptx::smem_desc_k_sw128(a_addr + BM * BK);
-#pragma unroll
-                    for (int p = 0; p < BK / 32; ++p) {
-                        // advance 32 bytes (one K = 32 slice) inside the swizzled row: +2 in 16-byte units
-                        if (CG == 2) ptx::mma_i8_ss_pair(d_tmem, a_desc + 2 * p, b_desc + 2 * p, idesc, (kb | p) != 0);
-                        else ptx::mma_i8_ss(d_tmem, a_desc + 2 * p, b_desc + 2 * p, idesc, (kb | p) != 0);
-                    }
-                    if (CG == 2) ptx::mma_commit_pair(bar_uempty + 8 * us, 3);
-                    else ptx::mma_commit(bar_uempty + 8 * us);
+                    gemmc::mma_kblock_i8<true>(d_tmem, a_addr, a_addr + BM * BK, idesc, kb == 0);
+                    ptx::mma_commit_pair(bar_uempty + 8 * us, 3);
                     if (++us == C::US) { us = 0; uph ^= 1; }
                 }
-                if (alive) {
-                    if (CG == 2) ptx::mma_commit_pair(bar_tfull + 8 * b, 3);
-                    else ptx::mma_commit(bar_tfull + 8 * b);
-                }
+                if (alive) ptx::mma_commit_pair(bar_tfull + 8 * b, 3);
             }
         }
         __syncwarp();
@@ -357,43 +249,21 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
 
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (CG == 2) ptx::cluster_sync();        // no remote arrival or multicast commit may target a CTA that has exited
+    ptx::cluster_sync();                     // no remote arrival or multicast commit may target a CTA that has exited
     if (warp == MMA_WARP) {
         ptx::tc_fence_after_sync();
-        if (CG == 2) ptx::tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
-        else ptx::tmem_dealloc(tmem_base, C::TMEM_COLS);
+        ptx::tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
     }
 }
 
-template <int CG, bool DUMP>
+template <bool DUMP>
 cudaError_t launch(const qvggt_weights *w, const unsigned char *Xq, const float *a_scale, int M, void *Y, long long ldy,
                    int *acc_debug, cudaStream_t st)
 {
-    using C = Cfg<CG>;
-    static int max_workers = 0;       // per process; one GPU type per process
-    cudaError_t e;
-    if (!max_workers) {
-        e = cudaFuncSetAttribute(gemm_w4a4_kernel<CG, DUMP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::DYN_SMEM);
-        if (e != cudaSuccess) return e;
-        if (CG == 1) {
-            max_workers = qvggt_sm_count();
-        } else {
-            cudaLaunchConfig_t probe = {};
-            probe.gridDim = dim3(2 * qvggt_sm_count());
-            probe.blockDim = dim3(THREADS);
-            probe.dynamicSmemBytes = C::DYN_SMEM;
-            cudaLaunchAttribute a;
-            a.id = cudaLaunchAttributeClusterDimension;
-            a.val.clusterDim.x = CG; a.val.clusterDim.y = 1; a.val.clusterDim.z = 1;
-            probe.attrs = &a;
-            probe.numAttrs = 1;
-            int clusters = 0;
-            e = cudaOccupancyMaxActiveClusters(&clusters, gemm_w4a4_kernel<CG, DUMP>, &probe);
-            if (e != cudaSuccess) return e;
-            if (clusters < 1) return cudaErrorLaunchOutOfResources;
-            max_workers = clusters;
-        }
-    }
+    static QvggtPerDevice cache;
+    int max_workers = 0;
+    cudaError_t e = qvggt_configure_kernel(gemm_w4a4_kernel<DUMP>, THREADS, C::DYN_SMEM, CG, cache, &max_workers);
+    if (e != cudaSuccess) return e;
     const int K = w->K, N = w->N;
     CUtensorMap map_x, map_w, map_y;
     if (!qvggt_make_map(&map_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, Xq, K / 2, M, K / 2, BK / 2, BM, CU_TENSOR_MAP_SWIZZLE_NONE) ||
@@ -412,7 +282,7 @@ cudaError_t launch(const qvggt_weights *w, const unsigned char *Xq, const float 
     attr.val.clusterDim.x = CG; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_w4a4_kernel<CG, DUMP>, map_x, map_w, map_y, a_scale, (const float *)w->w_scale,
+    return cudaLaunchKernelEx(&cfg, gemm_w4a4_kernel<DUMP>, map_x, map_w, map_y, a_scale, (const float *)w->w_scale,
                               (const uint16_t *)w->bias, acc_debug, M, N, K, w->status);
 }
 
@@ -424,6 +294,5 @@ cudaError_t qvggt_launch_gemm(const qvggt_weights *w, const unsigned char *Xq, c
     if (M == 0) return cudaSuccess;
     if (group == 128) return qvggt_launch_gemm_grouped(w, Xq, a_scale, M, Y, ldy, acc_debug, st);
     if (group != 0) return cudaErrorNotSupported;
-    // the single-CTA configuration (CG = 1) measured 10-35 % slower on every VGGT shape: the pair halves the weight traffic
-    return acc_debug ? launch<2, true>(w, Xq, a_scale, M, Y, ldy, acc_debug, st) : launch<2, false>(w, Xq, a_scale, M, Y, ldy, acc_debug, st);
+    return acc_debug ? launch<true>(w, Xq, a_scale, M, Y, ldy, acc_debug, st) : launch<false>(w, Xq, a_scale, M, Y, ldy, acc_debug, st);
 }

@@ -13,11 +13,14 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include "gemm_common.cuh"
 #include "qvggt_internal.cuh"
 #include "sm100_ptx.cuh"
 #include "tensor_map.cuh"
 
 namespace {
+
+using gemmc::STG_BYTES;
 
 constexpr int BM = 128, BN = 128, BK = 128;
 constexpr int EPI_WARPS = 8;       // warp w: TMEM lanes 32*(w%4).., columns 64*(w/4)..
@@ -27,28 +30,33 @@ constexpr int MMA_WARP = EPI_WARPS + CONV_WARPS;
 constexpr int TMA_WARP = MMA_WARP + 1;
 constexpr int THREADS = (TMA_WARP + 1) * 32;
 constexpr int ACC_BUFS = 2;
-constexpr int STG_BYTES = 32 * 64;             // per epilogue warp: 32 rows x 32 bf16, 64-byte swizzled
-constexpr int ROWS = BM + BN;                  // packed / operand rows per stage: tokens, then channels
-constexpr int PK_STAGE = ROWS * (BK / 2);
-constexpr int UP_STAGE = ROWS * BK;
-constexpr int PS = 4, US = 4;
-constexpr int GROUPS = 4;                      // converter groups, as in the token-wise kernel
-constexpr int GROUP_WARPS = CONV_WARPS / GROUPS;
-constexpr int GROUP_THREADS = GROUP_WARPS * 32;
-constexpr int CHUNKS = ROWS * 4 / GROUP_THREADS;
-constexpr int OFF_UP = 0;
-constexpr int OFF_STG = OFF_UP + US * UP_STAGE;
-constexpr int OFF_CH = OFF_STG + EPI_WARPS * STG_BYTES;      // [2][BN] channel scales, [2][BN] bias, fp32
-constexpr int OFF_PK = OFF_CH + 2 * 2 * BN * 4;
-constexpr int OFF_BAR = OFF_PK + PS * PK_STAGE;              // pfull[PS] pempty[PS] ufull[US] uempty[US] tfull[2] tempty[2]
-constexpr int NBARS = 2 * PS + 2 * US + 2 * ACC_BUFS;
-constexpr int OFF_TMEM = OFF_BAR + NBARS * 8;
-constexpr int OFF_ABORT = OFF_TMEM + 4;
-constexpr int OFF_FLAGS = OFF_ABORT + 4;
-constexpr int SMEM_BYTES = OFF_FLAGS + 8 * (2 + CONV_WARPS);
-constexpr int DYN_SMEM = SMEM_BYTES + 1024;
-constexpr int TMEM_COLS = ACC_BUFS * BN;                     // 256
-static_assert(DYN_SMEM <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
+
+struct C {
+    static constexpr int ROWS = BM + BN;                  // packed / operand rows per stage: tokens, then channels
+    static constexpr int PK_STAGE = ROWS * (BK / 2);
+    static constexpr int UP_STAGE = ROWS * BK;
+    static constexpr int PS = 4, US = 4;
+    static constexpr int GROUPS = 4;                      // converter groups, as in the token-wise kernel
+    static constexpr int GROUP_WARPS = CONV_WARPS / GROUPS;
+    static constexpr int GROUP_THREADS = GROUP_WARPS * 32;
+    static constexpr int CHUNKS = ROWS * 4 / GROUP_THREADS;
+    static constexpr int OFF_UP = 0;
+    static constexpr int OFF_STG = OFF_UP + US * UP_STAGE;
+    static constexpr int OFF_CH = OFF_STG + EPI_WARPS * STG_BYTES;      // [2][BN] channel scales, [2][BN] bias, fp32
+    static constexpr int OFF_PK = OFF_CH + 2 * 2 * BN * 4;
+    static constexpr int OFF_BAR = OFF_PK + PS * PK_STAGE;              // pfull[PS] pempty[PS] ufull[US] uempty[US] tfull[2] tempty[2]
+    static constexpr int NBARS = 2 * PS + 2 * US + 2 * ACC_BUFS;
+    static constexpr int OFF_TMEM = OFF_BAR + NBARS * 8;
+    static constexpr int OFF_ABORT = OFF_TMEM + 4;
+    static constexpr int OFF_FLAGS = OFF_ABORT + 4;
+    static constexpr int SMEM_BYTES = OFF_FLAGS + 8 * (2 + CONV_WARPS);
+    static constexpr int DYN_SMEM = SMEM_BYTES + 1024;
+    static constexpr int TMEM_COLS = ACC_BUFS * BN;                     // 256
+    static_assert(DYN_SMEM <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
+};
+constexpr int PS = C::PS, US = C::US, PK_STAGE = C::PK_STAGE, UP_STAGE = C::UP_STAGE;
+constexpr int OFF_UP = C::OFF_UP, OFF_STG = C::OFF_STG, OFF_CH = C::OFF_CH, OFF_PK = C::OFF_PK, OFF_BAR = C::OFF_BAR;
+constexpr int OFF_TMEM = C::OFF_TMEM, OFF_ABORT = C::OFF_ABORT, OFF_FLAGS = C::OFF_FLAGS, DYN_SMEM = C::DYN_SMEM, TMEM_COLS = C::TMEM_COLS;
 
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_w4a4_grouped_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
@@ -77,18 +85,12 @@ gemm_w4a4_grouped_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
     const int my_tiles = (total_tiles > worker) ? (total_tiles - 1 - worker) / workers + 1 : 0;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < PS; ++s) {
-            ptx::mbar_init(bar_pfull + 8 * s, 1);
-            ptx::mbar_init(bar_pempty + 8 * s, GROUP_WARPS);
-        }
-        for (int s = 0; s < US; ++s) {
-            ptx::mbar_init(bar_ufull + 8 * s, GROUP_WARPS);
-            ptx::mbar_init(bar_uempty + 8 * s, 1);
-        }
-        for (int b = 0; b < ACC_BUFS; ++b) {
-            ptx::mbar_init(bar_tfull + 8 * b, 1);
-            ptx::mbar_init(bar_tempty + 8 * b, EPI_WARPS);
-        }
+        gemmc::init_barriers(bar_pfull, PS, 1);                      // the producer's arrive.expect_tx
+        gemmc::init_barriers(bar_pempty, PS, C::GROUP_WARPS);
+        gemmc::init_barriers(bar_ufull, US, C::GROUP_WARPS);
+        gemmc::init_barriers(bar_uempty, US, 1);                     // tcgen05.commit
+        gemmc::init_barriers(bar_tfull, ACC_BUFS, 1);                // tcgen05.commit
+        gemmc::init_barriers(bar_tempty, ACC_BUFS, EPI_WARPS);
         *s_abort = 0;
         ptx::fence_mbar_init();
     }
@@ -126,9 +128,7 @@ gemm_w4a4_grouped_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
             const bool row_ok = gm < M;
             if (threadIdx.x < BN) {
                 // buffer tb was last read two tiles ago; every epilogue warp has passed a group barrier since
-                const int e = threadIdx.x;
-                s_ws[tb * BN + e] = __ldg(w_scale + nt0 + e);
-                s_bs[tb * BN + e] = bias ? __uint_as_float(static_cast<uint32_t>(__ldg(bias + nt0 + e)) << 16) : 0.0f;
+                gemmc::load_channel_params(s_ws + tb * BN, s_bs + tb * BN, w_scale, bias, nt0, N, threadIdx.x);
             }
             float sum[64];
 #pragma unroll
@@ -156,13 +156,7 @@ gemm_w4a4_grouped_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
                             sum[32 * c + j] = __fadd_rn(sum[32 * c + j], __fmul_rn(static_cast<float>(static_cast<int>(raw[j])), as));
-                        if (acc_debug && row_ok) {
-                            uint4 *dbg = reinterpret_cast<uint4 *>(acc_debug + ((long long)kb * M + gm) * N + n0 + c * 32);
-#pragma unroll
-                            for (int q = 0; q < 8; ++q)
-                                dbg[q] = make_uint4(static_cast<int>(raw[4 * q]) >> 8, static_cast<int>(raw[4 * q + 1]) >> 8,
-                                                    static_cast<int>(raw[4 * q + 2]) >> 8, static_cast<int>(raw[4 * q + 3]) >> 8);
-                        }
+                        if (acc_debug && row_ok) gemmc::dump_acc_x32<8>(acc_debug + ((long long)kb * M + gm) * N + n0 + c * 32, raw);
                     }
                 }
             }
@@ -178,74 +172,17 @@ gemm_w4a4_grouped_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                         const float z1 = __fadd_rn(__fmul_rn(sum[32 * c + j + 1], wsb[32 * c + j + 1]), bsb[32 * c + j + 1]);
                         out[j >> 1] = ptx::pack_bf16x2(z0, z1);
                     }
-                    if (lane == 0) ptx::tma_store_wait_read<0>();      // the previous store has read the staging tile
-                    __syncwarp();
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        *reinterpret_cast<uint4 *>(stg + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4)) =
-                            make_uint4(out[4 * q], out[4 * q + 1], out[4 * q + 2], out[4 * q + 3]);
-                    ptx::fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0 && m0 < M) {
-                        ptx::tma_store_2d(&map_y, stg_addr, n0 + c * 32, m0);     // rows >= M are clipped by the tensor map
-                        ptx::tma_store_commit();
-                    }
+                    gemmc::stage_row_32(stg, out, lane);
+                    gemmc::store_staged_32x32(&map_y, stg_addr, n0 + c * 32, m0, m0 < M, lane);
                 }
             }
         }
         if (lane == 0) ptx::tma_store_wait_all();
     } else if (warp < MMA_WARP) {
         // ------------------------------------------------------------ converters (see the token-wise kernel)
-        const int cw = warp - CONV_WARP0;
-        const int group = cw / GROUP_WARPS;
-        const int gt = (cw % GROUP_WARPS) * 32 + lane;
-        const int row = gt >> 2, piece = gt & 3;
-        constexpr int SRC_STEP = GROUP_THREADS * 16;
-        constexpr int DST_STEP = (GROUP_THREADS / 4) * 128;
-        const uint32_t src_off = gt * 16;
-        const uint32_t dst_off = row * 128 + (((2 * piece) ^ (row & 7)) << 4);   // even codes
-        const uint32_t dst_hi_off = dst_off ^ 16;                                // odd codes
-        const int total_kb = my_tiles * KB;
-        bool alive = true;
-        uint32_t toggle = 0;
-        for (int it = group; it < total_kb && alive; it += GROUPS) {
-            const int ps = it % PS, us = it % US;
-            alive = ptx::mbar_wait_group(bar_pfull + 8 * ps, (it / PS) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_PACKED, gt == 0,
-                                         2 + group, GROUP_THREADS, s_flags + 2 + 2 * group, toggle, 20);
-            if (!alive) break;
-            const unsigned char *src = smem + OFF_PK + ps * PK_STAGE + src_off;
-            uint4 pk[CHUNKS];
-#pragma unroll
-            for (int i = 0; i < CHUNKS; ++i) pk[i] = *reinterpret_cast<const uint4 *>(src + SRC_STEP * i);
-            uint32_t seen = 0;
-#pragma unroll
-            for (int i = 0; i < CHUNKS; ++i) seen |= pk[i].x;
-            // a real (if never taken) use of every loaded value: the loads must have returned before
-            // this branch resolves, hence before the arrival below lets the TMA overwrite the stage
-            if (seen == 0x9E3779B9u) s_flags[1 + 2 * CONV_WARPS] = 1;
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(bar_pempty + 8 * ps);
-            if (it >= US) {
-                alive = ptx::mbar_wait_group(bar_uempty + 8 * us, ((it / US) - 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_EMPTY,
-                                             gt == 0, 2 + group, GROUP_THREADS, s_flags + 2 + 2 * group, toggle, 20);
-                if (!alive) break;
-            }
-            unsigned char *dst = smem + OFF_UP + us * UP_STAGE;
-#pragma unroll
-            for (int i = 0; i < CHUNKS; ++i) {
-                const uint4 w = pk[i];
-                uint4 lo, hi;
-                lo.x = (w.x << 4) & 0xF0F0F0F0u; hi.x = w.x & 0xF0F0F0F0u;
-                lo.y = (w.y << 4) & 0xF0F0F0F0u; hi.y = w.y & 0xF0F0F0F0u;
-                lo.z = (w.z << 4) & 0xF0F0F0F0u; hi.z = w.z & 0xF0F0F0F0u;
-                lo.w = (w.w << 4) & 0xF0F0F0F0u; hi.w = w.w & 0xF0F0F0F0u;
-                *reinterpret_cast<uint4 *>(dst + dst_off + DST_STEP * i) = lo;
-                *reinterpret_cast<uint4 *>(dst + dst_hi_off + DST_STEP * i) = hi;
-            }
-            ptx::fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(bar_ufull + 8 * us);
-        }
+        gemmc::convert_packed_stages<C, false>(smem, warp - CONV_WARP0, lane, my_tiles * KB, bar_pfull, bar_pempty, bar_uempty,
+                                               bar_ufull, s_abort, status, s_flags + 2, s_flags + 1 + 2 * CONV_WARPS,
+                                               QVGGT_DEV_TIMEOUT_PACKED, QVGGT_DEV_TIMEOUT_EMPTY);
     } else if (warp == MMA_WARP) {
         // ------------------------------------------------------------ MMA issuer: one accumulator per K-block
         if (lane == 0) {
@@ -262,10 +199,7 @@ gemm_w4a4_grouped_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                 if (!alive) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t a_addr = sbase + OFF_UP + us * UP_STAGE;
-                const uint64_t a_desc = ptx::smem_desc_k_sw128(a_addr);
-                const uint64_t b_desc = ptx::smem_desc_k_sw128(a_addr + BM * BK);
-#pragma unroll
-                for (int p = 0; p < BK / 32; ++p) ptx::mma_i8_ss(tmem_base + b * BN, a_desc + 2 * p, b_desc + 2 * p, idesc, p != 0);
+                gemmc::mma_kblock_i8<false>(tmem_base + b * BN, a_addr, a_addr + BM * BK, idesc, true);
                 ptx::mma_commit(bar_uempty + 8 * us);
                 ptx::mma_commit(bar_tfull + 8 * b);
             }
@@ -308,12 +242,10 @@ gemm_w4a4_grouped_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
 cudaError_t qvggt_launch_gemm_grouped(const qvggt_weights *w, const unsigned char *Xq, const float *a_scale, int M, void *Y,
                                       long long ldy, int *acc_debug, cudaStream_t st)
 {
-    static bool configured = false;       // per process
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_w4a4_grouped_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DYN_SMEM);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static QvggtPerDevice cache;
+    int sms = 0;
+    cudaError_t e = qvggt_configure_kernel(gemm_w4a4_grouped_kernel, THREADS, DYN_SMEM, 1, cache, &sms);
+    if (e != cudaSuccess) return e;
     const int K = w->K, N = w->N;
     CUtensorMap map_x, map_w, map_y;
     if (!qvggt_make_map(&map_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, Xq, K / 2, M, K / 2, BK / 2, BM, CU_TENSOR_MAP_SWIZZLE_NONE) ||
@@ -321,7 +253,7 @@ cudaError_t qvggt_launch_gemm_grouped(const qvggt_weights *w, const unsigned cha
         !qvggt_make_map(&map_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Y, N, M, (uint64_t)ldy * 2, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B))
         return cudaErrorInvalidValue;
     const int total_tiles = ((M + BM - 1) / BM) * (N / BN);
-    const int grid = total_tiles < qvggt_sm_count() ? total_tiles : qvggt_sm_count();
+    const int grid = total_tiles < sms ? total_tiles : sms;
     gemm_w4a4_grouped_kernel<<<grid, THREADS, DYN_SMEM, st>>>(map_x, map_w, map_y, a_scale, w->w_scale, w->bias, acc_debug, M, N,
                                                               K, w->status);
     return cudaGetLastError();

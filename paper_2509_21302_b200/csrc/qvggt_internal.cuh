@@ -9,7 +9,7 @@ struct qvggt_weights {
     int N, K;
     int device;
     int bits;            // 4 (W4A4) or 8 (W8A8: codes one per byte only)
-    unsigned char *Wq;   // [N, K/2] packed int4 (nullptr when bits == 8)
+    unsigned char *Wq;   // [N, K/2] packed int4 (nullptr when bits == 8 or prepared with QVGGT_PREP_C8_ONLY)
     signed char *Wq8;    // [N, K] one code per byte, or nullptr (prepared without QVGGT_PREP_C8)
     float *w_scale;      // [N]
     float *amul;         // [K]
@@ -55,3 +55,7 @@ cudaError_t qvggt_launch_gemm_grouped(const qvggt_weights *w, const unsigned cha
 // gemm_c8.cu (codes in 8-bit containers: TMA feeds the tensor core directly)
 cudaError_t qvggt_launch_gemm_c8(const qvggt_weights *w, const signed char *Xq8, const float *a_scale, int M, void *Y,
                                  long long ldy, int *acc_debug, cudaStream_t st);
+// The same launch with the TMA producers switched off and a short wait limit: the first wait for operands runs
+// out and the kernel leaves through its timeout path (exercised by the tests; nothing asynchronous is in flight).
+cudaError_t qvggt_launch_gemm_c8_starved(const qvggt_weights *w, const signed char *Xq8, const float *a_scale, int M, void *Y,
+                                         long long ldy, long long wait_limit_cycles, cudaStream_t st);

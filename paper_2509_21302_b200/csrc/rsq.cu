@@ -10,6 +10,7 @@
 // The same kernel serves the activations (multiplier amul) and the weight rows (multiplier wmul).
 #include "qvggt_internal.cuh"
 #include "sm100_ptx.cuh"
+#include "tensor_map.cuh"
 
 namespace {
 
@@ -158,6 +159,10 @@ struct SqGeom {
     static constexpr int SMEM = ROWS * ROW_SMEM;
 };
 
+// Resident CTAs per SM the kernel is built for: 4 (K = 1024) or 3 (K = 4096); with the fused LayerNorm at K = 4096 the
+// CTA's shared-memory copy of gamma and beta (32 KB) leaves room for 2.
+constexpr int sq_ctas_per_sm(int logt, int ln) { return logt == 5 ? 4 : (ln != 0 ? 2 : 3); }
+
 template <int T>
 __device__ __forceinline__ void group_sync(int slot)
 {
@@ -215,7 +220,7 @@ struct LnArgs {
 // T contiguous elements, then the xor-shuffle tree over the row's threads -- together the halves-recursion over the
 // row), its output rounded to bf16 as a separate normalization kernel would store it; 2 = only that, written out.
 template <int LOGT, int GROUP, bool C8 = false, int QMAX = 7, bool STATIC = false, int LN = 0>
-__global__ void __launch_bounds__(SqGeom<LOGT>::CTA_THREADS, LOGT == 5 ? 4 : 3)
+__global__ void __launch_bounds__(SqGeom<LOGT>::CTA_THREADS, sq_ctas_per_sm(LOGT, LN))
 rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float *__restrict__ mul,
               unsigned char *__restrict__ Xq, float *__restrict__ scales, const float *__restrict__ static_delta,
               const LnArgs ln)
@@ -265,9 +270,10 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
     }
     cp_async_commit();
     const float delta = STATIC ? __ldg(static_delta) : 0.0f;
-    // LayerNorm parameters (T = 32): one copy per CTA in shared memory behind the row slots, as 16-byte pieces ordered
-    // [piece][thread], so that thread t reads its T contiguous gammas with conflict-free 16-byte loads
-    constexpr bool LN_SMEM = (LN != 0) && (LOGT == 5);
+    // LayerNorm parameters: one copy per CTA in shared memory behind the row slots, as 16-byte pieces ordered
+    // [piece][thread], so that thread t reads its T contiguous gammas with conflict-free 16-byte loads (read straight
+    // from global memory, thread t's T contiguous values are 4 T bytes away from its neighbour's: 32 sectors per load)
+    constexpr bool LN_SMEM = (LN != 0);
     float4 *g_sm = reinterpret_cast<float4 *>(dsm + G::SMEM), *b_sm = g_sm + K / 4;
     if constexpr (LN_SMEM) {
         for (int i = threadIdx.x; i < K / 4; i += G::CTA_THREADS) {
@@ -279,7 +285,7 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
     }
     float m[T];                                                // multipliers of elements T k + t (loaded behind the first row's copies)
 #pragma unroll
-    for (int k = 0; k < T; ++k) m[k] = __ldg(mul + T * k + t);
+    for (int k = 0; k < T; ++k) m[k] = (LN == 2) ? 0.0f : __ldg(mul + T * k + t);   // the normalization alone uses none
     int buf = 0;
     for (; row < M; row += stride, buf ^= 1) {
         const long long next = row + stride;
@@ -342,11 +348,10 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
             const float var = __fmul_rn(row_sum(tree_sum<T>(sq), 10), inv_k);
             const float rstd = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(var, ln.eps)));
             const uint64_t rstd2 = ptx::f32x2_pack(rstd, rstd);
-            const float4 *g4 = reinterpret_cast<const float4 *>(ln.gamma + T * t), *b4 = reinterpret_cast<const float4 *>(ln.beta + T * t);
             uint32_t packed[T / 2];
 #pragma unroll
             for (int k = 0; k < T; k += 4) {
-                const float4 g = LN_SMEM ? g_sm[(k / 4) * T + t] : __ldg(g4 + k / 4), b = LN_SMEM ? b_sm[(k / 4) * T + t] : __ldg(b4 + k / 4);
+                const float4 g = g_sm[(k / 4) * T + t], b = b_sm[(k / 4) * T + t];
                 float n0, n1, n2, n3;
                 ptx::f32x2_unpack(ptx::f32x2_mul(ptx::f32x2_mul(d2[k / 2], rstd2), ptx::f32x2_pack(g.x, g.y)), n0, n1);
                 ptx::f32x2_unpack(ptx::f32x2_mul(ptx::f32x2_mul(d2[k / 2 + 1], rstd2), ptx::f32x2_pack(g.z, g.w)), n2, n3);
@@ -537,9 +542,8 @@ __global__ void smooth_finalize_kernel(const float *__restrict__ ax, const float
 
 int rsq_grid(int M, int rows_per_cta, int ctas_per_sm = 6)
 {
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    int sms = qvggt_sm_count();
+    if (sms < 1) sms = 148;
     long long need = ((long long)M + rows_per_cta - 1) / rows_per_cta;
     long long cap = (long long)sms * ctas_per_sm;
     return (int)(need < cap ? need : cap);
@@ -563,18 +567,20 @@ cudaError_t launch_sq(const uint16_t *x, long long ldx, int M, const float *mul,
                       cudaStream_t st, const float *static_delta = nullptr, LnArgs ln = LnArgs{nullptr, nullptr, 0.0f, nullptr})
 {
     using G = SqGeom<LOGT>;
-    constexpr int SMEM = G::SMEM + ((LN != 0 && LOGT == 5) ? 2 * G::K * 4 : 0);   // + the CTA's copy of gamma and beta
-    static bool configured = false;       // per process and instantiation
-    if (!configured) {
+    constexpr int SMEM = G::SMEM + (LN != 0 ? 2 * G::K * 4 : 0);   // + the CTA's copy of gamma and beta
+    static QvggtPerDevice configured;     // per device and instantiation
+    const int dev = qvggt_current_device();
+    if (dev < 0) return cudaErrorInvalidDevice;
+    if (!configured.v[dev].load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(rsq_sq_kernel<LOGT, GROUP, C8, QMAX, STATIC, LN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
         if (e != cudaSuccess) return e;
-        configured = true;
+        configured.v[dev].store(1, std::memory_order_release);
     }
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr.val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(rsq_grid(M, G::ROWS, LOGT == 5 ? 4 : 3));
+    cfg.gridDim = dim3(rsq_grid(M, G::ROWS, sq_ctas_per_sm(LOGT, LN)));
     cfg.blockDim = dim3(G::CTA_THREADS);
     cfg.dynamicSmemBytes = SMEM;
     cfg.stream = st;

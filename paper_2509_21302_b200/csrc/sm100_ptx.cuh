@@ -42,13 +42,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-// Bounded wait: gives up after ~2e9 cycles or as soon as another thread of the CTA has given up
+constexpr long long kWaitLimitCycles = 2000000000LL;   // default bound of every device-side wait (about one second)
+
+// Bounded wait: gives up after `limit` cycles or as soon as another thread of the CTA has given up
 // (*abort_flag != 0, a shared-memory word).  On expiry sets the flag, records `code` in *status
 // (global memory, first writer wins) and returns false.  The caller must then skip its work and
 // fall through to the common exit path so that tensor memory is still released.
 // `sleep_ns` > 0 backs off between polls (for waits that are expected to be long).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code,
-                                          unsigned sleep_ns = 0)
+                                          unsigned sleep_ns = 0, long long limit = kWaitLimitCycles)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
@@ -59,24 +61,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (sleep_ns) __nanosleep(sleep_ns);
         }
         if (*abort_flag) return false;
-        if (clock64() - t0 > 2000000000LL) {
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             atomicCAS(status, 0, code);
             return false;
         }
     }
-}
-
-// Same wait, polled by lane 0 only; the other lanes park at the shuffle instead of hammering the
-// barrier (every poll is a shared-memory operation that competes with the operand traffic).
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
-                                               int code, int lane, unsigned sleep_ns = 0)
-{
-    int ok = 1;
-    if (lane == 0) ok = mbar_wait(bar, parity, abort_flag, status, code, sleep_ns) ? 1 : 0;
-    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-    __syncwarp();   // memory ordering between lane 0's acquire and the other lanes' reads
-    return ok != 0;
 }
 
 // Same wait for a group of `nthreads` threads (whole warps) that share named barrier `bar_id`:
@@ -87,11 +77,11 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
 // make every call: the outcome is uniform, so they all leave their loop together.
 __device__ __forceinline__ bool mbar_wait_group(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code,
                                                 bool leader, int bar_id, int nthreads, volatile int *flags, uint32_t &toggle,
-                                                unsigned sleep_ns = 0)
+                                                unsigned sleep_ns = 0, long long limit = kWaitLimitCycles)
 {
     volatile int *flag = flags + (toggle & 1);
     ++toggle;
-    if (leader) *flag = mbar_wait(bar, parity, abort_flag, status, code, sleep_ns) ? 1 : 0;
+    if (leader) *flag = mbar_wait(bar, parity, abort_flag, status, code, sleep_ns, limit) ? 1 : 0;
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(nthreads) : "memory");
     const bool ok = *flag != 0;
     // One thread of every warp observes the completed phase itself (it cannot advance again before this
@@ -242,7 +232,8 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
 }
 
 // Bounded wait with cluster-scope acquire (the arrivals come from both CTAs of the pair).
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code,
+                                                  long long limit = kWaitLimitCycles)
 {
     if (mbar_try_wait_cluster(bar, parity)) return true;
     const long long t0 = clock64();
@@ -251,7 +242,7 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait_cluster(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > 2000000000LL) {
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             atomicCAS(status, 0, code);
             return false;
@@ -354,52 +345,7 @@ __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepco
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // ---------------------------------------------------------------- packed fp32 pairs (one issue slot for two IEEE operations)
-__device__ __forceinline__ float2 mul_f32x2(float2 a, float2 b)
-{
-    float2 d;
-    asm("{\n\t"
-        ".reg .b64 ra, rb, rd;\n\t"
-        "mov.b64 ra, {%2, %3};\n\t"
-        "mov.b64 rb, {%4, %5};\n\t"
-        "mul.rn.f32x2 rd, ra, rb;\n\t"
-        "mov.b64 {%0, %1}, rd;\n\t"
-        "}\n"
-        : "=f"(d.x), "=f"(d.y)
-        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
-    return d;
-}
-
-__device__ __forceinline__ float2 add_f32x2(float2 a, float2 b)
-{
-    float2 d;
-    asm("{\n\t"
-        ".reg .b64 ra, rb, rd;\n\t"
-        "mov.b64 ra, {%2, %3};\n\t"
-        "mov.b64 rb, {%4, %5};\n\t"
-        "add.rn.f32x2 rd, ra, rb;\n\t"
-        "mov.b64 {%0, %1}, rd;\n\t"
-        "}\n"
-        : "=f"(d.x), "=f"(d.y)
-        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
-    return d;
-}
-
-__device__ __forceinline__ float2 sub_f32x2(float2 a, float2 b)
-{
-    float2 d;
-    asm("{\n\t"
-        ".reg .b64 ra, rb, rd;\n\t"
-        "mov.b64 ra, {%2, %3};\n\t"
-        "mov.b64 rb, {%4, %5};\n\t"
-        "sub.rn.f32x2 rd, ra, rb;\n\t"
-        "mov.b64 {%0, %1}, rd;\n\t"
-        "}\n"
-        : "=f"(d.x), "=f"(d.y)
-        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
-    return d;
-}
-
-// The same operations on pairs kept in 64-bit registers (no packing moves around each operation).
+// Pairs are kept in 64-bit registers (no packing moves around each operation).
 __device__ __forceinline__ uint64_t f32x2_pack(float lo, float hi)
 {
     uint64_t r;
@@ -447,49 +393,6 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     uint32_t d;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
     return d;
-}
-
-// ---------------------------------------------------------------- A operand in tensor memory
-// 32 lanes x 32 consecutive 32-bit columns: thread i of the warp writes lane (base+i), columns c..c+31.
-__device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r)[32])
-{
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
-        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
-        "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]),
-        "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]),
-        "r"(r[31])
-        : "memory");
-}
-
-__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-// D (+)= A * B with A in tensor memory (lane = row, one 32-bit column = four consecutive K bytes) and B in
-// shared memory; CTA pair: each CTA supplies its own 128 rows of A (same column in both) and N/2 rows of B.
-__device__ __forceinline__ void mma_i8_ts_pair(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t"
-        ".reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::i8 [%0], [%1], %2, %3, p;\n\t"
-        "}\n" ::"r"(d_tmem),
-        "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-
-// 32 lanes x 16 consecutive 32-bit columns
-__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr)
-        : "memory");
 }
 
 }  // namespace ptx

@@ -55,6 +55,10 @@ extern "C" int qvggt_quantize_weights_static(const void *W_bf16, const float *sm
     if ((reinterpret_cast<uintptr_t>(W_bf16) & 15u) || (reinterpret_cast<uintptr_t>(Wq) & 15u) ||
         (reinterpret_cast<uintptr_t>(w_scale) & 3u) || (reinterpret_cast<uintptr_t>(amul) & 3u))
         return QVGGT_ERR_ALIGN;
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+        return QVGGT_ERR_CUDA;
+    if (major != 10) return QVGGT_ERR_UNSUPPORTED;               // the kernels exist for sm_100 only
     float *wmul = nullptr;
     if (scratch_for_current_device(&wmul) != cudaSuccess) return QVGGT_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

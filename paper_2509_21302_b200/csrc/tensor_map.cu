@@ -35,13 +35,22 @@ bool qvggt_make_map(CUtensorMap *map, CUtensorMapDataType type, const void *base
               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+int qvggt_current_device()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kQvggtMaxDevices) return -1;
+    return dev;
+}
+
 int qvggt_sm_count()
 {
-    static int sms = 0;
+    static QvggtPerDevice cache;
+    const int dev = qvggt_current_device();
+    if (dev < 0) return 0;
+    int sms = cache.v[dev].load(std::memory_order_relaxed);
     if (!sms) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        cache.v[dev].store(sms, std::memory_order_relaxed);
     }
     return sms;
 }

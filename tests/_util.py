@@ -34,16 +34,21 @@ def assert_bf16_within_one_ulp(got_bits: np.ndarray, want_bits: np.ndarray, what
 
     Returns the fraction of elements that are not bit-equal (expected 0: the kernel uses the same
     separate multiply, multiply, add as the oracle)."""
+    same = got_bits == want_bits
+    if same.all():
+        return 0.0
+    # only the elements that differ go through the tolerance (whole-output comparisons hold ~10^9 elements)
+    n = got_bits.size
+    got_bits, want_bits = got_bits[~same], want_bits[~same]
     g = bf16_value(got_bits).astype(np.float64)
     w = bf16_value(want_bits).astype(np.float64)
     assert np.all(np.isfinite(g)), f"{what}: non-finite output"
-    same = got_bits == want_bits
     rel_ok = np.abs(g - w) <= 2.0 ** -7 * np.abs(w)
     # adjacent representable values: the ordered-integer views differ by one
     def key(b):
         b = b.astype(np.int32)
         return np.where(b & 0x8000, -(b & 0x7FFF), b & 0x7FFF)
     adj = np.abs(key(got_bits) - key(want_bits)) <= 1
-    bad = ~(same | rel_ok | adj)
-    assert not bad.any(), f"{what}: {bad.sum()} elements beyond 1 bf16 ulp; first at {np.argwhere(bad)[0]}"
-    return float(1.0 - same.mean())
+    bad = ~(rel_ok | adj)
+    assert not bad.any(), f"{what}: {bad.sum()} elements beyond 1 bf16 ulp"
+    return float(got_bits.size) / n

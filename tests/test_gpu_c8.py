@@ -215,7 +215,34 @@ def test_c8_entry_points_validate_their_arguments():
     assert L.qvggt_layernorm_rotate_smooth_quantize_c8(hp, xp, K, M, gp + 4, gp, 1e-5, qp, ap, st) == ALIGN
     assert L.qvggt_layernorm(xp, K, M, 2048, gp, gp, 1e-5, yp, st) == SHAPE                   # K must be 1024 or 4096
     out = ctypes.c_void_p()
-    assert L.qvggt_prepare_weights(xp, None, gp, None, N, K, 8, st, ctypes.byref(out)) == UNSUP   # unknown flag
+    assert L.qvggt_prepare_weights(xp, None, gp, None, N, K, 16, st, ctypes.byref(out)) == UNSUP  # unknown flag
     assert out.value is None
     torch.cuda.synchronize()
     assert h.device_status() == 0
+
+
+def test_c8_only_handle_keeps_one_byte_per_weight():
+    """QVGGT_PREP_C8_ONLY: the handle holds the codes one per byte and no packed copy (1 byte per weight instead of 1.5);
+    the one-code-per-byte entry points work as before, the packed ones refuse the handle."""
+    K, N, M = 1024, 256, 140
+    spec = workload.LinearSpec("only", K, N, workload.DIST_NORMAL, 21, 0)
+    W, b, X = spec.weight(), spec.bias(), spec.x_rows(0, M)
+    c = oracle.smooth_factors(spec.x_calib(128), W)
+    torch.cuda.synchronize()
+    used0 = torch.cuda.memory_allocated()
+    free0 = torch.cuda.mem_get_info()[0]
+    h = q.prepare_weights(dev_bf16(W), dev_bf16(b), torch.from_numpy(c).cuda(), None, c8="only")
+    torch.cuda.synchronize()
+    v = h.view()
+    assert v["wq"] is None and v["w_scale"].shape == (N,)
+    ref = oracle.w4a4_linear(X, oracle.prepare_weights(W, c), b, 0)
+    assert np.array_equal(h.view_c8().cpu().numpy(), oracle.prepare_weights(W, c)["wq"])
+    Xq8, a_scale = q.rotate_smooth_quantize_c8(h, dev_bf16(X))
+    Y = q.w4a4_linear_c8(h, Xq8, a_scale)
+    assert np.array_equal(Xq8.cpu().numpy(), ref["xq"]) and np.array_equal(host_bits(Y), ref["y"])
+    Xq = torch.zeros((M, K // 2), dtype=torch.uint8, device="cuda")
+    st = q.lib().qvggt_w4a4_linear(h.handle, Xq.data_ptr(), a_scale.data_ptr(), M, 0, Y.data_ptr(), N, None,
+                                   torch.cuda.current_stream().cuda_stream)
+    assert st == -4                                               # QVGGT_ERR_UNSUPPORTED: no packed weights in this handle
+    assert h.device_status() == 0
+    h.free()
