@@ -46,6 +46,8 @@ def _L():
             "orc_rotate_smooth_quantize_bits": [vp, i64, i64, i32, vp, i32, i32, vp, vp],
             "orc_rotate_smooth_quantize_static": [vp, i64, i64, i32, vp, ctypes.c_float, i32, vp],
             "orc_layernorm": [vp, i64, i64, i32, vp, vp, ctypes.c_float, vp],
+            "orc_rotate_smooth_quantize_wide": [vp, i64, i64, i32, vp, i32, vp, vp, vp, vp],
+            "orc_gelu": [vp, i64, i64, i32, vp],
             "orc_pack_int4": [vp, i64, i32, vp],
             "orc_unpack_int4": [vp, i64, i32, vp],
             "orc_gemm_i32": [vp, vp, i64, i32, i32, i32, vp],
@@ -58,6 +60,8 @@ def _L():
             fn = getattr(lib, name)
             fn.argtypes = args
             fn.restype = None
+        lib.orc_gelu_f64.argtypes = [dbl]
+        lib.orc_gelu_f64.restype = dbl
         _lib = lib
     return _lib
 
@@ -121,6 +125,34 @@ def rotate_smooth_quantize(X: np.ndarray, mul: np.ndarray, group: int = 0, bits:
         _L().orc_rotate_smooth_quantize_bits(X.ctypes.data, X.strides[0] // 2, M, K, mul.ctypes.data, group, bits,
                                              codes.ctypes.data, scales.ctypes.data)
     return codes, (scales if group else scales.reshape(M))
+
+
+def rotate_smooth_quantize_wide(X: np.ndarray, mul: np.ndarray, bits: int = 4):
+    """The quantizer behind a rotation evaluated in fp64 and rounded to fp32 once (reference of the tolerance contract
+    for rotations that do not follow the fp32 butterfly order).
+    -> dict(codes int8 [M, K], scales fp32 [M], y fp32 [M, K] rotated and smoothed rows, abs_sum fp64 [M] = sum |x|)."""
+    assert X.dtype == np.uint16 and X.ndim == 2 and X.strides[1] == 2 and 2 <= bits <= 8
+    M, K = X.shape
+    mul = _c(mul, np.float32)
+    codes, scales = np.empty((M, K), np.int8), np.empty(M, np.float32)
+    y, abs_sum = np.empty((M, K), np.float32), np.empty(M, np.float64)
+    _L().orc_rotate_smooth_quantize_wide(X.ctypes.data, X.strides[0] // 2, M, K, mul.ctypes.data, bits, codes.ctypes.data,
+                                         scales.ctypes.data, y.ctypes.data, abs_sum.ctypes.data)
+    return dict(codes=codes, scales=scales, y=y, abs_sum=abs_sum)
+
+
+def gelu_f64(x: float) -> float:
+    """x * Phi(x) in fp64 (Phi through erfc)."""
+    return _L().orc_gelu_f64(float(x))
+
+
+def gelu(X: np.ndarray) -> np.ndarray:
+    """bf16 bits [M, K] -> bf16 bits [M, K]: gelu evaluated in fp64, rounded to bf16 once."""
+    assert X.dtype == np.uint16 and X.ndim == 2 and X.strides[1] == 2
+    M, K = X.shape
+    out = np.empty((M, K), np.uint16)
+    _L().orc_gelu(X.ctypes.data, X.strides[0] // 2, M, K, out.ctypes.data)
+    return out
 
 
 def layernorm(X: np.ndarray, gamma: np.ndarray, beta: np.ndarray, eps: float = 1e-5) -> np.ndarray:

@@ -13,8 +13,11 @@
  * brute-force dense +-1 products on integer inputs, fp64 rotation/smoothing invariance,
  * |y - scale*q| <= scale/2, hand-built rounding ties, brute-force integer GEMMs, fp64 epilogue.
  * Unpinned by the paper (this build's conventions): the fp32 butterfly stage order, the
- * group-wise (per 128 channels) variant for G < K, and the end-to-end layer error vs. the
- * unquantized layer ("parity unpinned": information only).
+ * group-wise (per 128 channels) variant for G < K, the summation tree of the LayerNorm statistics, and the
+ * end-to-end layer error vs. the unquantized layer ("parity unpinned": information only).
+ * Further pins: the wide-rotation quantizer (rotation in fp64) coincides with the fp32 one wherever fp32 is exact
+ * and stays inside the rounding bound elsewhere; GELU against tabulated values of the normal distribution, the
+ * identity gelu(x) - gelu(-x) = x and a library normal CDF.
  */
 #include <math.h>
 #include <stdint.h>
@@ -68,7 +71,6 @@ void orc_fwht_f64(double *u, int K)
             }
 }
 
-/* K^{-1/2}: an exact power of two when log2 K is even (K = 1024, 4096). */
 /*
  * LayerNorm in front of the rotation (Sec. 3.2 places the quantized linear behind a normalization layer; the
  * upstream-fusion row fuses the two).  The paper does not say how the statistics are summed, so this build fixes it:
@@ -118,6 +120,7 @@ void orc_layernorm(const uint16_t *X, int64_t ldx, int64_t M, int K, const float
     }
 }
 
+/* K^{-1/2}: an exact power of two when log2 K is even (K = 1024, 4096). */
 static float orc_norm(int K)
 {
     return (float)(1.0 / sqrt((double)K));
@@ -224,6 +227,98 @@ void orc_rotate_smooth_quantize_static(const uint16_t *X, int64_t ldx, int64_t M
         }
         free(u);
     }
+}
+
+/*
+ * The same quantizer behind a rotation WITHOUT intermediate rounding: u = x H_K evaluated in fp64 (for bf16 inputs
+ * every partial sum of the transform is exact in fp64 unless the row spans more than ~40 binades) and rounded to
+ * fp32 once; the multiplier, the absolute maximum and Eq. "quantization" follow unchanged.  This is the reference of
+ * the tolerance contract for rotations that do not reproduce the fp32 butterfly order (a tensor-core Hadamard):
+ * such a rotation cannot match orc_rotate_smooth_quantize_bits bit for bit, because that one rounds after each of
+ * its log2 K stages in one particular order; it is judged by its distance from the exact rotation instead.
+ *   y_out   fp32 [M, K] or NULL: the rotated, smoothed row fl(fl32(u) * mul) the codes were taken from
+ *   abs_sum fp64 [M] or NULL: sum_k |x_k|, the quantity the rounding bound of any fp32 rotation scales with
+ * Per-row scales only (group = 0).
+ */
+void orc_rotate_smooth_quantize_wide(const uint16_t *X, int64_t ldx, int64_t M, int K, const float *mul, int bits,
+                                     int8_t *codes, float *scales, float *y_out, double *abs_sum)
+{
+    const float qmax = (float)((1 << (bits - 1)) - 1);
+    const double lo = -(double)(1 << (bits - 1)), hi = (double)qmax;
+#pragma omp parallel
+    {
+        double *u = (double *)malloc(sizeof(double) * (size_t)K);
+        float *y = (float *)malloc(sizeof(float) * (size_t)K);
+#pragma omp for schedule(static)
+        for (int64_t m = 0; m < M; ++m) {
+            const uint16_t *x = X + m * ldx;
+            double s = 0.0;
+            for (int k = 0; k < K; ++k) {
+                u[k] = (double)orc_bf16_to_f32(x[k]);
+                s += fabs(u[k]);
+            }
+            if (abs_sum) abs_sum[m] = s;
+            orc_fwht_f64(u, K);
+            float amax = 0.0f;
+            for (int k = 0; k < K; ++k) {
+                float r = (float)u[k];          /* the one rounding of the rotation */
+                y[k] = r * mul[k];
+                float a = fabsf(y[k]);
+                if (a > amax) amax = a;
+            }
+            if (amax < 1e-8f) amax = 1e-8f;
+            scales[m] = amax / qmax;
+            float inv = qmax / amax;
+            for (int k = 0; k < K; ++k) {
+                double r = nearbyint((double)y[k] * (double)inv);
+                if (r < lo) r = lo;
+                if (r > hi) r = hi;
+                codes[m * K + k] = (int8_t)r;
+                if (y_out) y_out[m * K + k] = y[k];
+            }
+        }
+        free(u);
+        free(y);
+    }
+}
+
+/*
+ * GELU, the activation between the two linears of the transformer MLP (the producer of fc2's input; the paper
+ * does not name it, the ViT blocks VGGT is built from use the exact form):
+ *   gelu(x) = x * Phi(x),  Phi(x) = erfc(-x / sqrt(2)) / 2  the standard normal distribution function.
+ * Written with erfc so that the negative tail keeps its relative accuracy (1 + erf cancels there).
+ */
+double orc_gelu_f64(double x)
+{
+    return x * 0.5 * erfc(-x * 0.70710678118654752440);
+}
+
+/* fp64 -> bf16 bits, round to nearest, ties to even, straight from the fp64 value (no fp32 step in between). */
+static uint16_t orc_f64_to_bf16(double v)
+{
+    uint16_t c = orc_f32_to_bf16((float)v);
+    /* the fp32 step may have rounded across a bf16 midpoint: look at the neighbours and keep the nearest */
+    uint16_t best = c;
+    double bd = fabs((double)orc_bf16_to_f32(c) - v);
+    for (int d = -1; d <= 1; d += 2) {
+        uint16_t n = (uint16_t)(c + d);
+        if (((n ^ c) & 0x8000u) || (n & 0x7F80u) == 0x7F80u) continue;   /* stay on this side of zero, finite */
+        double nd = fabs((double)orc_bf16_to_f32(n) - v);
+        if (nd < bd || (nd == bd && !(n & 1u))) {
+            best = n;
+            bd = nd;
+        }
+    }
+    return best;
+}
+
+/* X bf16 bits [M, K] (row stride ldx) -> out bf16 bits [M, K] contiguous: bf16(gelu(x)) evaluated in fp64. */
+void orc_gelu(const uint16_t *X, int64_t ldx, int64_t M, int K, uint16_t *out)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m)
+        for (int k = 0; k < K; ++k)
+            out[m * K + k] = orc_f64_to_bf16(orc_gelu_f64((double)orc_bf16_to_f32(X[m * ldx + k])));
 }
 
 /* The W4A4 setting (N = 4: Delta = max|y| / 7, codes in [-8, 7]). */

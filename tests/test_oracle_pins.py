@@ -44,6 +44,12 @@ def load_table(name):
     return np.array(rows)
 
 
+def ordered_bf16(bits):
+    """bf16 bit patterns -> integers ordered like the values (adjacent values differ by one)."""
+    b = np.asarray(bits).astype(np.int32)
+    return np.where(b & 0x8000, -(b & 0x7FFF), b & 0x7FFF)
+
+
 # ------------------------------------------------------------------ Hadamard (Sec. 3.2, Pre-Global-Rotation)
 def test_h8_matches_handwritten_kronecker_recursion():
     H8 = load_table("sylvester_h8.txt")
@@ -488,3 +494,88 @@ def test_quantized_layer_approximates_the_fp_layer(group):
         deq = out["acc"].astype(np.float64) * out["a_scale"][:, None] * prep["w_scale"][None, :] \
             + oracle.bf16_to_f32(b)[None, :]
         assert np.all(bf16_neighbors_ok(out["y"], deq))
+
+
+# ------------------------------------------------------------------ wide rotation (reference of the tolerance contract)
+@pytest.mark.parametrize("K", [1024, 4096])
+def test_wide_rotation_quantizer_equals_fp32_one_where_fp32_is_exact(K):
+    """On small-integer inputs every butterfly of the fp32 transform is exact, so rounding order cannot matter: the
+    quantizer behind the fp64 rotation must return the codes and scales of the fp32 one, bit for bit (Sec. 3.2,
+    Pre-Global-Rotation: the Kronecker recursion defines ONE transform, whatever the evaluation order)."""
+    rng = np.random.default_rng(K)
+    x = rng.integers(-3, 4, size=(9, K)).astype(np.float32)
+    x[3] = 0
+    X = f32_to_bf16_bits(x)
+    mul = (rng.choice([-1.0, 1.0], K) * 2.0 ** rng.integers(-7, -3, K)).astype(np.float32)
+    for bits in (4, 8):
+        codes, scales = oracle.rotate_smooth_quantize(X, mul, 0, bits)
+        wide = oracle.rotate_smooth_quantize_wide(X, mul, bits)
+        assert np.array_equal(wide["codes"], codes) and np.array_equal(wide["scales"], scales)
+        assert np.array_equal(wide["abs_sum"], np.abs(x.astype(np.float64)).sum(axis=1))
+        # its rotated rows are the dense +-1 product (exact in integers) times the multiplier
+        dense = (x.astype(np.int64) @ sylvester(K) if K <= 1024 else oracle.fwht_f64(x.astype(np.float64))).astype(np.float64)
+        assert np.array_equal(wide["y"].astype(np.float64), dense * mul.astype(np.float64))
+
+
+@pytest.mark.parametrize("K", [1024, 4096])
+def test_wide_rotation_quantizer_on_heavy_tailed_rows(K):
+    """On real-valued rows the two quantizers may differ, but only as far as the fp32 transform's rounding allows:
+    rotated values within log2(K) 2^-24 sum|x| |mul| of each other, quantizer error bound |y - Delta q| <= Delta / 2
+    (Eq. "quantization") for the wide one as well, codes apart by at most one and only next to a rounding boundary."""
+    X = workload.sweep_activations(5, K, 0, 64)
+    mul = oracle.multipliers(workload.loguniform_f32(5, 1, K, 0.1, 10.0), workload.signs_i8(5, 2, K))[0]
+    wide = oracle.rotate_smooth_quantize_wide(X, mul)
+    codes, scales = oracle.rotate_smooth_quantize(X, mul, 0)
+    y64 = oracle.rotate_f64(X, mul.astype(np.float64))
+    tol = (np.log2(K) * 2.0 ** -24 * wide["abs_sum"])[:, None] * np.abs(mul)[None, :].astype(np.float64)
+    assert np.all(np.abs(wide["y"].astype(np.float64) - y64) <= 2.0 ** -23 * np.abs(y64) + 1e-300)   # two roundings in all
+    delta = wide["scales"].astype(np.float64)[:, None]
+    assert np.all(np.abs(wide["y"].astype(np.float64) - delta * wide["codes"]) <= delta / 2 * (1 + 2.0 ** -20))
+    assert np.all(np.abs(wide["codes"]).max(axis=1) == 7) and wide["codes"].min() >= -7
+    assert np.all(np.abs(wide["scales"] - scales) <= (tol.max(axis=1) / 7 + 2.0 ** -22 * scales))
+    diff = wide["codes"].astype(np.int32) - codes
+    assert np.abs(diff).max() <= 1
+    pos = y64 * (7.0 / np.abs(y64).max(axis=1))[:, None]                  # position on the code axis, fp64
+    to_boundary = np.abs(pos - (np.floor(pos) + 0.5))
+    slack = 7.0 / np.abs(y64).max(axis=1)[:, None] * 2 * tol + 2.0 ** -20
+    assert np.all(to_boundary[diff != 0] <= slack[diff != 0])
+    assert (diff != 0).mean() < 1e-3
+
+
+# ------------------------------------------------------------------ GELU (the producer of fc2's input)
+def test_gelu_matches_tabulated_normal_distribution():
+    tab = load_table("normal_cdf.txt")
+    for x, phi in tab:
+        want = x * phi
+        got = oracle.gelu_f64(x)
+        assert abs(got - want) <= 2e-14 * abs(want) + 1e-300, (x, got, want)     # the table carries 15 digits
+
+
+def test_gelu_identities_and_library_cdf():
+    from scipy.special import ndtr
+    x = np.concatenate([np.linspace(-12.0, 8.0, 4001), [0.0, -0.0, 1e-30, -1e-30, 37.0, -37.0]])
+    g = np.array([oracle.gelu_f64(v) for v in x])
+    assert np.allclose(g, x * ndtr(x), rtol=1e-13, atol=0.0)
+    gm = np.array([oracle.gelu_f64(-v) for v in x])
+    assert np.allclose(g - gm, x, rtol=1e-15, atol=1e-300)                       # Phi(x) + Phi(-x) = 1
+    assert np.all(g[x > 0] > 0) and np.all(g[x < 0] <= 0) and g[list(x).index(0.0)] == 0.0
+    grid = x[:4001]
+    assert np.all(np.diff(g[:4001][(grid > -0.75) & (grid < 8.0)]) > 0)          # increasing right of its minimum (x ~ -0.7518)
+    assert abs(min(g) - (-0.16997120747990369)) < 2e-5                           # the minimum of x Phi(x)
+
+
+def test_gelu_bf16_is_the_nearest_bf16_of_the_fp64_value():
+    rng = np.random.default_rng(3)
+    xb = f32_to_bf16_bits((rng.standard_normal((37, 128)) * 3).astype(np.float32).view(np.uint32).__and__(0xFFFF0000).view(np.float32))
+    out = oracle.gelu(xb)
+    x = oracle.bf16_to_f32(xb).astype(np.float64)
+    want = x * __import__("scipy.special", fromlist=["ndtr"]).ndtr(x)
+    got = oracle.bf16_to_f32(out).astype(np.float64)
+    ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(want), 1e-300))) - 7)
+    assert np.all(np.abs(got - want) <= ulp / 2 * (1 + 1e-9))                    # correctly rounded: within half a bf16 ulp
+    # rows with a stride, zeros keep their sign
+    z = np.array([[0x0000, 0x8000, 0x3F80, 0xBF80]], np.uint16)
+    assert [int(v) & 0x7FFF for v in oracle.gelu(z)[0][:2]] == [0, 0]
+    wide = np.zeros((4, 256), np.uint16)
+    wide[:, :128] = xb[:4]
+    assert np.array_equal(oracle.gelu(wide[:, :128]), out[:4])
