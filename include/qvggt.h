@@ -135,6 +135,29 @@ int qvggt_w4a4_linear_c8(const qvggt_weights_t *w, const signed char *Xq8, const
                          void *Y_bf16, long long ldy, int *acc_debug, void *cuda_stream);
 
 /*
+ * The activation path with the bulk of the rotation on the tensor core (Sec. 3.2, Pre-Global-Rotation: the Kronecker
+ * recursion H_{2^n} = H_2 (x) H_{2^(n-1)} lets the transform factor over any split of the index bits).  Index bits
+ * 3..9 are transformed by one product with the +-1 matrix H_128 (bf16 operands: every product exact, fp32
+ * accumulation inside the tensor core), the other 3 (K = 1024) or 5 (K = 4096) bits by fp32 butterflies, then
+ * multiplier, per-token absolute maximum and Eq. "quantization" as in qvggt_rotate_smooth_quantize[_c8].
+ * Same arguments, same layouts, per-token scales only, about 2.5 x fewer instructions per row than the exact kernel.
+ * NOT bit-exact against the exact entry points: an fp32 transform depends on the order of its additions, and the
+ * tensor core's is its own.  Contract, against the rotation evaluated without intermediate rounding
+ * (u* = x H_K exactly, y* = u* amul, S = sum_k |x_k| of the row, tau = 2 log2(K) 2^-24):
+ *   rotated values   |y[k] - y*[k]| <= (tau S + 2^-24 |u*[k]|) |amul[k]|
+ *   scale            within max_k of that bound, divided by qmax, of max|y*| / qmax
+ *   codes            the nearest integer to qmax y*[k] / max|y*|, except within that bound (in code units) of a
+ *                    half-integer, where the other neighbour may be returned (off by one, never more)
+ * (the exact entry points' own fp32 transform is only guaranteed log2(K) 2^-24 S).  The GEMM entry points take the
+ * codes of either mode.
+ *   y_debug  NULL, or fp32 [M, K] (16-byte aligned): receives the rotated, smoothed rows y
+ */
+int qvggt_rotate_smooth_quantize_tc(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M,
+                                    unsigned char *Xq, float *a_scale, float *y_debug, void *cuda_stream);
+int qvggt_rotate_smooth_quantize_tc_c8(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M,
+                                       signed char *Xq8, float *a_scale, float *y_debug, void *cuda_stream);
+
+/*
  * Static tensor-wise activation quantizer: the other arm of the paper's granularity ablation (Tab. "granularity",
  * dynamic token-wise against static tensor-wise).  One step size for the whole tensor, fixed offline, instead of
  * one per token from the token's absolute maximum:  Xq8 = clamp(round(y * fl(1 / delta)), -2^(N-1), 2^(N-1) - 1)

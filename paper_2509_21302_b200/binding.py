@@ -22,7 +22,8 @@ EXPORTS = ("qvggt_prepare_weights", "qvggt_rotate_smooth_quantize", "qvggt_w4a4_
            "qvggt_weights_view", "qvggt_device_status", "qvggt_calibrate_smooth", "qvggt_status_string",
            "qvggt_quantize_weights_static", "qvggt_rotate_smooth_quantize_c8", "qvggt_w4a4_linear_c8",
            "qvggt_weights_view_c8", "qvggt_rotate_smooth_quantize_static_c8",
-           "qvggt_layernorm_rotate_smooth_quantize_c8", "qvggt_layernorm", "qvggt_debug_starved_linear_c8")
+           "qvggt_layernorm_rotate_smooth_quantize_c8", "qvggt_layernorm", "qvggt_debug_starved_linear_c8",
+           "qvggt_rotate_smooth_quantize_tc", "qvggt_rotate_smooth_quantize_tc_c8")
 PREP_C8 = 1   # QVGGT_PREP_C8: keep an int8 [N, K] copy of the weight codes for the *_c8 entry points
 PREP_W8A8 = 2  # QVGGT_PREP_W8A8: 8-bit codes (one per byte only)
 PREP_C8_ONLY = 4  # QVGGT_PREP_C8_ONLY: 4-bit codes one per byte only (no packed copy)
@@ -56,6 +57,8 @@ def lib() -> ctypes.CDLL:
         L.qvggt_rotate_smooth_quantize_static_c8.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp]
         L.qvggt_layernorm_rotate_smooth_quantize_c8.argtypes = [vp, vp, i64, i32, vp, vp, f32, vp, vp, vp]
         L.qvggt_layernorm.argtypes = [vp, i64, i32, i32, vp, vp, f32, vp, vp]
+        L.qvggt_rotate_smooth_quantize_tc.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp]
+        L.qvggt_rotate_smooth_quantize_tc_c8.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp]
         L.qvggt_debug_starved_linear_c8.argtypes = [vp, vp, vp, i32, vp, i64, i64, vp]
         L.qvggt_weights_view_c8.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(i32)]
         L.qvggt_free_weights.argtypes = [vp]
@@ -230,6 +233,25 @@ def rotate_smooth_quantize_c8(w: Weights, X: torch.Tensor, Xq8: torch.Tensor | N
     _check(lib().qvggt_rotate_smooth_quantize_c8(w.handle, _ptr(X), ldx, M, _ptr(Xq8), _ptr(a_scale), _stream()),
            "qvggt_rotate_smooth_quantize_c8")
     return Xq8, a_scale
+
+
+def rotate_smooth_quantize_tc(w: Weights, X: torch.Tensor, c8: bool = False, Xq: torch.Tensor | None = None,
+                              a_scale: torch.Tensor | None = None, y_debug: torch.Tensor | None = None):
+    """Tensor-core Hadamard mode (tolerance contract, see include/qvggt.h): X [M,K] bf16 ->
+    (Xq [M,K/2] uint8, or [M,K] int8 with c8=True; a_scale fp32 [M]).  y_debug: optional fp32 [M,K] receiving the rotated rows."""
+    assert X.dim() == 2 and X.element_size() == 2 and X.stride(1) == 1 and X.shape[1] == w.K
+    M = X.shape[0]
+    if Xq is None:
+        Xq = torch.empty((M, w.K) if c8 else (M, w.K // 2), dtype=torch.int8 if c8 else torch.uint8, device=X.device)
+    if a_scale is None:
+        a_scale = torch.empty((M,), dtype=torch.float32, device=X.device)
+    assert Xq.is_contiguous() and a_scale.dtype == torch.float32
+    if y_debug is not None:
+        assert y_debug.dtype == torch.float32 and y_debug.is_contiguous() and y_debug.shape == (M, w.K)
+    ldx = X.stride(0) if M > 1 else w.K
+    fn = lib().qvggt_rotate_smooth_quantize_tc_c8 if c8 else lib().qvggt_rotate_smooth_quantize_tc
+    _check(fn(w.handle, _ptr(X), ldx, M, _ptr(Xq), _ptr(a_scale), _ptr(y_debug), _stream()), "qvggt_rotate_smooth_quantize_tc")
+    return Xq, a_scale
 
 
 def rotate_smooth_quantize_static_c8(w: Weights, X: torch.Tensor, delta: torch.Tensor, Xq8: torch.Tensor | None = None,

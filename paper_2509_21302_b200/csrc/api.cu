@@ -130,6 +130,37 @@ int qvggt_rotate_smooth_quantize_c8(const qvggt_weights_t *w, const void *X_bf16
     return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
 }
 
+int qvggt_rotate_smooth_quantize_tc(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M, unsigned char *Xq,
+                                    float *a_scale, float *y_debug, void *cuda_stream)
+{
+    if (!w) return QVGGT_ERR_NULL;
+    if (M < 0) return QVGGT_ERR_SHAPE;
+    if (w->bits != 4) return QVGGT_ERR_UNSUPPORTED;
+    if (M == 0) return QVGGT_OK;
+    if (!X_bf16 || !Xq || !a_scale) return QVGGT_ERR_NULL;
+    if (ldx < w->K) return QVGGT_ERR_SHAPE;
+    if (ldx % 8 != 0 || !aligned16(X_bf16) || !aligned16(Xq) || (reinterpret_cast<uintptr_t>(a_scale) & 3u) || (y_debug && !aligned16(y_debug)))
+        return QVGGT_ERR_ALIGN;
+    cudaError_t e = qvggt_launch_rsq_tc(X_bf16, ldx, M, w->K, w->amul, 4, false, Xq, a_scale, y_debug, w->status,
+                                        static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
+}
+
+int qvggt_rotate_smooth_quantize_tc_c8(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M, signed char *Xq8,
+                                       float *a_scale, float *y_debug, void *cuda_stream)
+{
+    if (!w) return QVGGT_ERR_NULL;
+    if (M < 0) return QVGGT_ERR_SHAPE;
+    if (M == 0) return QVGGT_OK;
+    if (!X_bf16 || !Xq8 || !a_scale) return QVGGT_ERR_NULL;
+    if (ldx < w->K) return QVGGT_ERR_SHAPE;
+    if (ldx % 8 != 0 || !aligned16(X_bf16) || !aligned16(Xq8) || (reinterpret_cast<uintptr_t>(a_scale) & 3u) || (y_debug && !aligned16(y_debug)))
+        return QVGGT_ERR_ALIGN;
+    cudaError_t e = qvggt_launch_rsq_tc(X_bf16, ldx, M, w->K, w->amul, w->bits, true, Xq8, a_scale, y_debug, w->status,
+                                        static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
+}
+
 int qvggt_rotate_smooth_quantize_static_c8(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M,
                                            const float *delta, signed char *Xq8, float *a_scale, void *cuda_stream)
 {

@@ -14,10 +14,9 @@
 //   warp  8      one thread issues tcgen05.mma and the commits that release stages / publish accumulators
 //   warp  9      one thread per CTA issues the TMA loads of its half of every operand stage; both CTAs signal
 //                the leader's "full" barrier (cta_group::2 form of the load)
-// Work items: the tiles are dealt round-robin to the workers.  When the last round would occupy at most half
-// of the workers, its tiles are cut into two halves of 128 channels each, so that the round takes about two
-// thirds of a whole tile's time instead of a whole one (a 256 x 128 tile moves 3/4 of the operand bytes for 1/2
-// of the products).
+// The tiles are dealt round-robin to the workers.  (Cutting the tiles of a short last round into halves of 128
+// channels was built and measured: an N = 128 MMA takes ~0.75 of an N = 256 one, a half tile ~0.9 of a whole
+// one, and the extra bookkeeping cost the main path 5 %: not kept.)
 // Every wait is bounded; on expiry the kernel records a code in *status and all roles fall through to the
 // common exit, where tensor memory is released.
 #include <cuda.h>
@@ -57,42 +56,13 @@ constexpr int TMEM_COLS = ACC_BUFS * BN;               // 512
 static_assert(DYN_SMEM <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 static_assert(2 * STAGE < (1 << 20), "transaction count of a stage must fit the barrier");
 
-// The work list every role of a worker walks in the same order.
-struct Schedule {
-    int n_tiles;       // whole tiles along N
-    int whole;         // tiles [0, whole) are processed whole, tiles [whole, total) as two halves
-    int items;         // whole + 2 * (total - whole)
-    __host__ __device__ Schedule(int M, int N, int workers)
-    {
-        n_tiles = (N + BN - 1) / BN;
-        const int total = ((M + 2 * BM - 1) / (2 * BM)) * n_tiles;
-        const int rem = total % workers;
-        const bool split = total > workers && rem > 0 && 2 * rem <= workers;
-        whole = split ? total - rem : total;
-        items = whole + 2 * (total - whole);
-    }
-    // item -> first token row of the pair's tile, first channel, channels covered
-    __device__ __forceinline__ void locate(int item, int &m0, int &n0, int &ncols) const
-    {
-        int tile = item, half = 0;
-        ncols = BN;
-        if (item >= whole) {
-            tile = whole + ((item - whole) >> 1);
-            half = (item - whole) & 1;
-            ncols = BN / 2;
-        }
-        m0 = (tile / n_tiles) * (2 * BM);
-        n0 = (tile % n_tiles) * BN + half * (BN / 2);
-    }
-};
-
 // DUMP: also write the int32 sums to acc_debug (its own instantiation keeps that code out of the production kernel).
 // wait_limit: bound of every device-side wait, in cycles.  skip_loads: the TMA producers issue nothing, so that the
 // first wait for operands runs out (used only to exercise the timeout path; no asynchronous operation is in flight).
 template <bool DUMP>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_c8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-               const __grid_constant__ CUtensorMap map_w_half, const __grid_constant__ CUtensorMap map_y,
+               const __grid_constant__ CUtensorMap map_y,
                const float *__restrict__ a_scale, const float *__restrict__ w_scale, const uint16_t *__restrict__ bias,
                int *__restrict__ acc_debug, int M, int N, int K, int *status, long long wait_limit, int skip_loads)
 {
@@ -111,8 +81,9 @@ gemm_c8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     const uint32_t rank = ptx::cluster_ctarank();                       // 0 = leader of the pair
     const int worker = blockIdx.x / 2, workers = gridDim.x / 2;
     const int KB = K / BK;
-    const Schedule sched(M, N, workers);
-    const int my_items = (sched.items > worker) ? (sched.items - 1 - worker) / workers + 1 : 0;
+    const int n_tiles = (N + BN - 1) / BN;
+    const int total_tiles = ((M + 2 * BM - 1) / (2 * BM)) * n_tiles;
+    const int my_tiles = (total_tiles > worker) ? (total_tiles - 1 - worker) / workers + 1 : 0;
 
     if (threadIdx.x == 0) {
         gemmc::init_barriers(bar_full, STAGES, 1);                     // the leader's arrive.expect_tx (bytes of both CTAs)
@@ -126,7 +97,6 @@ gemm_c8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     if (warp == TMA_WARP && lane == 0) {
         ptx::prefetch_tensormap(&map_x);
         ptx::prefetch_tensormap(&map_w);
-        ptx::prefetch_tensormap(&map_w_half);
         ptx::prefetch_tensormap(&map_y);
     }
     ptx::tc_fence_before_sync();
@@ -149,19 +119,19 @@ gemm_c8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         const uint32_t leader_tempty = ptx::map_to_cta(bar_tempty, 0);
         bool alive = true;
         uint32_t toggle = 0;
-        for (int t = 0; t < my_items; ++t) {
-            int tm0, nt0, ncols;
-            sched.locate(worker + t * workers, tm0, nt0, ncols);
-            const int m0 = tm0 + (int)rank * BM + quarter * 32;
-            const int cw = ncols >> 1;                         // columns of this warp's part: 128 or 64
-            const int n0 = nt0 + cpart * cw;                   // first channel of this warp's part
+        constexpr int CW = BN / 2, NCH = CW / 32;              // columns and 32-column chunks of one warp's part
+        for (int t = 0; t < my_tiles; ++t) {
+            const int tile = worker + t * workers;
+            const int m0 = (tile / n_tiles) * (2 * BM) + (int)rank * BM + quarter * 32;
+            const int nt0 = (tile % n_tiles) * BN;             // first channel of the tile
+            const int n0 = nt0 + cpart * CW;                   // first channel of this warp's part
             const int b = t & 1;
             const int gm = m0 + lane;
             const bool row_ok = gm < M;
             const bool cols_ok = n0 < N;                       // N is a multiple of 128: a part is all in or all out
             // per-channel scale and bias of the tile -> shared memory; buffer b was last read two tiles ago,
             // and every epilogue warp has passed the group barrier of the tile in between since then
-            if (threadIdx.x < ncols) gemmc::load_channel_params(s_ws + b * BN, s_bs + b * BN, w_scale, bias, nt0, N, threadIdx.x);
+            gemmc::load_channel_params(s_ws + b * BN, s_bs + b * BN, w_scale, bias, nt0, N, threadIdx.x);
             const float as = row_ok ? __ldg(a_scale + gm) : 0.0f;
             const uint64_t as2 = ptx::f32x2_pack(as, as);
             // one thread polls for all epilogue warps (named barrier 1); the barrier also publishes s_ws / s_bs
@@ -169,25 +139,23 @@ gemm_c8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                                          threadIdx.x == 0, 1, EPI_WARPS * 32, s_flags, toggle, 64, wait_limit) && alive;
             ptx::tc_fence_after_sync();
             if (alive) {
-                const float *wsb = s_ws + b * BN + cpart * cw;
-                const float *bsb = s_bs + b * BN + cpart * cw;
-                const int nch = cw >> 5;                               // 32-column chunks of this warp: 4 or 2
+                const float *wsb = s_ws + b * BN + cpart * CW;
+                const float *bsb = s_bs + b * BN + cpart * CW;
                 // the warp's whole share of the accumulator goes to registers first, so that tensor memory is
                 // handed back to the MMA thread a few hundred cycles after the tile completed, not after the
                 // conversions and stores of the first chunks
-                uint32_t raw[4][32];
+                uint32_t raw[NCH][32];
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    if (c < nch)
-                        ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + b * BN + cpart * cw + c * 32, raw[c]);
+                for (int c = 0; c < NCH; ++c)
+                    ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + b * BN + cpart * CW + c * 32, raw[c]);
                 ptx::tmem_ld_wait();
                 ptx::tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive_cluster(leader_tempty + 8 * b);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < NCH; ++c) {
                     const int col = c * 32;                               // within this warp's columns
-                    if (c < nch && cols_ok) {
+                    if (cols_ok) {
                         uint32_t out[16];
                         gemmc::scale_bias_bf16_x32(raw[c], as2, wsb + col, bsb + col, out);
                         gemmc::stage_row_32(stg, out, lane);
@@ -197,16 +165,16 @@ gemm_c8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 }
             }
         }
-        if (lane == 0) ptx::tma_store_wait_all();
+        // the staging tiles must outlive the stores' reads; the writes themselves are complete when the grid is
+        if (lane == 0) ptx::tma_store_wait_read<0>();
     } else if (warp == MMA_WARP) {
         // ------------------------------------------------------------ MMA issuer (one thread of the leader CTA)
         if (lane == 0 && rank == 0) {
-            constexpr uint32_t idesc_whole = ptx::idesc_i8(2 * BM, BN), idesc_half = ptx::idesc_i8(2 * BM, BN / 2);
+            constexpr uint32_t idesc = ptx::idesc_i8(2 * BM, BN);
             bool alive = true;
             Ring r;
-            for (int t = 0; t < my_items && alive; ++t) {
+            for (int t = 0; t < my_tiles && alive; ++t) {
                 const int b = t & 1;
-                const uint32_t idesc = (worker + t * workers >= sched.whole) ? idesc_half : idesc_whole;
                 if (t >= ACC_BUFS) {
                     alive = ptx::mbar_wait_cluster(bar_tempty + 8 * b, ((t >> 1) - 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_TMEM_FREE, wait_limit);
                     if (!alive) break;
@@ -233,13 +201,10 @@ gemm_c8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             bool alive = true;
             Ring r;
             int it = 0;
-            for (int t = 0; t < my_items && alive; ++t) {
-                int tm0, nt0, ncols;
-                sched.locate(worker + t * workers, tm0, nt0, ncols);
-                const int m0 = tm0 + (int)rank * BM;
-                const int b_rows = ncols >> 1;                          // weight rows this CTA stages: 128 or 64
-                const int n0 = nt0 + (int)rank * b_rows;
-                const CUtensorMap *mw = (ncols == BN) ? &map_w : &map_w_half;
+            for (int t = 0; t < my_tiles && alive; ++t) {
+                const int tile = worker + t * workers;
+                const int m0 = (tile / n_tiles) * (2 * BM) + (int)rank * BM;
+                const int n0 = (tile % n_tiles) * BN + (int)rank * B_ROWS;
                 for (int kb = 0; kb < KB; ++kb, ++it) {
                     if (it >= STAGES) {
                         alive = ptx::mbar_wait(bar_empty + 8 * r.s, r.ph ^ 1, s_abort, status, QVGGT_DEV_TIMEOUT_EMPTY, 20, wait_limit);
@@ -248,9 +213,9 @@ gemm_c8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     const uint32_t dst = sbase + r.s * STAGE;
                     // the leader's barrier expects the bytes of both CTAs; the peer's completions may arrive first
                     // (the count goes negative for a while), the phase cannot end before the leader has arrived
-                    if (rank == 0) ptx::mbar_arrive_expect_tx(bar_full + 8 * r.s, 2 * (BM + b_rows) * BK);
+                    if (rank == 0) ptx::mbar_arrive_expect_tx(bar_full + 8 * r.s, 2 * STAGE);
                     ptx::tma_load_2d_pair(&map_x, leader_full + 8 * r.s, dst, kb * BK, m0);
-                    ptx::tma_load_2d_pair(mw, leader_full + 8 * r.s, dst + BM * BK, kb * BK, n0);
+                    ptx::tma_load_2d_pair(&map_w, leader_full + 8 * r.s, dst + BM * BK, kb * BK, n0);
                     r.advance(STAGES);
                 }
             }
@@ -276,10 +241,9 @@ cudaError_t launch(const qvggt_weights *w, const signed char *Xq8, const float *
     cudaError_t e = qvggt_configure_kernel(gemm_c8_kernel<DUMP>, THREADS, DYN_SMEM, 2, cache, &max_workers);
     if (e != cudaSuccess) return e;
     const int K = w->K, N = w->N;
-    CUtensorMap map_x, map_w, map_w_half, map_y;
+    CUtensorMap map_x, map_w, map_y;
     if (!qvggt_make_map(&map_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, Xq8, K, M, K, BK, BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
         !qvggt_make_map(&map_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, w->Wq8, K, N, K, BK, B_ROWS, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !qvggt_make_map(&map_w_half, CU_TENSOR_MAP_DATA_TYPE_UINT8, w->Wq8, K, N, K, BK, B_ROWS / 2, CU_TENSOR_MAP_SWIZZLE_128B) ||
         !qvggt_make_map(&map_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Y, N, M, (uint64_t)ldy * 2, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B))
         return cudaErrorInvalidValue;
     const int total_tiles = ((M + 2 * BM - 1) / (2 * BM)) * ((N + BN - 1) / BN);
@@ -296,7 +260,7 @@ cudaError_t launch(const qvggt_weights *w, const signed char *Xq8, const float *
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, gemm_c8_kernel<DUMP>, map_x, map_w, map_w_half, map_y, a_scale, (const float *)w->w_scale,
+    return cudaLaunchKernelEx(&cfg, gemm_c8_kernel<DUMP>, map_x, map_w, map_y, a_scale, (const float *)w->w_scale,
                               (const uint16_t *)w->bias, acc_debug, M, N, K, w->status, wait_limit, skip_loads);
 }
 

@@ -43,6 +43,10 @@ cudaError_t qvggt_launch_colmax(const void *X, int M, int K, float *colmax, cuda
 cudaError_t qvggt_launch_smooth_finalize(const float *ax, const float *aw, int K, float alpha, float lo, float hi,
                                          float *c, cudaStream_t st);
 
+// rsq_tc.cu (tensor-core Hadamard mode; per-token scales; c8: one code per byte; y_debug fp32 [M, K] or nullptr)
+cudaError_t qvggt_launch_rsq_tc(const void *X, long long ldx, int M, int K, const float *mul, int bits, bool c8, void *Xq,
+                                float *scales, float *y_debug, int *status, cudaStream_t st);
+
 // gemm.cu
 cudaError_t qvggt_launch_gemm(const qvggt_weights *w, const unsigned char *Xq, const float *a_scale, int M,
                               int group, void *Y, long long ldy, int *acc_debug, cudaStream_t st);

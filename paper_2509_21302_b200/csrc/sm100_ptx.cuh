@@ -138,6 +138,19 @@ __device__ __forceinline__ void mma_i8_ss(uint32_t d_tmem, uint64_t a_desc, uint
         : "memory");
 }
 
+// D[tmem] (+)= A[smem] * B[smem], bf16 x bf16 -> fp32 (both operands the same 16-bit type), issued by ONE thread.
+__device__ __forceinline__ void mma_bf16_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
+        "}\n" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
 // Arrive on an mbarrier once every tcgen05 operation issued so far by this thread has completed.
 __device__ __forceinline__ void mma_commit(uint32_t bar)
 {
@@ -176,6 +189,29 @@ __device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t saddr)
     d |= static_cast<uint64_t>(1) << 46;                   // descriptor version for sm_100
     d |= static_cast<uint64_t>(2) << 61;                   // 128-byte swizzle
     return d;
+}
+
+// Shared-memory matrix descriptor for an operand stored WITHOUT swizzle as "core matrices" of 8 x 16 bytes (128
+// contiguous bytes each).  K-major operand: a core matrix holds 8 rows (M or N) x 16 bytes of K.  MN-major operand:
+// a core matrix holds 8 K-steps x 16 bytes of M or N.  In both cases `k_stride` is the byte distance between core
+// matrices that are neighbours along K (the "leading" offset field) and `mn_stride` the distance between
+// neighbours along M / N (the "stride" offset field).
+__device__ __forceinline__ uint64_t smem_desc_noswizzle(uint32_t saddr, uint32_t k_stride, uint32_t mn_stride)
+{
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
+    d |= static_cast<uint64_t>((k_stride >> 4) & 0x3FFFu) << 16;
+    d |= static_cast<uint64_t>((mn_stride >> 4) & 0x3FFFu) << 32;
+    d |= static_cast<uint64_t>(1) << 46;                   // descriptor version for sm_100
+    return d;                                              // layout type 0: no swizzle
+}
+
+// Instruction descriptor for kind::f16 with bf16 A and B and an fp32 accumulator; A is K-major, B is K-major or
+// MN-major (b_mn_major).
+__host__ __device__ constexpr uint32_t idesc_bf16_f32(int m, int n, bool b_mn_major)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | (static_cast<uint32_t>(n >> 3) << 17) |
+           (static_cast<uint32_t>(m >> 4) << 24);
 }
 
 // Instruction descriptor for kind::i8: signed 8-bit A and B (both K-major), int32 accumulator.
@@ -312,6 +348,13 @@ __device__ __forceinline__ void tma_load_2d(const void *tmap, uint32_t bar, uint
 {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(smem_dst),
                  "l"(tmap), "r"(x), "r"(y), "r"(bar)
+                 : "memory");
+}
+
+__device__ __forceinline__ void tma_load_3d(const void *tmap, uint32_t bar, uint32_t smem_dst, int x, int y, int z)
+{
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(smem_dst),
+                 "l"(tmap), "r"(x), "r"(y), "r"(z), "r"(bar)
                  : "memory");
 }
 

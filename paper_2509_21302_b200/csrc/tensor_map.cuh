@@ -12,6 +12,11 @@
 bool qvggt_make_map(CUtensorMap *map, CUtensorMapDataType type, const void *base, uint64_t inner, uint64_t rows,
                     uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swizzle);
 
+// 3-D tensor: `d0` contiguous elements, then `d1` pieces `pitch1_bytes` apart, then `d2` pieces `pitch2_bytes` apart;
+// the box is b0 x b1 x b2 elements, no swizzle.
+bool qvggt_make_map3(CUtensorMap *map, CUtensorMapDataType type, const void *base, uint64_t d0, uint64_t d1, uint64_t d2,
+                     uint64_t pitch1_bytes, uint64_t pitch2_bytes, uint32_t b0, uint32_t b1, uint32_t b2);
+
 // Per-device host-side caches.  Function attributes (the opt-in to large dynamic shared memory), occupancy
 // results and SM counts belong to a device, and one process may drive several: every cache is an array indexed
 // by the device ordinal.  Zero means "not set yet"; concurrent first calls both compute the same value.

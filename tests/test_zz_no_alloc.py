@@ -39,9 +39,11 @@ def _both_ways(q, K, N, seed, signs=True, watch_memory=False):
     assert st == 0, q.lib().qvggt_status_string(st)
     torch.cuda.synchronize()
     if watch_memory:
-        # the point of the entry point: neither the driver's free memory nor torch's allocator moved across the call
-        # (the first call on a device may load the kernels' module, so only later calls are watched)
-        assert torch.cuda.mem_get_info()[0] == free0 and torch.cuda.memory_allocated() == used0
+        # the point of the entry point: the call took nothing from the driver's free memory (an allocation would
+        # lower the reading; it may rise when the pool behind an EARLIER stream-ordered allocation is trimmed at a
+        # synchronisation) and torch's allocator did not move.  A kernel's first launch may load its code, so only
+        # calls after the first of each size are watched.
+        assert torch.cuda.mem_get_info()[0] >= free0 and torch.cuda.memory_allocated() == used0
     # against the oracle directly: codes bit-exact, scales and multipliers bit-equal
     ref = oracle.prepare_weights(Wb, ch, vh)
     assert np.array_equal(Wq.cpu().numpy(), ref["wq_packed"])
