@@ -4,9 +4,11 @@
 One "step" = one pass of the whole online hot path over one batch: for each of the four linears of
 one aggregator block (qkv 1024->3072, proj 1024->1024, fc1 1024->4096, fc2 4096->1024) at 8 frames
 (M = 10992 tokens): rotate-smooth-quantize, then W4A4 GEMM + rescale + bias + bf16.  Weight
-preparation is offline and untimed.  Prints ONE JSON line.
+preparation is offline and untimed.  Prints ONE JSON line; with the default workload the line also
+carries the other benchmark configurations (single linear, quantize-kernel sweep, 100-frame scene,
+48-block stack) under "configs" and the other storage formats under "formats".
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload ...]
 """
 from __future__ import annotations
 
@@ -26,8 +28,10 @@ sys.path.insert(0, ROOT)
 import workload  # noqa: E402
 
 FRAMES = 8
+F = workload.TOKENS_PER_FRAME
 NOMINAL_INT8_OVER_BF16 = 2.0      # dense tensor peaks: int8 4.5 POPS vs bf16 2.25 PFLOP/s (nominal ratio)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+MIN_TIMED_S = 0.5                 # the K-step region is repeated until at least this much has been timed
 
 
 def load_peaks():
@@ -43,34 +47,43 @@ def layer_ops(M, spec):
     return 2.0 * M * spec.N * spec.K
 
 
-def gemm_bytes(M, spec, code_bytes=0.5):
-    return M * spec.K * code_bytes + 4 * M + spec.N * spec.K * code_bytes + 6 * spec.N + 2.0 * M * spec.N
+def gemm_bytes(M, K, N, code_bytes=0.5, groups=1):
+    """Algorithmic bytes of one GEMM + epilogue: codes of both operands, scales, bias, bf16 output."""
+    return M * K * code_bytes + 4 * M * groups + N * K * code_bytes + 6 * N + 2.0 * M * N
 
 
-def rsq_bytes(M, K, code_bytes=0.5):
-    return M * (2 * K + K * code_bytes + 4)
+def rsq_bytes(M, K, groups=1):
+    """Algorithmic bytes of rotate-smooth-quantize, whatever the storage format: the bf16 row in, two 4-bit codes per
+    byte and one fp32 scale (per group) out.  A format that writes one code per byte moves K/2 more per row: that shows
+    in the DRAM traffic, not here."""
+    return M * (2 * K + K * 0.5 + 4 * groups)
 
 
 class Path:
-    """The two storage formats of the codes between the quantize kernel and the GEMM: `packed` (two codes per
-    byte) and `c8` (one code per byte, TMA-fed GEMM without an unpacking stage).  Same codes, scales and outputs."""
+    """Storage format of the codes between the quantize kernel and the GEMM, and the quantize kernel used:
+    `packed` (two codes per byte), `c8` (one code per byte, TMA-fed GEMM), `w8a8` (8-bit codes); `tc=True` takes the
+    tensor-core Hadamard mode of the quantize kernel (tolerance contract) instead of the exact one."""
 
-    def __init__(self, q, torch, fmt: str):
-        self.fmt = fmt
+    def __init__(self, q, torch, fmt: str, tc: bool = False):
+        self.fmt, self.tc = fmt, tc
         self.code_bytes = 0.5 if fmt == "packed" else 1.0
         self.bits = 8 if fmt == "w8a8" else 4
+        self.name = fmt + ("_tc" if tc else "")
         if fmt in ("c8", "w8a8"):
-            self.prepare = lambda W, b, c: q.prepare_weights(W, b, c, None, c8=True, bits=self.bits)
-            self.rsq = lambda h, x, xq, a: q.rotate_smooth_quantize_c8(h, x, xq, a)
+            self.prepare = lambda W, b, c: q.prepare_weights(W, b, c, None, c8=(True if fmt == "w8a8" else "only"), bits=self.bits)
+            self.rsq = (lambda h, x, xq, a: q.rotate_smooth_quantize_tc(h, x, True, xq, a)) if tc else \
+                       (lambda h, x, xq, a: q.rotate_smooth_quantize_c8(h, x, xq, a))
             self.gemm = lambda h, xq, a, y: q.w4a4_linear_c8(h, xq, a, y)
             self.new_xq = lambda M, K: torch.empty((M, K), dtype=torch.int8, device="cuda")
-            self.gemm_kernel, self.rsq_kernel = "gemm_c8_kernel", "rsq_sq_kernel<.., c8>"
+            self.gemm_kernel = "gemm_c8_kernel"
         else:
             self.prepare = lambda W, b, c: q.prepare_weights(W, b, c, None)
-            self.rsq = lambda h, x, xq, a: q.rotate_smooth_quantize(h, x, 0, xq, a)
+            self.rsq = (lambda h, x, xq, a: q.rotate_smooth_quantize_tc(h, x, False, xq, a)) if tc else \
+                       (lambda h, x, xq, a: q.rotate_smooth_quantize(h, x, 0, xq, a))
             self.gemm = lambda h, xq, a, y: q.w4a4_linear(h, xq, a, 0, y)
             self.new_xq = lambda M, K: torch.empty((M, K // 2), dtype=torch.uint8, device="cuda")
-            self.gemm_kernel, self.rsq_kernel = "gemm_w4a4_kernel", "rsq_sq_kernel"
+            self.gemm_kernel = "gemm_w4a4_kernel"
+        self.rsq_kernel = "rsq_tc_kernel" if tc else "rsq_sq_kernel"
 
 
 def rank_row0(rank: int, rows_per_rank: int) -> int:
@@ -131,7 +144,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, smax, reasons = [], None, set()
+        sm, smax, power, reasons = [], None, [], set()
         inside = [r for (t, r) in self.rows if t_begin <= t <= t_end]
         if not inside:                       # region shorter than one sampling period: take the nearest samples
             inside = [r for (_, r) in self.rows[-3:]]
@@ -139,13 +152,48 @@ class ClockSampler:
             try:
                 sm.append(float(r[0]))
                 smax = float(r[1])
+                power.append(float(r[2]))
                 for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
                     if val.lower().startswith("active"):
                         reasons.add(name)
             except Exception:
                 pass
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": smax, "reasons": sorted(reasons),
-                "samples": len(sm)}
+                "samples": len(sm), "power_w_max": max(power) if power else None}
+
+
+def dev_bf16(torch, bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def timed_us(torch, fn, reps, flush=None):
+    """Median duration of fn() in microseconds over `reps` launches, each between its own event pair; with `flush` (a
+    buffer larger than L2) zeroed before every launch, so that the launch starts with a cold L2."""
+    times = []
+    for _ in range(reps):
+        if flush is not None:
+            flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    return float(np.median(times)) * 1e3
+
+
+def back_to_back_us(torch, fn, reps=20):
+    """Duration per launch of fn(i) when launched `reps` times back to back between one event pair."""
+    for i in range(3):
+        fn(i)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(reps):
+        fn(i)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps * 1e3
 
 
 # ------------------------------------------------------------------------------------------------ oracle arm
@@ -186,7 +234,7 @@ def run_reference(args, rank, world):
     }))
 
 
-def cpu_baseline(rows=FRAMES * workload.TOKENS_PER_FRAME):
+def cpu_baseline(rows=FRAMES * F):
     import oracle
     specs = workload.block_specs(0, 0)
     ops, dt, timings = 0.0, 0.0, {}
@@ -203,7 +251,167 @@ def cpu_baseline(rows=FRAMES * workload.TOKENS_PER_FRAME):
             "tokens_per_s": rows / dt, "seconds": {k: round(v, 3) for k, v in timings.items()}}
 
 
-# ------------------------------------------------------------------------------------------------ CUDA arm
+# ------------------------------------------------------------------------------------------------ one block (configs[1])
+class Block:
+    """The four linears of one aggregator block at 8 frames with device-resident inputs and NBUF buffer sets."""
+
+    NBUF = 2
+
+    def __init__(self, q, torch, path, row0, keep_host=False):
+        self.q, self.torch, self.path = q, torch, path
+        self.M = FRAMES * F
+        self.specs = workload.block_specs(0, 0)
+        self.layers = []
+        for s in self.specs:
+            W = dev_bf16(torch, s.weight())
+            c = q.calibrate_smooth(dev_bf16(torch, s.x_calib()), W)
+            h = path.prepare(W, dev_bf16(torch, s.bias()), c)
+            host_x = torch.from_numpy(s.x_rows(row0, self.M).view(np.int16))
+            if keep_host:
+                host_x = host_x.pin_memory()
+            L = dict(spec=s, h=h, x=[host_x.cuda().view(torch.bfloat16) for _ in range(self.NBUF)],
+                     xq=[path.new_xq(self.M, s.K) for _ in range(self.NBUF)],
+                     a=[torch.empty((self.M,), dtype=torch.float32, device="cuda") for _ in range(self.NBUF)],
+                     y=[torch.empty((self.M, s.N), dtype=torch.bfloat16, device="cuda") for _ in range(self.NBUF)])
+            if keep_host:
+                L["host_x"] = host_x
+                L["host_y"] = torch.empty((self.M, s.N), dtype=torch.bfloat16).pin_memory()
+            self.layers.append(L)
+        torch.cuda.synchronize()
+        self.ops = sum(layer_ops(self.M, s) for s in self.specs)
+
+    def step(self, i, ev=None):
+        b = i % self.NBUF
+        p = self.path
+        for li, L in enumerate(self.layers):
+            if ev is not None:
+                ev[li][0].record()
+            p.rsq(L["h"], L["x"][b], L["xq"][b], L["a"][b])
+            if ev is not None:
+                ev[li][1].record()
+            p.gemm(L["h"], L["xq"][b], L["a"][b], L["y"][b])
+            if ev is not None:
+                ev[li][2].record()
+
+    def timed(self, steps, warmup, barrier, min_s=MIN_TIMED_S, max_repeats=400):
+        """The K-step region, repeated back to back until at least min_s has been timed: one event pair per repeat.
+        Returns the per-step milliseconds of every repeat."""
+        torch = self.torch
+        for i in range(max(warmup, 3)):
+            self.step(i)
+        barrier()
+        probe0, probe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        probe0.record()
+        for i in range(steps):
+            self.step(i)
+        probe1.record()
+        barrier()
+        est_s = max(probe0.elapsed_time(probe1) * 1e-3, 1e-6)
+        repeats = int(min(max_repeats, max(1, np.ceil(min_s / est_s))))
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(repeats + 1)]
+        barrier()
+        wall0 = time.time()
+        evs[0].record()
+        for r in range(repeats):
+            for i in range(steps):
+                self.step(i)
+            evs[r + 1].record()
+        barrier()
+        wall1 = time.time()
+        ms = np.array([evs[r].elapsed_time(evs[r + 1]) / steps for r in range(repeats)])
+        return ms, wall0, wall1
+
+    def per_kernel(self, ksteps):
+        """The same steps with an event after every launch: serialised per-kernel durations (ms), [ksteps, layers]."""
+        torch = self.torch
+        kev = [[[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in self.layers] for _ in range(ksteps)]
+        for i in range(ksteps):
+            self.step(i, kev[i])
+        torch.cuda.synchronize()
+        n = len(self.layers)
+        rsq = np.array([[kev[i][li][0].elapsed_time(kev[i][li][1]) for li in range(n)] for i in range(ksteps)])
+        gemm = np.array([[kev[i][li][1].elapsed_time(kev[i][li][2]) for li in range(n)] for i in range(ksteps)])
+        return rsq, gemm
+
+    def back_to_back(self):
+        torch, p, NB = self.torch, self.path, self.NBUF
+        g = np.array([back_to_back_us(torch, lambda i, L=L: p.gemm(L["h"], L["xq"][i % NB], L["a"][i % NB], L["y"][i % NB])) for L in self.layers])
+        r = np.array([back_to_back_us(torch, lambda i, L=L: p.rsq(L["h"], L["x"][i % NB], L["xq"][i % NB], L["a"][i % NB])) for L in self.layers])
+        return r, g
+
+    def check_status(self):
+        for L in self.layers:
+            assert L["h"].device_status() == 0, "a device-side wait expired"
+
+    def free(self):
+        for L in self.layers:
+            L["h"].free()
+        self.layers = []
+        self.torch.cuda.empty_cache()
+
+
+def e2e_ms(torch, blk, steps, barrier):
+    """End to end: host buffers in, host buffers out, copies inside the timed region.  Three streams (host->device,
+    kernels, device->host) chained by events, two buffer sets: the copies of neighbouring layers and steps overlap the
+    kernels and each other (PCIe is full duplex), as a serving loop would run them; every step still moves all of its
+    inputs from pinned host memory and all of its outputs back."""
+    NB, layers, path = blk.NBUF, blk.layers, blk.path
+    s_in, s_k, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+    ev_in = [[torch.cuda.Event() for _ in range(NB)] for _ in layers]       # input copy done
+    ev_x_free = [[torch.cuda.Event() for _ in range(NB)] for _ in layers]   # quantize kernel has read x[b]
+    ev_y = [[torch.cuda.Event() for _ in range(NB)] for _ in layers]        # GEMM done
+    ev_y_free = [[torch.cuda.Event() for _ in range(NB)] for _ in layers]   # output copy done
+
+    def e2e_step(i):
+        b = i % NB
+        for li, L in enumerate(layers):
+            with torch.cuda.stream(s_in):
+                if i >= NB:
+                    s_in.wait_event(ev_x_free[li][b])
+                L["x"][b].view(torch.int16).copy_(L["host_x"], non_blocking=True)
+                ev_in[li][b].record()
+            with torch.cuda.stream(s_k):
+                s_k.wait_event(ev_in[li][b])
+                path.rsq(L["h"], L["x"][b], L["xq"][b], L["a"][b])
+                ev_x_free[li][b].record()
+                if i >= NB:
+                    s_k.wait_event(ev_y_free[li][b])
+                path.gemm(L["h"], L["xq"][b], L["a"][b], L["y"][b])
+                ev_y[li][b].record()
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_y[li][b])
+                L["host_y"].copy_(L["y"][b], non_blocking=True)
+                ev_y_free[li][b].record()
+
+    def run(n):
+        cur = torch.cuda.current_stream()
+        for st in (s_in, s_k, s_out):
+            st.wait_stream(cur)
+        for i in range(n):
+            e2e_step(i)
+        for st in (s_in, s_k, s_out):
+            cur.wait_stream(st)
+
+    n = max(4, min(steps, 10))
+    run(2)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    run(n)
+    e1.record()
+    barrier()
+    return e0.elapsed_time(e1) / n
+
+
+def load_traffic(fmt):
+    """DRAM bytes per launch from the committed ncu summaries (profiles/dram_traffic.txt), keyed by the code format."""
+    tpath = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    if not os.path.exists(tpath):
+        return {}
+    with open(tpath) as f:
+        return json.load(f).get(fmt, {})
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
     import paper_2509_21302_b200 as q
@@ -214,219 +422,116 @@ def run_ours(args, rank, world, local_rank):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     q.build()
-    path = Path(q, torch, args.format)
-    cb = path.code_bytes
     peaks = load_peaks()
-    M = FRAMES * workload.TOKENS_PER_FRAME
-    specs = workload.block_specs(0, 0)
+    int8_peak = peaks["bf16_tflops"] * NOMINAL_INT8_OVER_BF16
+    int8_peak_sus = peaks["bf16_tflops_sustained"] * NOMINAL_INT8_OVER_BF16
+    M = FRAMES * F
     row0 = rank_row0(rank, M)                           # weak scaling: every rank gets its own 8 frames
-
-    def dev_bf16(bits):
-        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
-
-    layers = []
-    NBUF = 2                                            # input/output buffer sets, alternated per step
-    for s in specs:
-        W = dev_bf16(s.weight())
-        c = q.calibrate_smooth(dev_bf16(s.x_calib()), W)
-        h = path.prepare(W, dev_bf16(s.bias()), c)
-        host_x = torch.from_numpy(s.x_rows(row0, M).view(np.int16)).pin_memory()
-        xs = [host_x.cuda().view(torch.bfloat16) for _ in range(NBUF)]
-        layers.append(dict(spec=s, h=h, host_x=host_x, x=xs,
-                           xq=[path.new_xq(M, s.K) for _ in range(NBUF)],
-                           a=[torch.empty((M,), dtype=torch.float32, device="cuda") for _ in range(NBUF)],
-                           y=[torch.empty((M, s.N), dtype=torch.bfloat16, device="cuda") for _ in range(NBUF)],
-                           host_y=torch.empty((M, s.N), dtype=torch.bfloat16).pin_memory()))
-    torch.cuda.synchronize()
-
-    def step(i, ev=None):
-        b = i % NBUF
-        for li, L in enumerate(layers):
-            if ev is not None:
-                ev[li][0].record()
-            path.rsq(L["h"], L["x"][b], L["xq"][b], L["a"][b])
-            if ev is not None:
-                ev[li][1].record()
-            path.gemm(L["h"], L["xq"][b], L["a"][b], L["y"][b])
-            if ev is not None:
-                ev[li][2].record()
 
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(max(args.warmup, 3)):
-        step(i)
-    barrier()
-    # timed region: K steps back to back, CUDA events on the launching stream around the whole region (an event
-    # between two kernels would keep the next kernel's preamble from overlapping the previous kernel's tail)
+    path = Path(q, torch, args.format, tc=args.tc)
+    blk = Block(q, torch, path, row0, keep_host=True)
+    specs = blk.specs
     sampler = ClockSampler(local_rank)
     sampler.start()
     sampler.wait_first_sample()
-    t_start, t_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    wall0 = time.time()
-    t_start.record()
-    for i in range(args.steps):
-        step(i)
-    t_stop.record()
-    barrier()
-    wall1 = time.time()
-    total_ms = max_over_ranks(t_start.elapsed_time(t_stop), dist, "cuda")
-    # per-kernel durations: the same steps again with an event after every launch (still under the clock sampler)
-    ksteps = min(args.steps, 500)
-    kev = [[[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in layers] for _ in range(ksteps)]
-    for i in range(ksteps):
-        step(i, kev[i])
-    barrier()
-    wall2 = time.time()
-    clocks = sampler.stop(wall0, wall2)
-    for L in layers:
-        assert L["h"].device_status() == 0, "a device-side wait expired"
-
-    rsq_ms = np.array([[kev[i][li][0].elapsed_time(kev[i][li][1]) for li in range(len(layers))] for i in range(ksteps)])
-    gemm_ms = np.array([[kev[i][li][1].elapsed_time(kev[i][li][2]) for li in range(len(layers))] for i in range(ksteps)])
-
-    # the same launches once more, each kernel back to back with itself (alternating buffer sets) between one event
-    # pair: its duration at pipeline throughput, without the gaps the per-launch events of the pass above open
-    def back_to_back(fn, reps=20):
-        for i in range(3):
-            fn(i)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        e0.record()
-        for i in range(reps):
-            fn(i)
-        e1.record()
-        torch.cuda.synchronize()
-        return e0.elapsed_time(e1) / reps
-
-    b2b_gemm_ms = np.array([back_to_back(lambda i, L=L: path.gemm(L["h"], L["xq"][i % NBUF], L["a"][i % NBUF], L["y"][i % NBUF]))
-                            for L in layers])
-    b2b_rsq_ms = np.array([back_to_back(lambda i, L=L: path.rsq(L["h"], L["x"][i % NBUF], L["xq"][i % NBUF], L["a"][i % NBUF]))
-                           for L in layers])
-
-    # end-to-end: host buffers in, host buffers out, copies inside the timed region.  Three streams (host->device,
-    # kernels, device->host) chained by events, two buffer sets: the copies of neighbouring layers and steps overlap the
-    # kernels and each other (PCIe is full duplex), as a serving loop would run them; every step still moves all of its
-    # inputs from pinned host memory and all of its outputs back.
-    s_in, s_k, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
-    ev_in = [[torch.cuda.Event() for _ in range(NBUF)] for _ in layers]       # input copy done
-    ev_x_free = [[torch.cuda.Event() for _ in range(NBUF)] for _ in layers]   # quantize kernel has read x[b]
-    ev_y = [[torch.cuda.Event() for _ in range(NBUF)] for _ in layers]        # GEMM done
-    ev_y_free = [[torch.cuda.Event() for _ in range(NBUF)] for _ in layers]   # output copy done
-
-    def e2e_step(i):
-        b = i % NBUF
-        for li, L in enumerate(layers):
-            with torch.cuda.stream(s_in):
-                if i >= NBUF:
-                    s_in.wait_event(ev_x_free[li][b])
-                L["x"][b].view(torch.int16).copy_(L["host_x"], non_blocking=True)
-                ev_in[li][b].record()
-            with torch.cuda.stream(s_k):
-                s_k.wait_event(ev_in[li][b])
-                path.rsq(L["h"], L["x"][b], L["xq"][b], L["a"][b])
-                ev_x_free[li][b].record()
-                if i >= NBUF:
-                    s_k.wait_event(ev_y_free[li][b])
-                path.gemm(L["h"], L["xq"][b], L["a"][b], L["y"][b])
-                ev_y[li][b].record()
-            with torch.cuda.stream(s_out):
-                s_out.wait_event(ev_y[li][b])
-                L["host_y"].copy_(L["y"][b], non_blocking=True)
-                ev_y_free[li][b].record()
-
-    def e2e_run(n):
-        cur = torch.cuda.current_stream()
-        for st in (s_in, s_k, s_out):
-            st.wait_stream(cur)
-        for i in range(n):
-            e2e_step(i)
-        for st in (s_in, s_k, s_out):
-            cur.wait_stream(st)
-
-    e2e_steps = max(4, min(args.steps, 10))
-    e2e_run(2)
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    e2e_run(e2e_steps)
-    e1.record()
-    barrier()
-    e2e_ms = max_over_ranks(e0.elapsed_time(e1) / e2e_steps, dist, "cuda")
-
+    ms_rep, wall0, wall1 = blk.timed(args.steps, args.warmup, barrier)
+    ms_med = max_over_ranks(float(np.median(ms_rep)), dist, "cuda")
+    clocks = sampler.stop(wall0, wall1)
+    # per-kernel durations: the same steps again with an event after every launch
+    rsq_ms, gemm_ms = blk.per_kernel(min(args.steps, 500))
+    b2b_rsq_us, b2b_gemm_us = blk.back_to_back()
+    e2e = max_over_ranks(e2e_ms(torch, blk, args.steps, barrier), dist, "cuda")
+    blk.check_status()
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
-    ops_step = sum(layer_ops(M, s) for s in specs)
-    ms_per_step = total_ms / args.steps
-    tops = whole_job_value(world, ops_step, ms_per_step)
-    gemm_ops = sum(layer_ops(M, s) for s in specs)
-    gemm_avg_ms = gemm_ms.mean(axis=0)                    # per layer
-    gemm_tops = gemm_ops / (gemm_avg_ms.sum() * 1e-3) / 1e12
-    int8_peak = peaks["bf16_tflops"] * NOMINAL_INT8_OVER_BF16
-    int8_peak_sus = peaks["bf16_tflops_sustained"] * NOMINAL_INT8_OVER_BF16
-    rsq_avg_ms = rsq_ms.mean(axis=0)
-    rsq_b = sum(rsq_bytes(M, s.K, cb) for s in specs)
+    ops_step = blk.ops
+    tops = whole_job_value(world, ops_step, ms_med)
+    gemm_avg_ms, rsq_avg_ms = gemm_ms.mean(axis=0), rsq_ms.mean(axis=0)
+    gemm_tops = ops_step / (gemm_avg_ms.sum() * 1e-3) / 1e12
+    rsq_b = sum(rsq_bytes(M, s.K) for s in specs)
     rsq_gbs = rsq_b / (rsq_avg_ms.sum() * 1e-3) / 1e9
-    # DRAM bytes per launch from the committed ncu summary (None once a kernel has changed since the capture).
-    # The quantize kernel was captured at M = 137400; its traffic grows with the rows, so it is scaled per row.
-    traffic, rsq_traffic = None, None
-    tpath = os.path.join(ROOT, "profiles", "dram_traffic.txt")
-    if os.path.exists(tpath):
-        with open(tpath) as f:
-            tj = json.load(f)
-        tj = tj.get(path.fmt, {})
-        traffic = tj.get("gemm_bytes_per_launch_avg")
-        per_row = tj.get("rsq_bytes_per_row")
-        if per_row:
-            rsq_traffic = sum(per_row[str(s.K)] * M for s in specs) / len(specs)
+    tj = load_traffic(path.fmt)
+    traffic = tj.get("gemm_bytes_per_launch_avg")
+    per_row = tj.get("rsq_bytes_per_row") if not path.tc else tj.get("rsq_tc_bytes_per_row")
+    rsq_traffic = sum(per_row[str(s.K)] * M for s in specs) / len(specs) if per_row else None
     per_layer = {}
     for li, s in enumerate(specs):
         t_g, t_r = gemm_avg_ms[li] * 1e-3, rsq_avg_ms[li] * 1e-3
-        bound = max(layer_ops(M, s) / (int8_peak * 1e12), gemm_bytes(M, s, cb) / (peaks["hbm_gbs"] * 1e9))
+        bound = max(layer_ops(M, s) / (int8_peak * 1e12), gemm_bytes(M, s.K, s.N) / (peaks["hbm_gbs"] * 1e9))
         per_layer[s.name] = {"gemm_us": round(t_g * 1e6, 2), "gemm_tops": round(layer_ops(M, s) / t_g / 1e12, 1),
                              "gemm_roofline_frac": round(bound / t_g, 4),
-                             "rsq_us": round(t_r * 1e6, 2), "rsq_gbs": round(rsq_bytes(M, s.K, cb) / t_r / 1e9, 1),
-                             "rsq_hbm_frac": round(rsq_bytes(M, s.K, cb) / t_r / 1e9 / peaks["hbm_gbs"], 4)}
+                             "rsq_us": round(t_r * 1e6, 2), "rsq_gbs": round(rsq_bytes(M, s.K) / t_r / 1e9, 1),
+                             "rsq_hbm_frac": round(rsq_bytes(M, s.K) / t_r / 1e9 / peaks["hbm_gbs"], 4)}
+    mhz = clocks.get("sm_mhz") or 0.0
     out = {
         "metric": "w4a4_linear_tops" if path.bits == 4 else "w8a8_linear_tops", "value": tops, "unit": "TOPS", "n_gpus": world,
-        "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_med,
+        "repeats": int(len(ms_rep)), "ms_per_step_min": float(ms_rep.min()), "ms_per_step_max": float(ms_rep.max()),
+        "ms_per_step_x_sm_ghz": ms_med * mhz * 1e-3,
+        "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": f"int{path.bits} x int{path.bits} -> int32 (fp32 rotation and scales)", "data": "synthetic",
-        "tokens_per_s": world * M / (ms_per_step * 1e-3),
+        "tokens_per_s": world * M / (ms_med * 1e-3),
         "config": {"workload": "aggregator block, 4 linears (qkv/proj/fc1/fc2), 8 frames M=10992 per GPU",
-                   "l2": f"step working set ~400 MB > 126 MB L2; {NBUF} buffer sets alternated per step",
-                   "timed": "rotate-smooth-quantize + W4A4 GEMM/epilogue per linear; weight prep offline; one event pair "
-                            "around the K steps; the per-kernel durations behind roofline / per_layer come from a second pass "
-                            "of the same steps with an event after every launch",
+                   "l2": f"step working set ~400 MB > 126 MB L2; {blk.NBUF} buffer sets alternated per step",
+                   "timed": f"rotate-smooth-quantize + W4A4 GEMM/epilogue per linear; weight prep offline; the K-step region is repeated "
+                            f"back to back until >= {MIN_TIMED_S} s has been timed (one event pair per repeat; ms_per_step = median over the "
+                            "repeats); the per-kernel durations behind roofline / per_layer come from a further pass of the same steps "
+                            "with an event after every launch",
                    "code_format": {"c8": "int4 codes one per byte between the kernels (c8)", "packed": "int4 codes packed two per byte",
-                                   "w8a8": "W8A8: int8 codes (Eq. quantization with N = 8), one per byte"}[path.fmt]},
+                                   "w8a8": "W8A8: int8 codes (Eq. quantization with N = 8), one per byte"}[path.fmt],
+                   "quantize_kernel": "tensor-core Hadamard mode (tolerance contract)" if path.tc else "exact fp32 butterflies (bit-exact contract)"},
         "clocks": clocks,
-        "gpu_launches": int(2 * len(layers) * args.steps),
-        "e2e": {"value": world * ops_step / (e2e_ms * 1e-3) / 1e12, "unit": "TOPS", "ms_per_step": e2e_ms,
+        "gpu_launches": int(2 * len(specs) * args.steps * len(ms_rep)),
+        "e2e": {"value": world * ops_step / (e2e * 1e-3) / 1e12, "unit": "TOPS", "ms_per_step": e2e,
                 "h2d_bytes_per_step": int(sum(M * s.K * 2 for s in specs)),
                 "d2h_bytes_per_step": int(sum(M * s.N * 2 for s in specs))},
         "roofline": {"kernel": f"{path.gemm_kernel} (4 launches per step)", "bound": "tensor", "achieved": gemm_tops,
                      "peak": int8_peak, "unit": "TOP/s", "frac": gemm_tops / int8_peak,
                      "peak_note": f"int8 dense = {NOMINAL_INT8_OVER_BF16:g} x bf16 burst, of {peaks['source']}",
                      "frac_of_sustained": gemm_tops / int8_peak_sus, "traffic": traffic,
-                     "back_to_back": {"achieved": gemm_ops / (b2b_gemm_ms.sum() * 1e-3) / 1e12,
-                                      "frac": gemm_ops / (b2b_gemm_ms.sum() * 1e-3) / 1e12 / int8_peak,
-                                      "us": [round(float(x) * 1e3, 2) for x in b2b_gemm_ms],
+                     "back_to_back": {"achieved": ops_step / (b2b_gemm_us.sum() * 1e-6) / 1e12,
+                                      "frac": ops_step / (b2b_gemm_us.sum() * 1e-6) / 1e12 / int8_peak,
+                                      "us": [round(float(x), 2) for x in b2b_gemm_us],
                                       "note": "each GEMM launched 20 x back to back between one event pair (operands L2-warm)"}},
         "roofline_rsq": {"kernel": f"{path.rsq_kernel} (4 launches per step)", "bound": "hbm", "achieved": rsq_gbs,
                          "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": rsq_gbs / peaks["hbm_gbs"],
-                         "peak_note": f"of {peaks['source']}", "traffic": rsq_traffic,
-                         "back_to_back": {"achieved": rsq_b / (b2b_rsq_ms.sum() * 1e-3) / 1e9,
-                                          "frac": rsq_b / (b2b_rsq_ms.sum() * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                                          "us": [round(float(x) * 1e3, 2) for x in b2b_rsq_ms]}},
+                         "peak_note": f"of {peaks['source']}; algorithmic bytes 2K + K/2 + 4 per row for every format", "traffic": rsq_traffic,
+                         "traffic_over_algorithmic": (rsq_traffic * len(specs) / rsq_b) if rsq_traffic else None,
+                         "back_to_back": {"achieved": rsq_b / (b2b_rsq_us.sum() * 1e-6) / 1e9,
+                                          "frac": rsq_b / (b2b_rsq_us.sum() * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                                          "us": [round(float(x), 2) for x in b2b_rsq_us]}},
         "per_layer": per_layer,
     }
+    blk.free()
+    if world == 1 and not args.no_extras:
+        # the other storage formats / quantize modes on the same block, same protocol (shorter: 0.25 s each)
+        formats = {path.name: {"ms_per_step": ms_med, "tops": tops, "gemm_roofline_frac": gemm_tops / int8_peak,
+                               "rsq_hbm_frac": rsq_gbs / peaks["hbm_gbs"]}}
+        for fmt, tc in (("c8", False), ("packed", False), ("c8", True), ("packed", True)):
+            p2 = Path(q, torch, fmt, tc)
+            if p2.name in formats:
+                continue
+            b2 = Block(q, torch, p2, row0)
+            ms2, _, _ = b2.timed(args.steps, 3, barrier, min_s=0.25)
+            r2, g2 = b2.per_kernel(min(args.steps, 100))
+            b2.check_status()
+            formats[p2.name] = {"ms_per_step": float(np.median(ms2)), "tops": b2.ops / (float(np.median(ms2)) * 1e-3) / 1e12,
+                                "gemm_roofline_frac": b2.ops / (g2.mean(axis=0).sum() * 1e-3) / 1e12 / int8_peak,
+                                "rsq_hbm_frac": rsq_b / (r2.mean(axis=0).sum() * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+            b2.free()
+        out["formats"] = formats
+        out["configs"] = {"single": measure_single(q, torch, peaks), "sweep": measure_sweep(q, torch, peaks, [100], reps=10),
+                          "scene": measure_scene(q, torch, peaks, reps=5)}
+        if not args.no_stack:
+            out["configs"]["stack"] = measure_stack(q, torch, Path(q, torch, "c8"), reps=3)
     if world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline()
     print(json.dumps(out))
@@ -434,158 +539,245 @@ def run_ours(args, rank, world, local_rank):
         dist.destroy_process_group()
 
 
-def run_rsq_sweep(args):
-    """The quantize-kernel sweep: rotate-smooth-quantize alone, M = 1374 x {1..100}, K in {1024, 4096}, Student-t(3)
-    entries with 1 % outlier channels; achieved GB/s against the measured copy bandwidth (one JSON line)."""
-    import torch
-    import paper_2509_21302_b200 as q
+# ------------------------------------------------------------------------------------------------ configs[0]: one linear, one frame
+def measure_single(q, torch, peaks):
+    """Single W4A4 linear, 1 frame (M = 1374, K = N = 1024, seed 0): launch-bound (the step is two launches of a few
+    microseconds each); reported for completeness, not against a roofline target."""
+    s = workload.block_specs(0, 0)[1]
+    out = {"workload": "single linear K=N=1024, one frame M=1374, seed 0 (launch-bound)"}
+    for fmt in ("c8", "packed"):
+        p = Path(q, torch, fmt)
+        W = dev_bf16(torch, s.weight())
+        h = p.prepare(W, dev_bf16(torch, s.bias()), q.calibrate_smooth(dev_bf16(torch, s.x_calib()), W))
+        x = dev_bf16(torch, s.x_rows(0, F))
+        xq, a = p.new_xq(F, s.K), torch.empty(F, dtype=torch.float32, device="cuda")
+        y = torch.empty((F, s.N), dtype=torch.bfloat16, device="cuda")
 
-    torch.cuda.set_device(0)
-    q.build()
-    path = Path(q, torch, args.format)
-    peaks = load_peaks()
+        def step(i=0):
+            p.rsq(h, x, xq, a)
+            p.gemm(h, xq, a, y)
+
+        us = back_to_back_us(torch, step, reps=200)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        cold = timed_us(torch, step, 20, flush)
+        assert h.device_status() == 0
+        ops = layer_ops(F, s)
+        out[fmt] = {"us_back_to_back": round(us, 2), "us_cold_l2": round(cold, 2), "tops_back_to_back": round(ops / us / 1e6, 1),
+                    "tokens_per_s": round(F / (us * 1e-6))}
+        h.free()
+        del flush
+    return out
+
+
+# ------------------------------------------------------------------------------------------------ configs[2]: quantize kernel sweep
+def measure_sweep(q, torch, peaks, frames_list, reps=10, extras=False):
+    """Rotate-smooth-quantize alone on Student-t(3) entries with 1 % outlier channels x50, L2 flushed before every launch.
+    Fractions of the measured copy bandwidth use the method's algorithmic bytes (2K + K/2 + 4 per row) for every format."""
     out = {}
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     for K in (1024, 4096):
         W = torch.zeros((128, K), dtype=torch.bfloat16, device="cuda")
-        h = path.prepare(W, None, torch.ones(K, device="cuda"))
-        for frames in (1, 8, 32, 100):
-            M = frames * workload.TOKENS_PER_FRAME
-            X = torch.from_numpy(workload.sweep_activations(3, K, 0, M).view(np.int16)).cuda().view(torch.bfloat16)
-            xq = path.new_xq(M, K)
+        h = q.prepare_weights(W, None, torch.ones(K, device="cuda"), None, c8=True)
+        for frames in frames_list:
+            M = frames * F
+            X = dev_bf16(torch, workload.sweep_activations(3, K, 0, M))
             a = torch.empty((M,), dtype=torch.float32, device="cuda")
-            flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-            for _ in range(3):
-                path.rsq(h, X, xq, a)
-            times = []
-            for _ in range(max(5, min(args.steps, 30))):
-                flush.zero_()                                     # larger than L2: the next launch starts cold
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record()
-                path.rsq(h, X, xq, a)
-                e1.record()
-                torch.cuda.synchronize()
-                times.append(e0.elapsed_time(e1))
-            us = float(np.median(times)) * 1e3
-            gbs = rsq_bytes(M, K, path.code_bytes) / us / 1e3
-            out[f"K{K}_M{M}"] = {"us": round(us, 2), "gbs": round(gbs, 1), "hbm_frac": round(gbs / peaks["hbm_gbs"], 4)}
-            if path.fmt != "packed":
+            xq4 = torch.empty((M, K // 2), dtype=torch.uint8, device="cuda")
+            xq8 = torch.empty((M, K), dtype=torch.int8, device="cuda")
+            row = {}
+            modes = (("exact_packed", lambda: q.rotate_smooth_quantize(h, X, 0, xq4, a)),
+                     ("exact_c8", lambda: q.rotate_smooth_quantize_c8(h, X, xq8, a)),
+                     ("tc_packed", lambda: q.rotate_smooth_quantize_tc(h, X, False, xq4, a)),
+                     ("tc_c8", lambda: q.rotate_smooth_quantize_tc(h, X, True, xq8, a)))
+            for name, fn in modes:
+                for _ in range(3):
+                    fn()
+                us = timed_us(torch, fn, reps, flush)
+                gbs = rsq_bytes(M, K) / us / 1e3
+                row[name] = {"us": round(us, 2), "gbs": round(gbs, 1), "hbm_frac": round(gbs / peaks["hbm_gbs"], 4)}
+            if frames <= 8:
+                for name, fn in modes:
+                    row[name]["us_back_to_back"] = round(back_to_back_us(torch, lambda i: fn(), reps=50), 2)
+            if extras:
                 # the granularity ablation's other arm: static tensor-wise step size (no absolute maximum per token)
                 delta = a.median().reshape(1).contiguous()
-                times = []
-                for _ in range(max(5, min(args.steps, 30))):
-                    flush.zero_()
-                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    e0.record()
-                    q.rotate_smooth_quantize_static_c8(h, X, delta, xq, a)
-                    e1.record()
-                    torch.cuda.synchronize()
-                    times.append(e0.elapsed_time(e1))
-                out[f"K{K}_M{M}"]["static_tensorwise_us"] = round(float(np.median(times)) * 1e3, 2)
-                # upstream fusion: LayerNorm + quantize as two kernels against the fused kernel (same results, bit for bit)
+                row["static_tensorwise_c8_us"] = round(timed_us(torch, lambda: q.rotate_smooth_quantize_static_c8(h, X, delta, xq8, a), reps, flush), 2)
+                # upstream fusion: LayerNorm (or GELU) + quantize as two kernels against the fused kernel
                 gamma = torch.rand(K, device="cuda") + 0.5
                 beta = torch.randn(K, device="cuda") * 0.1
-                ln_out = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+                tmp = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
 
-                def two_kernels():
-                    q.layernorm(X, gamma, beta, 1e-5, ln_out)
-                    path.rsq(h, ln_out, xq, a)
+                def ln_two():
+                    q.layernorm(X, gamma, beta, 1e-5, tmp)
+                    q.rotate_smooth_quantize_c8(h, tmp, xq8, a)
 
-                for name, fn in (("ln_then_quantize_us", two_kernels),
-                                 ("ln_fused_us", lambda: q.layernorm_rotate_smooth_quantize_c8(h, X, gamma, beta, 1e-5, xq, a))):
-                    fn()
-                    times = []
-                    for _ in range(max(5, min(args.steps, 30))):
-                        flush.zero_()
-                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                        e0.record()
-                        fn()
-                        e1.record()
-                        torch.cuda.synchronize()
-                        times.append(e0.elapsed_time(e1))
-                    out[f"K{K}_M{M}"][name] = round(float(np.median(times)) * 1e3, 2)
-                del ln_out
-            del X, xq, a, flush
-    best = max(v["gbs"] for v in out.values())
-    print(json.dumps({"metric": "rsq_gbs", "value": best, "unit": "GB/s", "n_gpus": 1, "higher_is_better": True,
-                      "dtype": "fp32 rotation -> int4", "data": "synthetic",
-                      "config": {"workload": "rotate-smooth-quantize sweep, M = 1374 x {1, 8, 32, 100}; L2 flushed between launches",
-                                 "code_format": path.fmt},
-                      "roofline": {"bound": "hbm", "achieved": best, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                                   "frac": best / peaks["hbm_gbs"], "peak_note": f"of {peaks['source']}", "traffic": None},
-                      "sweep": out}))
+                row["ln_then_quantize_us"] = round(timed_us(torch, ln_two, reps, flush), 2)
+                row["ln_fused_us"] = round(timed_us(torch, lambda: q.layernorm_rotate_smooth_quantize_c8(h, X, gamma, beta, 1e-5, xq8, a), reps, flush), 2)
+                if hasattr(q, "gelu"):
+                    def gelu_two():
+                        q.gelu(X, tmp)
+                        q.rotate_smooth_quantize_c8(h, tmp, xq8, a)
+
+                    row["gelu_then_quantize_us"] = round(timed_us(torch, gelu_two, reps, flush), 2)
+                    row["gelu_fused_us"] = round(timed_us(torch, lambda: q.gelu_rotate_smooth_quantize_c8(h, X, xq8, a), reps, flush), 2)
+                del tmp
+            out[f"K{K}_M{M}"] = row
+            del X, xq4, xq8, a
+        assert h.device_status() == 0
+        h.free()
+    del flush
+    return out
 
 
-def run_stack(args):
-    """The full 48-block linear stack (24 frame + 24 global blocks, 4 linears each) at 32
-    frames (M = 43968): per-layer seeded weights, bias and smoothing factors; activations of the four layer
-    kinds come from the seeded heavy-tailed generator (one tensor per kind, reused by every block: there is no
-    data dependence between layers in this benchmark).  Reports end-to-end linear time and tokens/s."""
+def run_rsq_sweep(args):
     import torch
     import paper_2509_21302_b200 as q
 
     torch.cuda.set_device(0)
     q.build()
-    path = Path(q, torch, args.format)
-    M, blocks = 32 * workload.TOKENS_PER_FRAME, 48
+    peaks = load_peaks()
+    frames = [int(f) for f in args.frames.split(",")]
+    sweep = measure_sweep(q, torch, peaks, frames, reps=max(5, min(args.steps, 30)), extras=not args.no_extras)
+    best = max(v["exact_packed"]["gbs"] for v in sweep.values())
+    print(json.dumps({"metric": "rsq_gbs", "value": best, "unit": "GB/s", "n_gpus": 1, "higher_is_better": True,
+                      "dtype": "fp32 rotation -> int4", "data": "synthetic",
+                      "config": {"workload": f"rotate-smooth-quantize sweep, M = 1374 x {{{args.frames}}}; L2 flushed between launches",
+                                 "bytes": "2K + K/2 + 4 per row for every format and mode"},
+                      "roofline": {"bound": "hbm", "achieved": best, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                   "frac": best / peaks["hbm_gbs"], "peak_note": f"of {peaks['source']}; exact kernel, packed format", "traffic": None},
+                      "sweep": sweep}))
 
-    def dev_bf16(bits):
-        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
 
+# ------------------------------------------------------------------------------------------------ configs[4]: 100-frame scene
+def measure_scene(q, torch, peaks, reps=5):
+    """Large-scene stress: 100 frames (M = 137400) through fc1 1024->4096 and fc2 4096->1024, per-token scales (both
+    storage formats) and one scale per token per 128 channels (packed format, its own GEMM kernel); seed 4."""
+    M = 100 * F
+    int8_peak = peaks["bf16_tflops"] * NOMINAL_INT8_OVER_BF16
+    out = {"workload": "100 frames M=137400, fc1 1024->4096 and fc2 4096->1024, seed 4; each kernel timed alone, operands > L2"}
+    for which in (2, 3):
+        s = workload.block_specs(4, 0)[which]
+        W = dev_bf16(torch, s.weight())
+        c = q.calibrate_smooth(dev_bf16(torch, s.x_calib()), W)
+        h = q.prepare_weights(W, dev_bf16(torch, s.bias()), c, None, c8=True)
+        x = dev_bf16(torch, s.x_rows(0, M))
+        y = torch.empty((M, s.N), dtype=torch.bfloat16, device="cuda")
+        a = torch.empty(M, dtype=torch.float32, device="cuda")
+        ag = torch.empty((M, s.K // 128), dtype=torch.float32, device="cuda")
+        xq4 = torch.empty((M, s.K // 2), dtype=torch.uint8, device="cuda")
+        xq8 = torch.empty((M, s.K), dtype=torch.int8, device="cuda")
+        row = {}
+        ops = layer_ops(M, s)
+        variants = (("per_token_c8", lambda: q.rotate_smooth_quantize_c8(h, x, xq8, a), lambda: q.w4a4_linear_c8(h, xq8, a, y), 1),
+                    ("per_token_packed", lambda: q.rotate_smooth_quantize(h, x, 0, xq4, a), lambda: q.w4a4_linear(h, xq4, a, 0, y), 1),
+                    ("group128_packed", lambda: q.rotate_smooth_quantize(h, x, 128, xq4, ag), lambda: q.w4a4_linear(h, xq4, ag, 128, y), s.K // 128))
+        for name, rsq, gemm, groups in variants:
+            for fn in (rsq, gemm):
+                for _ in range(2):
+                    fn()
+            t_r, t_g = timed_us(torch, rsq, reps), timed_us(torch, gemm, reps)
+            bound_us = max(ops / (int8_peak * 1e6), gemm_bytes(M, s.K, s.N, 0.5, groups) / (peaks["hbm_gbs"] * 1e3))
+            row[name] = {"rsq_us": round(t_r, 1), "rsq_hbm_frac": round(rsq_bytes(M, s.K, groups) / t_r / 1e3 / peaks["hbm_gbs"], 4),
+                         "gemm_us": round(t_g, 1), "gemm_tops": round(ops / t_g / 1e6, 1), "gemm_roofline_frac": round(bound_us / t_g, 4),
+                         "layer_tokens_per_s": round(M / ((t_r + t_g) * 1e-6))}
+        assert h.device_status() == 0
+        out[s.name] = row
+        h.free()
+        del x, y, a, ag, xq4, xq8
+    return out
+
+
+# ------------------------------------------------------------------------------------------------ configs[3]: 48-block stack
+def measure_stack(q, torch, path, reps=3):
+    """The full 48-block linear stack (24 frame + 24 global blocks, 4 linears each) at 32 frames (M = 43968): per-layer
+    seeded weights, bias, smoothing factors AND activations (every one of the 192 layers reads its own input tensor from
+    the seeded heavy-tailed generator, ~30 GB resident in HBM; there is no data dependence between layers).  Generation,
+    upload and weight preparation are outside the timed region."""
+    M, blocks = 32 * F, 48
     kinds = workload.block_specs(1, 0)
-    xs = [dev_bf16(s.x_rows(0, M)) for s in kinds]
-    xcal = [dev_bf16(s.x_calib()) for s in kinds]
-    handles = []
+    host = {K: np.empty((M, K), dtype=np.uint16) for K in (1024, 4096)}
+    layers = []
+    t0 = time.time()
     for blk in range(blocks):
         for i, s in enumerate(workload.block_specs(1, blk)):
-            W = dev_bf16(s.weight())
-            c = q.calibrate_smooth(xcal[i], W)
-            handles.append((i, path.prepare(W, dev_bf16(s.bias()), c)))
+            W = dev_bf16(torch, s.weight())
+            c = q.calibrate_smooth(dev_bf16(torch, s.x_calib()), W)
+            x = dev_bf16(torch, s.x_rows(0, M, out=host[s.K]))
+            layers.append((i, path.prepare(W, dev_bf16(torch, s.bias()), c), x))
+    setup_s = time.time() - t0
     xq = [path.new_xq(M, s.K) for s in kinds]
     a = torch.empty((M,), dtype=torch.float32, device="cuda")
     y = [torch.empty((M, s.N), dtype=torch.bfloat16, device="cuda") for s in kinds]
     torch.cuda.synchronize()
 
     def stack():
-        for i, h in handles:
-            path.rsq(h, xs[i], xq[i], a)
+        for i, h, x in layers:
+            path.rsq(h, x, xq[i], a)
             path.gemm(h, xq[i], a, y[i])
 
-    for _ in range(2):
-        stack()
+    stack()
     torch.cuda.synchronize()
-    reps = max(3, min(args.steps, 10))
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
+    times = []
     for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
         stack()
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / reps
-    for _, h in handles:
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    ms = float(np.median(times))
+    for _, h, _x in layers:
         assert h.device_status() == 0
     ops = blocks * sum(layer_ops(M, s) for s in kinds)
-    print(json.dumps({"metric": "w4a4_linear_tops", "value": ops / (ms * 1e-3) / 1e12, "unit": "TOPS", "n_gpus": 1,
-                      "steps": reps, "ms_per_step": ms, "higher_is_better": True, "data": "synthetic",
-                      "dtype": "int4 x int4 -> int32 (fp32 rotation and scales)", "tokens_per_s": M / (ms * 1e-3),
-                      "gpu_launches": 2 * len(handles) * reps,
-                      "config": {"workload": "48-block linear stack, 32 frames M=43968",
-                                 "l2": "per-layer working set 90-450 MB > 126 MB L2", "code_format": path.fmt}}))
+    res = {"workload": "48-block linear stack, 32 frames M=43968, activations regenerated per layer (192 tensors, ~30 GB in HBM)",
+           "code_format": path.name, "ms": round(ms, 3), "tops": round(ops / (ms * 1e-3) / 1e12, 1), "tokens_per_s": round(M / (ms * 1e-3)),
+           "gpu_launches": 2 * len(layers) * reps, "reps": reps, "setup_s": round(setup_s, 1)}
+    for _, h, _x in layers:
+        h.free()
+    del layers, xq, y
+    torch.cuda.empty_cache()
+    return res
+
+
+def run_one(args, fn_name):
+    import torch
+    import paper_2509_21302_b200 as q
+
+    torch.cuda.set_device(0)
+    q.build()
+    peaks = load_peaks()
+    if fn_name == "single":
+        res = measure_single(q, torch, peaks)
+        val = res["c8"]["tops_back_to_back"]
+    elif fn_name == "scene":
+        res = measure_scene(q, torch, peaks, reps=max(3, min(args.steps, 10)))
+        val = res["fc1"]["per_token_c8"]["gemm_tops"]
+    else:
+        res = measure_stack(q, torch, Path(q, torch, args.format, tc=args.tc), reps=max(3, min(args.steps, 10)))
+        val = res["tops"]
+    print(json.dumps({"metric": "w4a4_linear_tops", "value": val, "unit": "TOPS", "n_gpus": 1, "higher_is_better": True,
+                      "data": "synthetic", "dtype": "int4 x int4 -> int32 (fp32 rotation and scales)",
+                      "config": {"workload": res["workload"]}, fn_name: res}))
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--ref-rows", type=int, default=512, help="token rows per step of the oracle arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="block workload only: skip the formats / configs keys")
+    ap.add_argument("--no-stack", action="store_true", help="skip the 48-block stack inside the default line (about a minute of input generation)")
     ap.add_argument("--format", choices=["c8", "packed", "w8a8"], default="c8",
                     help="storage of the int4 codes between the kernels: c8 = one per byte (default), packed = two per byte; "
                          "w8a8 = the paper's 8-bit setting through the same kernels (not the headline metric)")
-    ap.add_argument("--workload", choices=["block", "rsq_sweep", "stack"], default="block",
-                    help="block = one aggregator block at 8 frames (the default line); rsq_sweep = the quantize kernel alone over M; "
-                         "stack = all 48 blocks at 32 frames")
+    ap.add_argument("--frames", default="1,2,4,8,16,32,64,100", help="rsq_sweep only: frame counts (M = 1374 x frames), comma-separated")
+    ap.add_argument("--tc", action="store_true", help="quantize kernel in its tensor-core Hadamard mode (tolerance contract; not the headline)")
+    ap.add_argument("--workload", choices=["block", "single", "rsq_sweep", "stack", "scene"], default="block",
+                    help="block = one aggregator block at 8 frames (the default line, which also carries the others in brief); single = one "
+                         "linear at one frame; rsq_sweep = the quantize kernel alone over M; stack = all 48 blocks at 32 frames; scene = 100 frames")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -595,9 +787,9 @@ def main():
     elif args.workload == "rsq_sweep":
         if rank == 0:
             run_rsq_sweep(args)
-    elif args.workload == "stack":
+    elif args.workload in ("single", "stack", "scene"):
         if rank == 0:
-            run_stack(args)
+            run_one(args, args.workload)
     else:
         run_ours(args, rank, world, local_rank)
 

@@ -18,11 +18,13 @@
 // No data is reshuffled for the tensor core: a token row lands in shared memory as it is in global memory (TMA, no
 // swizzle), and is read as an MN-major B operand whose 16-byte units are the 8 consecutive elements (c = 0..7) of one j.
 // Persistent, one CTA per SM:
-//   warps 0..7  epilogue (TMEM lane quarter w % 4, column half w / 4): TMEM -> registers, butterflies, multiplier,
-//               absolute maximum (warp reduction + exchange through shared memory: a token spans all 128 lanes),
-//               quantize, pack, coalesced global stores (thread j' owns 8 consecutive codes of a token)
-//   warp 8      one thread issues the 8 tcgen05.mma (K = 16 each) of a tile and the commits
-//   warp 9      one thread issues the TMA loads (4 boxes of 16 KB per 64 KB stage)
+//   warps 0..15 epilogue (TMEM lane quarter w % 4, column group w / 4 of 64 columns): TMEM -> registers, butterflies,
+//               multiplier, absolute maximum (warp reduction + exchange through shared memory: a token spans all 128
+//               lanes), quantize, pack, coalesced global stores (thread j' owns 8 consecutive codes of a token)
+//   warp 16     one thread issues the 8 tcgen05.mma (K = 16 each) of a tile and the commits
+//   warp 17     one thread issues the TMA loads (4 boxes of 16 KB per 64 KB stage)
+// The epilogue is latency-bound, not issue-bound (two barriers and a division sit on every tile's critical path), hence
+// the 16 warps: four per scheduler, each with 64 live values.
 #include <cuda.h>
 
 #include "qvggt_internal.cuh"
@@ -31,7 +33,7 @@
 
 namespace {
 
-constexpr int EPI_WARPS = 8;
+constexpr int EPI_WARPS = 16;
 constexpr int MMA_WARP = EPI_WARPS, TMA_WARP = EPI_WARPS + 1;
 constexpr int THREADS = (EPI_WARPS + 2) * 32;
 constexpr int NCOL = 256;                         // columns of one tile = (token, a, c) triples
@@ -45,10 +47,9 @@ constexpr int OFF_BAR = OFF_STAGE + STAGES * STAGE;          // full[STAGES] emp
 constexpr int NBARS = 2 * STAGES + 2 * ACC_BUFS;
 constexpr int OFF_TMEM = OFF_BAR + NBARS * 8;
 constexpr int OFF_ABORT = OFF_TMEM + 4;
-constexpr int OFF_FLAGS = OFF_ABORT + 4;                      // 2 outcome words of the epilogue's group wait
-constexpr int OFF_EXCH = (OFF_FLAGS + 8 + 15) & ~15;          // [2 halves][16 tokens][4 lane quarters] partial maxima
-constexpr int OFF_INV = OFF_EXCH + 2 * 16 * 4 * 4;            // [2 halves][16 tokens] quantization factors
-constexpr int SMEM_BYTES = OFF_INV + 2 * 16 * 4;
+constexpr int OFF_FLAGS = OFF_ABORT + 4;                      // 2 outcome words per column group for its group wait
+constexpr int OFF_EXCH = (OFF_FLAGS + 32 + 15) & ~15;         // [2 tile parities][4 column groups][8 tokens][4 lane quarters] partial maxima
+constexpr int SMEM_BYTES = OFF_EXCH + 2 * 4 * 8 * 4 * 4;
 constexpr int DYN_SMEM = SMEM_BYTES + 128;                    // slack to align the base to 128 bytes
 static_assert(DYN_SMEM <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 
@@ -102,7 +103,7 @@ rsq_tc_kernel(const __grid_constant__ CUtensorMap map_x, int M, const float *__r
     constexpr int PIECES = K / 1024;                 // 1024-element pieces per token (the index bits above bit 9)
     constexpr int VPT = 8 * PIECES;                  // values of one token in one thread: 8 or 32
     constexpr int TOK_TILE = NCOL / VPT;             // tokens per tile: 32 or 8
-    constexpr int TOK_HALF = TOK_TILE / 2;           // tokens per column half: 16 or 4
+    constexpr int TOK_G = 64 / VPT;                  // tokens per column group of 64 columns: 8 or 2
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     const uint32_t sbase = ptx::smem_addr(smem);
@@ -155,56 +156,63 @@ rsq_tc_kernel(const __grid_constant__ CUtensorMap map_x, int M, const float *__r
 
     if (warp < EPI_WARPS) {
         // ------------------------------------------------------------ epilogue
-        const int quarter = warp & 3, half = warp >> 2;
+        const int quarter = warp & 3, cg = warp >> 2;
         const int j = quarter * 32 + lane;                       // TMEM lane = transformed index bits 3..9
-        const int ht = threadIdx.x & 127;                        // thread within the column half's 4 warps
-        float *exch = reinterpret_cast<float *>(smem + OFF_EXCH) + half * 64;     // [token][quarter]
-        float *invs = reinterpret_cast<float *>(smem + OFF_INV) + half * 16;
-        // multipliers of this thread's elements: register 8 a + c <-> element 1024 a + 8 j + c
-        float m[VPT];
-#pragma unroll
-        for (int a = 0; a < PIECES; ++a) {
-            const float4 lo = __ldg(reinterpret_cast<const float4 *>(mul + 1024 * a + 8 * j));
-            const float4 hi = __ldg(reinterpret_cast<const float4 *>(mul + 1024 * a + 8 * j + 4));
-            m[8 * a] = lo.x; m[8 * a + 1] = lo.y; m[8 * a + 2] = lo.z; m[8 * a + 3] = lo.w;
-            m[8 * a + 4] = hi.x; m[8 * a + 5] = hi.y; m[8 * a + 6] = hi.z; m[8 * a + 7] = hi.w;
+        float *exch = reinterpret_cast<float *>(smem + OFF_EXCH) + cg * 32;       // [parity][group][token][quarter]
+        // multipliers of this thread's elements: register 8 a + c <-> element 1024 a + 8 j + c.  K = 1024 keeps them in
+        // registers; K = 4096 re-reads them per token (they stay in L1): 32 more live registers would spill.
+        float m[8];
+        if (PIECES == 1) {
+            const float4 lo = __ldg(reinterpret_cast<const float4 *>(mul + 8 * j));
+            const float4 hi = __ldg(reinterpret_cast<const float4 *>(mul + 8 * j + 4));
+            m[0] = lo.x; m[1] = lo.y; m[2] = lo.z; m[3] = lo.w; m[4] = hi.x; m[5] = hi.y; m[6] = hi.z; m[7] = hi.w;
         }
         bool alive = true;
         uint32_t toggle = 0;
-        for (int t = 0; t < my_tiles; ++t) {
+        for (int t = 0; t < my_tiles && alive; ++t) {
             const int tile = blockIdx.x + t * gridDim.x;
             const int b = t & 1;
-            const long long row0 = (long long)tile * TOK_TILE + half * TOK_HALF;     // first token of this warp's column half
-            alive = ptx::mbar_wait_group(bar_tfull + 8 * b, (t >> 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM, threadIdx.x == 0, 1,
-                                         EPI_WARPS * 32, s_flags, toggle, 32) && alive;
+            const long long row0 = (long long)tile * TOK_TILE + cg * TOK_G;         // first token of this warp's column group
+            // one thread of the column group polls; the outcome is the same for its four warps, which meet again below
+            alive = ptx::mbar_wait_group(bar_tfull + 8 * b, (t >> 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM, (threadIdx.x & 127) == 0,
+                                         1 + cg, 128, s_flags + 2 * cg, toggle, 32);
+            if (!alive) break;
             ptx::tc_fence_after_sync();
-            if (!alive) continue;
-            // the warp's 32 lanes x 128 columns of the accumulator -> registers; tensor memory is handed back at once
-            uint32_t raw[4][32];
+            // the warp's 32 lanes x 64 columns of the accumulator -> registers; tensor memory is handed back at once
+            uint32_t raw[2][32];
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
-                ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + b * NCOL + half * 128 + c * 32, raw[c]);
+            for (int c = 0; c < 2; ++c)
+                ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + b * NCOL + cg * 64 + c * 32, raw[c]);
             ptx::tmem_ld_wait();
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(bar_tempty + 8 * b);
-            float *v = reinterpret_cast<float *>(&raw[0][0]);   // v[VPT * i + r]: token i of the half, register r
+            float *v = reinterpret_cast<float *>(&raw[0][0]);   // v[VPT * i + r]: token i of the group, register r
             // remaining index bits in registers, multiplier, per-token maximum of this warp's 32 lanes
+            uint32_t mine = 0;                                   // lane i keeps the warp's maximum of token i
 #pragma unroll
-            for (int i = 0; i < TOK_HALF; ++i) {
+            for (int i = 0; i < TOK_G; ++i) {
                 float *y = v + VPT * i;
                 stages_over_registers<VPT>(y);
 #pragma unroll
-                for (int r = 0; r < VPT; r += 2) {
-                    const uint64_t p = ptx::f32x2_mul(ptx::f32x2_pack(y[r], y[r + 1]), ptx::f32x2_pack(m[r], m[r + 1]));
-                    ptx::f32x2_unpack(p, y[r], y[r + 1]);
+                for (int a = 0; a < PIECES; ++a) {
+                    if (PIECES > 1) {
+                        const float4 lo = __ldg(reinterpret_cast<const float4 *>(mul + 1024 * a + 8 * j));
+                        const float4 hi = __ldg(reinterpret_cast<const float4 *>(mul + 1024 * a + 8 * j + 4));
+                        m[0] = lo.x; m[1] = lo.y; m[2] = lo.z; m[3] = lo.w; m[4] = hi.x; m[5] = hi.y; m[6] = hi.z; m[7] = hi.w;
+                    }
+#pragma unroll
+                    for (int r = 0; r < 8; r += 2) {
+                        const uint64_t p = ptx::f32x2_mul(ptx::f32x2_pack(y[8 * a + r], y[8 * a + r + 1]), ptx::f32x2_pack(m[r], m[r + 1]));
+                        ptx::f32x2_unpack(p, y[8 * a + r], y[8 * a + r + 1]);
+                    }
                 }
                 float am = fmaxf(fabsf(y[0]), fabsf(y[1]));
 #pragma unroll
                 for (int r = 2; r < VPT; r += 2) asm("max.abs.f32 %0, %1, %2, %3;" : "=f"(am) : "f"(am), "f"(y[r]), "f"(y[r + 1]));
                 // non-negative floats order like their bit patterns: one integer warp reduction
                 const uint32_t wm = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(am));
-                if (lane == 0) exch[i * 4 + quarter] = __uint_as_float(wm);
+                if (lane == i) mine = wm;
                 if (DUMP && y_debug && row0 + i < M) {
 #pragma unroll
                     for (int a = 0; a < PIECES; ++a) {
@@ -214,19 +222,23 @@ rsq_tc_kernel(const __grid_constant__ CUtensorMap map_x, int M, const float *__r
                     }
                 }
             }
-            asm volatile("bar.sync %0, %1;" ::"r"(2 + half), "r"(128) : "memory");
-            if (ht < TOK_HALF) {
-                const float4 q4 = *reinterpret_cast<const float4 *>(exch + ht * 4);
+            // the four warps of the column group exchange their maxima (buffers alternate with the tile parity: a warp may
+            // already write the next tile's maxima while a slower one still reads this tile's)
+            float *ex = exch + b * 128;
+            if (lane < TOK_G) ex[lane * 4 + quarter] = __uint_as_float(mine);
+            asm volatile("bar.sync %0, %1;" ::"r"(1 + cg), "r"(128) : "memory");
+            float inv_mine = 0.0f;
+            if (lane < TOK_G) {
+                const float4 q4 = *reinterpret_cast<const float4 *>(ex + lane * 4);
                 const float amax = fmaxf(fmaxf(fmaxf(q4.x, q4.y), fmaxf(q4.z, q4.w)), 1e-8f);
-                invs[ht] = __fdiv_rn(static_cast<float>(QMAX), amax);
-                if (row0 + ht < M) scales[row0 + ht] = __fdiv_rn(amax, static_cast<float>(QMAX));
+                inv_mine = __fdiv_rn(static_cast<float>(QMAX), amax);
+                if (quarter == 0 && row0 + lane < M) scales[row0 + lane] = __fdiv_rn(amax, static_cast<float>(QMAX));
             }
-            asm volatile("bar.sync %0, %1;" ::"r"(2 + half), "r"(128) : "memory");
             const uint64_t magic2 = ptx::f32x2_pack(12582912.0f, 12582912.0f);
 #pragma unroll
-            for (int i = 0; i < TOK_HALF; ++i) {
+            for (int i = 0; i < TOK_G; ++i) {
                 const float *y = v + VPT * i;
-                const float inv = invs[i];
+                const float inv = __shfl_sync(0xFFFFFFFFu, inv_mine, i);
                 const uint64_t inv2 = ptx::f32x2_pack(inv, inv);
                 const bool row_ok = row0 + i < M;
 #pragma unroll
