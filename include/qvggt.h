@@ -198,6 +198,20 @@ int qvggt_layernorm(const void *X_bf16, long long ldx, int M, int K, const float
 int qvggt_debug_starved_linear_c8(const qvggt_weights_t *w, const signed char *Xq8, const float *a_scale, int M,
                                   void *Y_bf16, long long ldy, long long wait_limit_cycles, void *cuda_stream);
 
+/*
+ * The other half of the upstream fusion: fc2's input is the MLP's activation function applied to fc1's output.  The
+ * paper does not name the function; the transformer blocks VGGT is built from use the exact GELU x Phi(x) (Phi the
+ * standard normal distribution function), which is what is computed here, in fp32, to within one bf16 ulp of the
+ * exactly rounded value (results of magnitude below 2^-120, i.e. x < -12.9, may be flushed to zero).
+ * qvggt_gelu_rotate_smooth_quantize_c8 applies it to every element on its way into the activation path of
+ * qvggt_rotate_smooth_quantize_c8 -- the activated tensor (the largest activation of the block) never goes to memory --
+ * and returns, bit for bit, the result of qvggt_gelu followed by qvggt_rotate_smooth_quantize_c8.
+ * Arguments as for qvggt_rotate_smooth_quantize_c8 / qvggt_layernorm (Y_bf16 [M, K] contiguous; K = 1024 or 4096).
+ */
+int qvggt_gelu_rotate_smooth_quantize_c8(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M,
+                                         signed char *Xq8, float *a_scale, void *cuda_stream);
+int qvggt_gelu(const void *X_bf16, long long ldx, int M, int K, void *Y_bf16, void *cuda_stream);
+
 /* Frees the handle and its device memory (synchronises the device first).  NULL is allowed. */
 void qvggt_free_weights(qvggt_weights_t *w);
 

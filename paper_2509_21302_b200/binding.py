@@ -23,7 +23,8 @@ EXPORTS = ("qvggt_prepare_weights", "qvggt_rotate_smooth_quantize", "qvggt_w4a4_
            "qvggt_quantize_weights_static", "qvggt_rotate_smooth_quantize_c8", "qvggt_w4a4_linear_c8",
            "qvggt_weights_view_c8", "qvggt_rotate_smooth_quantize_static_c8",
            "qvggt_layernorm_rotate_smooth_quantize_c8", "qvggt_layernorm", "qvggt_debug_starved_linear_c8",
-           "qvggt_rotate_smooth_quantize_tc", "qvggt_rotate_smooth_quantize_tc_c8")
+           "qvggt_rotate_smooth_quantize_tc", "qvggt_rotate_smooth_quantize_tc_c8", "qvggt_gelu",
+           "qvggt_gelu_rotate_smooth_quantize_c8")
 PREP_C8 = 1   # QVGGT_PREP_C8: keep an int8 [N, K] copy of the weight codes for the *_c8 entry points
 PREP_W8A8 = 2  # QVGGT_PREP_W8A8: 8-bit codes (one per byte only)
 PREP_C8_ONLY = 4  # QVGGT_PREP_C8_ONLY: 4-bit codes one per byte only (no packed copy)
@@ -59,6 +60,8 @@ def lib() -> ctypes.CDLL:
         L.qvggt_layernorm.argtypes = [vp, i64, i32, i32, vp, vp, f32, vp, vp]
         L.qvggt_rotate_smooth_quantize_tc.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp]
         L.qvggt_rotate_smooth_quantize_tc_c8.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp]
+        L.qvggt_gelu.argtypes = [vp, i64, i32, i32, vp, vp]
+        L.qvggt_gelu_rotate_smooth_quantize_c8.argtypes = [vp, vp, i64, i32, vp, vp, vp]
         L.qvggt_debug_starved_linear_c8.argtypes = [vp, vp, vp, i32, vp, i64, i64, vp]
         L.qvggt_weights_view_c8.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(i32)]
         L.qvggt_free_weights.argtypes = [vp]
@@ -297,6 +300,30 @@ def layernorm(X: torch.Tensor, gamma: torch.Tensor, beta: torch.Tensor, eps: flo
     ldx = X.stride(0) if M > 1 else K
     _check(lib().qvggt_layernorm(_ptr(X), ldx, M, K, _ptr(gamma), _ptr(beta), eps, _ptr(Y), _stream()), "qvggt_layernorm")
     return Y
+
+
+def gelu(X: torch.Tensor, Y: torch.Tensor | None = None) -> torch.Tensor:
+    """GELU x Phi(x) alone: X [M,K] bf16 -> Y [M,K] bf16 (K = 1024 or 4096)."""
+    assert X.dim() == 2 and X.element_size() == 2 and X.stride(1) == 1
+    M, K = X.shape
+    if Y is None:
+        Y = torch.empty((M, K), dtype=torch.bfloat16, device=X.device)
+    assert Y.is_contiguous() and Y.element_size() == 2
+    _check(lib().qvggt_gelu(_ptr(X), X.stride(0) if M > 1 else K, M, K, _ptr(Y), _stream()), "qvggt_gelu")
+    return Y
+
+
+def gelu_rotate_smooth_quantize_c8(w: Weights, X: torch.Tensor, Xq8: torch.Tensor | None = None, a_scale: torch.Tensor | None = None):
+    """GELU fused in front of rotate_smooth_quantize_c8 -> (Xq8 [M,K] int8, a_scale [M])."""
+    assert X.dim() == 2 and X.element_size() == 2 and X.stride(1) == 1 and X.shape[1] == w.K
+    M = X.shape[0]
+    if Xq8 is None:
+        Xq8 = torch.empty((M, w.K), dtype=torch.int8, device=X.device)
+    if a_scale is None:
+        a_scale = torch.empty((M,), dtype=torch.float32, device=X.device)
+    _check(lib().qvggt_gelu_rotate_smooth_quantize_c8(w.handle, _ptr(X), X.stride(0) if M > 1 else w.K, M, _ptr(Xq8), _ptr(a_scale),
+                                                      _stream()), "qvggt_gelu_rotate_smooth_quantize_c8")
+    return Xq8, a_scale
 
 
 def w4a4_linear_c8(w: Weights, Xq8: torch.Tensor, a_scale: torch.Tensor, Y: torch.Tensor | None = None,

@@ -208,6 +208,31 @@ int qvggt_layernorm(const void *X_bf16, long long ldx, int M, int K, const float
     return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
 }
 
+int qvggt_gelu_rotate_smooth_quantize_c8(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M, signed char *Xq8,
+                                         float *a_scale, void *cuda_stream)
+{
+    if (!w) return QVGGT_ERR_NULL;
+    if (M < 0) return QVGGT_ERR_SHAPE;
+    if (M == 0) return QVGGT_OK;
+    if (!X_bf16 || !Xq8 || !a_scale) return QVGGT_ERR_NULL;
+    if (ldx < w->K) return QVGGT_ERR_SHAPE;
+    if (ldx % 8 != 0 || !aligned16(X_bf16) || !aligned16(Xq8) || (reinterpret_cast<uintptr_t>(a_scale) & 3u)) return QVGGT_ERR_ALIGN;
+    cudaError_t e = qvggt_launch_gelu_rsq_c8(X_bf16, ldx, M, w->K, w->amul, w->bits, Xq8, a_scale, nullptr, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
+}
+
+int qvggt_gelu(const void *X_bf16, long long ldx, int M, int K, void *Y_bf16, void *cuda_stream)
+{
+    if (M < 0 || !valid_k(K)) return QVGGT_ERR_SHAPE;
+    if (M == 0) return QVGGT_OK;
+    if (!X_bf16 || !Y_bf16) return QVGGT_ERR_NULL;
+    if (ldx < K) return QVGGT_ERR_SHAPE;
+    if (ldx % 8 != 0 || !aligned16(X_bf16) || !aligned16(Y_bf16)) return QVGGT_ERR_ALIGN;
+    if (!device_is_sm100()) return QVGGT_ERR_UNSUPPORTED;
+    cudaError_t e = qvggt_launch_gelu_rsq_c8(X_bf16, ldx, M, K, nullptr, 4, nullptr, nullptr, Y_bf16, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
+}
+
 int qvggt_w4a4_linear_c8(const qvggt_weights_t *w, const signed char *Xq8, const float *a_scale, int M, void *Y_bf16,
                          long long ldy, int *acc_debug, void *cuda_stream)
 {

@@ -39,6 +39,8 @@ cudaError_t qvggt_launch_rsq_static_c8(const void *X, long long ldx, int M, int 
                                        signed char *Xq8, float *scales, cudaStream_t st);
 cudaError_t qvggt_launch_ln_rsq_c8(const void *X, long long ldx, int M, int K, const float *mul, int bits, const float *gamma,
                                    const float *beta, float eps, signed char *Xq8, float *scales, void *ln_out, cudaStream_t st);
+cudaError_t qvggt_launch_gelu_rsq_c8(const void *X, long long ldx, int M, int K, const float *mul, int bits, signed char *Xq8,
+                                     float *scales, void *gelu_out, cudaStream_t st);
 cudaError_t qvggt_launch_colmax(const void *X, int M, int K, float *colmax, cudaStream_t st);
 cudaError_t qvggt_launch_smooth_finalize(const float *ax, const float *aw, int K, float alpha, float lo, float hi,
                                          float *c, cudaStream_t st);

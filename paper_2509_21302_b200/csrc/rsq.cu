@@ -161,7 +161,7 @@ struct SqGeom {
 
 // Resident CTAs per SM the kernel is built for: 4 (K = 1024) or 3 (K = 4096); with the fused LayerNorm at K = 4096 the
 // CTA's shared-memory copy of gamma and beta (32 KB) leaves room for 2.
-constexpr int sq_ctas_per_sm(int logt, int ln) { return logt == 5 ? 4 : (ln != 0 ? 2 : 3); }
+constexpr int sq_ctas_per_sm(int logt, int ln) { return logt == 5 ? 4 : ((ln == 1 || ln == 2) ? 2 : 3); }
 
 template <int T>
 __device__ __forceinline__ void group_sync(int slot)
@@ -204,11 +204,35 @@ __device__ __forceinline__ float tree_sum(const float (&a)[N])
     }
 }
 
+// GELU x Phi(x) (the activation between the two linears of the MLP: the producer of fc2's input), evaluated so that the
+// negative tail keeps its RELATIVE accuracy.  With t = |x|, z = t / sqrt(2):
+//   Q(t) = 1 - Phi(t) = exp(-z^2) E(z) / 2,   E(z) = exp(z^2) erfc(z)  (smooth, from 1 down to ~1 / (z sqrt(pi))),
+//   E(z) ~ s P(s),  s = 1 / (1 + 0.55 z),  P a degree-4 polynomial (own weighted least-squares fit on z in [0, 9.6]: relative
+//   error below 6e-5), then gelu(x) = x - x Q for x >= 0 and x Q for x < 0.
+// About 16 instructions, two of them special-function (reciprocal, exp2); relative error ~1e-4 wherever the result is a
+// normal number above 2^-120, i.e. at most one bf16 ulp after rounding; below that (x < -12.9) the exponential
+// flushes to zero.  The fused multiply-adds are written explicitly (the file is compiled without contraction).
+__device__ __forceinline__ float gelu_f32(float x)
+{
+    const float z = __fmul_rn(fabsf(x), 0.70710678f);
+    float s;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(s) : "f"(__fmaf_rn(0.55f, z, 1.0f)));
+    float p = -0.17450283f;
+    p = __fmaf_rn(p, s, 0.33387650f);
+    p = __fmaf_rn(p, s, 0.21415194f);
+    p = __fmaf_rn(p, s, 0.31633197f);
+    p = __fmaf_rn(p, s, 0.31008677f);
+    float e;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(__fmul_rn(__fmul_rn(z, z), -1.44269504f)));
+    const float q = __fmul_rn(__fmul_rn(0.5f, e), __fmul_rn(s, p));
+    return x >= 0.0f ? __fmaf_rn(-x, q, x) : __fmul_rn(x, q);
+}
+
 // Parameters of the LayerNorm that may run in front of the rotation (gamma == nullptr: none).
 struct LnArgs {
     const float *gamma, *beta;   // fp32 [K]
     float eps;
-    uint16_t *out;               // LN == 2 only: bf16 [M, K], the normalized rows (nothing else is computed)
+    uint16_t *out;               // LN == 2 / 4 only: bf16 [M, K], the normalized / activated rows (nothing else is computed)
 };
 
 // C8: one code per byte (int8, natural element order, row pitch K) instead of two per byte.
@@ -216,7 +240,8 @@ struct LnArgs {
 // STATIC (C8 only): one given step size *static_delta for the whole tensor (the static tensor-wise arm of the
 // granularity ablation) instead of one per row from the row's absolute maximum; the clamp of Eq. "quantization"
 // to [-QMAX - 1, QMAX] is then active, and every row's scale is written as that step size.
-// LN: 1 = every row goes through LayerNorm first (fp32, statistics summed pairwise: in-thread tree over the thread's
+// LN (the operation fused in front of the rotation): 3 = GELU on every element, rounded to bf16 as a separate activation
+// kernel would store it; 4 = only that, written out.  1 = every row goes through LayerNorm first (fp32, statistics summed pairwise: in-thread tree over the thread's
 // T contiguous elements, then the xor-shuffle tree over the row's threads -- together the halves-recursion over the
 // row), its output rounded to bf16 as a separate normalization kernel would store it; 2 = only that, written out.
 template <int LOGT, int GROUP, bool C8 = false, int QMAX = 7, bool STATIC = false, int LN = 0>
@@ -273,7 +298,7 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
     // LayerNorm parameters: one copy per CTA in shared memory behind the row slots, as 16-byte pieces ordered
     // [piece][thread], so that thread t reads its T contiguous gammas with conflict-free 16-byte loads (read straight
     // from global memory, thread t's T contiguous values are 4 T bytes away from its neighbour's: 32 sectors per load)
-    constexpr bool LN_SMEM = (LN != 0);
+    constexpr bool LN_SMEM = (LN == 1 || LN == 2);
     float4 *g_sm = reinterpret_cast<float4 *>(dsm + G::SMEM), *b_sm = g_sm + K / 4;
     if constexpr (LN_SMEM) {
         for (int i = threadIdx.x; i < K / 4; i += G::CTA_THREADS) {
@@ -285,7 +310,7 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
     }
     float m[T];                                                // multipliers of elements T k + t (loaded behind the first row's copies)
 #pragma unroll
-    for (int k = 0; k < T; ++k) m[k] = (LN == 2) ? 0.0f : __ldg(mul + T * k + t);   // the normalization alone uses none
+    for (int k = 0; k < T; ++k) m[k] = (LN == 2 || LN == 4) ? 0.0f : __ldg(mul + T * k + t);   // the prologue alone uses none
     int buf = 0;
     for (; row < M; row += stride, buf ^= 1) {
         const long long next = row + stride;
@@ -321,7 +346,23 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
                 }
             }
         }
-        if constexpr (LN != 0) {
+        if constexpr (LN == 3 || LN == 4) {
+            uint32_t packed[T / 2];
+#pragma unroll
+            for (int k = 0; k < T; k += 2) {
+                const uint32_t p01 = ptx::pack_bf16x2(gelu_f32(v[k]), gelu_f32(v[k + 1]));   // what an activation kernel would store
+                v[k] = __uint_as_float(p01 << 16);
+                v[k + 1] = __uint_as_float(p01 & 0xFFFF0000u);
+                packed[k / 2] = p01;
+            }
+            if constexpr (LN == 4) {
+                uint4 *dst = reinterpret_cast<uint4 *>(ln.out + row * K + T * t);
+#pragma unroll
+                for (int k = 0; k < T / 8; ++k) dst[k] = make_uint4(packed[4 * k], packed[4 * k + 1], packed[4 * k + 2], packed[4 * k + 3]);
+                continue;
+            }
+            stages_in_registers<T, true>(v);    // strides 1 .. T/2
+        } else if constexpr (LN != 0) {
             // row sum over the tree: registers, lanes, and (T = 64) the two warps of the row
             auto row_sum = [&](float part, int word) {
 #pragma unroll
@@ -567,7 +608,7 @@ cudaError_t launch_sq(const uint16_t *x, long long ldx, int M, const float *mul,
                       cudaStream_t st, const float *static_delta = nullptr, LnArgs ln = LnArgs{nullptr, nullptr, 0.0f, nullptr})
 {
     using G = SqGeom<LOGT>;
-    constexpr int SMEM = G::SMEM + (LN != 0 ? 2 * G::K * 4 : 0);   // + the CTA's copy of gamma and beta
+    constexpr int SMEM = G::SMEM + ((LN == 1 || LN == 2) ? 2 * G::K * 4 : 0);   // + the CTA's copy of gamma and beta
     static QvggtPerDevice configured;     // per device and instantiation
     const int dev = qvggt_current_device();
     if (dev < 0) return cudaErrorInvalidDevice;
@@ -630,6 +671,23 @@ cudaError_t qvggt_launch_ln_rsq_c8(const void *X, long long ldx, int M, int K, c
                          : launch_sq<6, 0, true, 127, false, 1>(x, ldx, M, mul, out, scales, st, nullptr, ln);
     return K == 1024 ? launch_sq<5, 0, true, 7, false, 1>(x, ldx, M, mul, out, scales, st, nullptr, ln)
                      : launch_sq<6, 0, true, 7, false, 1>(x, ldx, M, mul, out, scales, st, nullptr, ln);
+}
+
+cudaError_t qvggt_launch_gelu_rsq_c8(const void *X, long long ldx, int M, int K, const float *mul, int bits, signed char *Xq8,
+                                     float *scales, void *gelu_out, cudaStream_t st)
+{
+    if (M == 0) return cudaSuccess;
+    const uint16_t *x = static_cast<const uint16_t *>(X);
+    unsigned char *out = reinterpret_cast<unsigned char *>(Xq8);
+    const LnArgs ln = {nullptr, nullptr, 0.0f, static_cast<uint16_t *>(gelu_out)};
+    if (gelu_out)     // the activation alone
+        return K == 1024 ? launch_sq<5, 0, true, 7, false, 4>(x, ldx, M, mul, out, scales, st, nullptr, ln)
+                         : launch_sq<6, 0, true, 7, false, 4>(x, ldx, M, mul, out, scales, st, nullptr, ln);
+    if (bits == 8)
+        return K == 1024 ? launch_sq<5, 0, true, 127, false, 3>(x, ldx, M, mul, out, scales, st, nullptr, ln)
+                         : launch_sq<6, 0, true, 127, false, 3>(x, ldx, M, mul, out, scales, st, nullptr, ln);
+    return K == 1024 ? launch_sq<5, 0, true, 7, false, 3>(x, ldx, M, mul, out, scales, st, nullptr, ln)
+                     : launch_sq<6, 0, true, 7, false, 3>(x, ldx, M, mul, out, scales, st, nullptr, ln);
 }
 
 cudaError_t qvggt_launch_rsq(const void *X, long long ldx, int M, int K, const float *mul, int group,

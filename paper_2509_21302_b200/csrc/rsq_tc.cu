@@ -38,20 +38,27 @@ constexpr int MMA_WARP = EPI_WARPS, TMA_WARP = EPI_WARPS + 1;
 constexpr int THREADS = (EPI_WARPS + 2) * 32;
 constexpr int NCOL = 256;                         // columns of one tile = (token, a, c) triples
 constexpr int STAGE = NCOL / 8 * 2048;            // 32 pieces of 1024 bf16: 64 KB
-constexpr int STAGES = 3;
 constexpr int ACC_BUFS = 2;
 constexpr int H_BYTES = 128 * 128 * 2;            // the bf16 matrix H_128
 constexpr int OFF_H = 0;
 constexpr int OFF_STAGE = OFF_H + H_BYTES;
-constexpr int OFF_BAR = OFF_STAGE + STAGES * STAGE;          // full[STAGES] empty[STAGES] tfull[2] tempty[2]
-constexpr int NBARS = 2 * STAGES + 2 * ACC_BUFS;
-constexpr int OFF_TMEM = OFF_BAR + NBARS * 8;
-constexpr int OFF_ABORT = OFF_TMEM + 4;
-constexpr int OFF_FLAGS = OFF_ABORT + 4;                      // 2 outcome words per column group for its group wait
-constexpr int OFF_EXCH = (OFF_FLAGS + 32 + 15) & ~15;         // [2 tile parities][4 column groups][8 tokens][4 lane quarters] partial maxima
-constexpr int SMEM_BYTES = OFF_EXCH + 2 * 4 * 8 * 4 * 4;
-constexpr int DYN_SMEM = SMEM_BYTES + 128;                    // slack to align the base to 128 bytes
-static_assert(DYN_SMEM <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
+
+// Shared-memory layout behind H_128: K = 1024 has three 64 KB stages and keeps a thread's 8 multipliers in registers;
+// K = 4096 has two stages (the loads still run up to four tiles ahead of the epilogue: two stages plus two
+// accumulators) and a 16 KB copy of the multipliers, [register r][lane j], that every epilogue thread reads per token.
+template <int PIECES>
+struct Lay {
+    static constexpr int STAGES = (PIECES == 1) ? 3 : 2;
+    static constexpr int OFF_MUL = OFF_STAGE + STAGES * STAGE;
+    static constexpr int OFF_BAR = OFF_MUL + ((PIECES == 1) ? 0 : 32 * 128 * 4);       // full[STAGES] empty[STAGES] tfull[2] tempty[2]
+    static constexpr int NBARS = 2 * STAGES + 2 * ACC_BUFS;
+    static constexpr int OFF_TMEM = OFF_BAR + NBARS * 8;
+    static constexpr int OFF_ABORT = OFF_TMEM + 4;
+    static constexpr int OFF_EXCH = (OFF_ABORT + 4 + 15) & ~15;     // [2 tile parities][4 column groups][8 tokens][4 lane quarters] partial maxima
+    static constexpr int SMEM_BYTES = OFF_EXCH + 2 * 4 * 8 * 4 * 4;
+    static constexpr int DYN_SMEM = SMEM_BYTES + 128;               // slack to align the base to 128 bytes
+    static_assert(DYN_SMEM <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
+};
 
 // H_128 as the K-major A operand, no swizzle: core matrix (8 rows m) x (8 elements k) = 128 contiguous bytes;
 // core matrices that are neighbours along k are 128 bytes apart, 8-row groups 2048 bytes.
@@ -104,16 +111,17 @@ rsq_tc_kernel(const __grid_constant__ CUtensorMap map_x, int M, const float *__r
     constexpr int VPT = 8 * PIECES;                  // values of one token in one thread: 8 or 32
     constexpr int TOK_TILE = NCOL / VPT;             // tokens per tile: 32 or 8
     constexpr int TOK_G = 64 / VPT;                  // tokens per column group of 64 columns: 8 or 2
+    using L = Lay<PIECES>;
+    constexpr int STAGES = L::STAGES;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     const uint32_t sbase = ptx::smem_addr(smem);
-    const uint32_t bar_full = sbase + OFF_BAR;
+    const uint32_t bar_full = sbase + L::OFF_BAR;
     const uint32_t bar_empty = bar_full + STAGES * 8;
     const uint32_t bar_tfull = bar_empty + STAGES * 8;
     const uint32_t bar_tempty = bar_tfull + ACC_BUFS * 8;
-    uint32_t *s_tmem = reinterpret_cast<uint32_t *>(smem + OFF_TMEM);
-    volatile int *s_abort = reinterpret_cast<volatile int *>(smem + OFF_ABORT);
-    volatile int *s_flags = reinterpret_cast<volatile int *>(smem + OFF_FLAGS);
+    uint32_t *s_tmem = reinterpret_cast<uint32_t *>(smem + L::OFF_TMEM);
+    volatile int *s_abort = reinterpret_cast<volatile int *>(smem + L::OFF_ABORT);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tiles = (M + TOK_TILE - 1) / TOK_TILE;
@@ -130,6 +138,11 @@ rsq_tc_kernel(const __grid_constant__ CUtensorMap map_x, int M, const float *__r
             w[e] = lo | (hi << 16);
         }
         *reinterpret_cast<uint4 *>(smem + OFF_H + (m >> 3) * A_MN_STRIDE + kc * A_K_STRIDE + (m & 7) * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    if (PIECES > 1) {
+        // multiplier of element 1024 a + 8 j + c -> slot [8 a + c][j]
+        float *m_s = reinterpret_cast<float *>(smem + L::OFF_MUL);
+        for (int e = threadIdx.x; e < K; e += THREADS) m_s[(((e >> 10) << 3) | (e & 7)) * 128 + ((e >> 3) & 127)] = __ldg(mul + e);
     }
     ptx::fence_proxy_async_smem();            // generic-proxy writes -> visible to the tensor core's reads
     if (threadIdx.x == 0) {
@@ -158,9 +171,10 @@ rsq_tc_kernel(const __grid_constant__ CUtensorMap map_x, int M, const float *__r
         // ------------------------------------------------------------ epilogue
         const int quarter = warp & 3, cg = warp >> 2;
         const int j = quarter * 32 + lane;                       // TMEM lane = transformed index bits 3..9
-        float *exch = reinterpret_cast<float *>(smem + OFF_EXCH) + cg * 32;       // [parity][group][token][quarter]
+        float *exch = reinterpret_cast<float *>(smem + L::OFF_EXCH) + cg * 32;    // [parity][group][token][quarter]
+        const float *m_s = reinterpret_cast<const float *>(smem + L::OFF_MUL) + j;
         // multipliers of this thread's elements: register 8 a + c <-> element 1024 a + 8 j + c.  K = 1024 keeps them in
-        // registers; K = 4096 re-reads them per token (they stay in L1): 32 more live registers would spill.
+        // registers; K = 4096 re-reads them per token from shared memory: 32 more live registers would spill.
         float m[8];
         if (PIECES == 1) {
             const float4 lo = __ldg(reinterpret_cast<const float4 *>(mul + 8 * j));
@@ -168,15 +182,18 @@ rsq_tc_kernel(const __grid_constant__ CUtensorMap map_x, int M, const float *__r
             m[0] = lo.x; m[1] = lo.y; m[2] = lo.z; m[3] = lo.w; m[4] = hi.x; m[5] = hi.y; m[6] = hi.z; m[7] = hi.w;
         }
         bool alive = true;
-        uint32_t toggle = 0;
-        for (int t = 0; t < my_tiles && alive; ++t) {
+        // The loop is NOT left when a wait expires: the four warps of a column group meet at a hardware barrier in
+        // every tile, so a warp whose wait gave up keeps taking part (its remaining waits return at once, the abort
+        // flag being set; what it computes is discarded by the caller, who finds the expiry in *status).
+        for (int t = 0; t < my_tiles; ++t) {
             const int tile = blockIdx.x + t * gridDim.x;
             const int b = t & 1;
             const long long row0 = (long long)tile * TOK_TILE + cg * TOK_G;         // first token of this warp's column group
-            // one thread of the column group polls; the outcome is the same for its four warps, which meet again below
-            alive = ptx::mbar_wait_group(bar_tfull + 8 * b, (t >> 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM, (threadIdx.x & 127) == 0,
-                                         1 + cg, 128, s_flags + 2 * cg, toggle, 32);
-            if (!alive) break;
+            {   // lane 0 polls, the warp follows
+                int ok = 1;
+                if (lane == 0) ok = (alive && ptx::mbar_wait(bar_tfull + 8 * b, (t >> 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM, 32)) ? 1 : 0;
+                alive = __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
+            }
             ptx::tc_fence_after_sync();
             // the warp's 32 lanes x 64 columns of the accumulator -> registers; tensor memory is handed back at once
             uint32_t raw[2][32];
@@ -197,9 +214,8 @@ rsq_tc_kernel(const __grid_constant__ CUtensorMap map_x, int M, const float *__r
 #pragma unroll
                 for (int a = 0; a < PIECES; ++a) {
                     if (PIECES > 1) {
-                        const float4 lo = __ldg(reinterpret_cast<const float4 *>(mul + 1024 * a + 8 * j));
-                        const float4 hi = __ldg(reinterpret_cast<const float4 *>(mul + 1024 * a + 8 * j + 4));
-                        m[0] = lo.x; m[1] = lo.y; m[2] = lo.z; m[3] = lo.w; m[4] = hi.x; m[5] = hi.y; m[6] = hi.z; m[7] = hi.w;
+#pragma unroll
+                        for (int r = 0; r < 8; ++r) m[r] = m_s[(8 * a + r) * 128];
                     }
 #pragma unroll
                     for (int r = 0; r < 8; r += 2) {
@@ -213,7 +229,7 @@ rsq_tc_kernel(const __grid_constant__ CUtensorMap map_x, int M, const float *__r
                 // non-negative floats order like their bit patterns: one integer warp reduction
                 const uint32_t wm = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(am));
                 if (lane == i) mine = wm;
-                if (DUMP && y_debug && row0 + i < M) {
+                if (DUMP && y_debug && alive && row0 + i < M) {
 #pragma unroll
                     for (int a = 0; a < PIECES; ++a) {
                         float4 *d = reinterpret_cast<float4 *>(y_debug + (row0 + i) * K + 1024 * a + 8 * j);
@@ -232,7 +248,7 @@ rsq_tc_kernel(const __grid_constant__ CUtensorMap map_x, int M, const float *__r
                 const float4 q4 = *reinterpret_cast<const float4 *>(ex + lane * 4);
                 const float amax = fmaxf(fmaxf(fmaxf(q4.x, q4.y), fmaxf(q4.z, q4.w)), 1e-8f);
                 inv_mine = __fdiv_rn(static_cast<float>(QMAX), amax);
-                if (quarter == 0 && row0 + lane < M) scales[row0 + lane] = __fdiv_rn(amax, static_cast<float>(QMAX));
+                if (alive && quarter == 0 && row0 + lane < M) scales[row0 + lane] = __fdiv_rn(amax, static_cast<float>(QMAX));
             }
             const uint64_t magic2 = ptx::f32x2_pack(12582912.0f, 12582912.0f);
 #pragma unroll
@@ -240,7 +256,7 @@ rsq_tc_kernel(const __grid_constant__ CUtensorMap map_x, int M, const float *__r
                 const float *y = v + VPT * i;
                 const float inv = __shfl_sync(0xFFFFFFFFu, inv_mine, i);
                 const uint64_t inv2 = ptx::f32x2_pack(inv, inv);
-                const bool row_ok = row0 + i < M;
+                const bool row_ok = alive && row0 + i < M;   // nothing is stored after an expired wait
 #pragma unroll
                 for (int a = 0; a < PIECES; ++a) {
                     // exact product + 1.5 * 2^23, rounded once (half-to-even): the low mantissa bits are the code
@@ -334,7 +350,7 @@ cudaError_t launch(const uint16_t *x, long long ldx, int M, const float *mul, un
     const int dev = qvggt_current_device();
     if (dev < 0) return cudaErrorInvalidDevice;
     if (!configured.v[dev].load(std::memory_order_acquire)) {
-        cudaError_t e = cudaFuncSetAttribute(rsq_tc_kernel<LOGK, C8, QMAX, DUMP>, cudaFuncAttributeMaxDynamicSharedMemorySize, DYN_SMEM);
+        cudaError_t e = cudaFuncSetAttribute(rsq_tc_kernel<LOGK, C8, QMAX, DUMP>, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay<PIECES>::DYN_SMEM);
         if (e != cudaSuccess) return e;
         configured.v[dev].store(1, std::memory_order_release);
     }
@@ -351,7 +367,7 @@ cudaError_t launch(const uint16_t *x, long long ldx, int M, const float *mul, un
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(tiles < sms ? tiles : sms);
     cfg.blockDim = dim3(THREADS);
-    cfg.dynamicSmemBytes = DYN_SMEM;
+    cfg.dynamicSmemBytes = Lay<PIECES>::DYN_SMEM;
     cfg.stream = st;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
