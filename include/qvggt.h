@@ -135,6 +135,20 @@ int qvggt_w4a4_linear_c8(const qvggt_weights_t *w, const signed char *Xq8, const
                          void *Y_bf16, long long ldy, int *acc_debug, void *cuda_stream);
 
 /*
+ * The one-code-per-byte GEMM for a handle that keeps ONLY the packed weight codes (flags = 0 at preparation: 0.5 bytes
+ * per weight, the paper's memory footprint, Tab. "efficiency").  A small kernel in front of the GEMM unpacks the
+ * layer's codes into w_scratch, from where the GEMM's TMA loads read them back (a few megabytes: they stay in L2), so
+ * the weights exist unpacked only transiently and only one layer at a time.  Activations as written by
+ * qvggt_rotate_smooth_quantize_c8 / _tc_c8 (which need nothing but the handle's multipliers).  Results are those of
+ * qvggt_w4a4_linear_c8 bit for bit.
+ *   w_scratch  int8 [N, K] device scratch supplied by the caller, 16-byte aligned, overwritten; one scratch may serve
+ *              every layer as long as the calls that share it are ordered on one stream
+ */
+int qvggt_w4a4_linear_c8_packed_weights(const qvggt_weights_t *w, const signed char *Xq8, const float *a_scale, int M,
+                                        void *Y_bf16, long long ldy, signed char *w_scratch, int *acc_debug,
+                                        void *cuda_stream);
+
+/*
  * The activation path with the bulk of the rotation on the tensor core (Sec. 3.2, Pre-Global-Rotation: the Kronecker
  * recursion H_{2^n} = H_2 (x) H_{2^(n-1)} lets the transform factor over any split of the index bits).  Index bits
  * 3..9 are transformed by one product with the +-1 matrix H_128 (bf16 operands: every product exact, fp32

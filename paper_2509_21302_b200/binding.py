@@ -24,7 +24,7 @@ EXPORTS = ("qvggt_prepare_weights", "qvggt_rotate_smooth_quantize", "qvggt_w4a4_
            "qvggt_weights_view_c8", "qvggt_rotate_smooth_quantize_static_c8",
            "qvggt_layernorm_rotate_smooth_quantize_c8", "qvggt_layernorm", "qvggt_debug_starved_linear_c8",
            "qvggt_rotate_smooth_quantize_tc", "qvggt_rotate_smooth_quantize_tc_c8", "qvggt_gelu",
-           "qvggt_gelu_rotate_smooth_quantize_c8")
+           "qvggt_gelu_rotate_smooth_quantize_c8", "qvggt_w4a4_linear_c8_packed_weights")
 PREP_C8 = 1   # QVGGT_PREP_C8: keep an int8 [N, K] copy of the weight codes for the *_c8 entry points
 PREP_W8A8 = 2  # QVGGT_PREP_W8A8: 8-bit codes (one per byte only)
 PREP_C8_ONLY = 4  # QVGGT_PREP_C8_ONLY: 4-bit codes one per byte only (no packed copy)
@@ -60,6 +60,7 @@ def lib() -> ctypes.CDLL:
         L.qvggt_layernorm.argtypes = [vp, i64, i32, i32, vp, vp, f32, vp, vp]
         L.qvggt_rotate_smooth_quantize_tc.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp]
         L.qvggt_rotate_smooth_quantize_tc_c8.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp]
+        L.qvggt_w4a4_linear_c8_packed_weights.argtypes = [vp, vp, vp, i32, vp, i64, vp, vp, vp]
         L.qvggt_gelu.argtypes = [vp, i64, i32, i32, vp, vp]
         L.qvggt_gelu_rotate_smooth_quantize_c8.argtypes = [vp, vp, i64, i32, vp, vp, vp]
         L.qvggt_debug_starved_linear_c8.argtypes = [vp, vp, vp, i32, vp, i64, i64, vp]
@@ -322,7 +323,7 @@ def gelu_rotate_smooth_quantize_c8(w: Weights, X: torch.Tensor, Xq8: torch.Tenso
     if a_scale is None:
         a_scale = torch.empty((M,), dtype=torch.float32, device=X.device)
     _check(lib().qvggt_gelu_rotate_smooth_quantize_c8(w.handle, _ptr(X), X.stride(0) if M > 1 else w.K, M, _ptr(Xq8), _ptr(a_scale),
-                                                      _stream()), "qvggt_gelu_rotate_smooth_quantize_c8")
+                                                      _stream()), "qvggt_gelu_rotate_smooth_quantize_c8", "qvggt_w4a4_linear_c8_packed_weights")
     return Xq8, a_scale
 
 
@@ -340,6 +341,20 @@ def w4a4_linear_c8(w: Weights, Xq8: torch.Tensor, a_scale: torch.Tensor, Y: torc
         assert acc_debug.dtype == torch.int32 and acc_debug.is_contiguous()
     _check(lib().qvggt_w4a4_linear_c8(w.handle, _ptr(Xq8), _ptr(a_scale), M, _ptr(Y), ldy, _ptr(acc_debug), _stream()),
            "qvggt_w4a4_linear_c8")
+    return Y
+
+
+def w4a4_linear_c8_packed_weights(w: Weights, Xq8: torch.Tensor, a_scale: torch.Tensor, w_scratch: torch.Tensor,
+                                  Y: torch.Tensor | None = None, acc_debug: torch.Tensor | None = None) -> torch.Tensor:
+    """The one-code-per-byte GEMM on a handle that keeps only packed weight codes; w_scratch: int8, at least N*K elements."""
+    M = Xq8.shape[0]
+    assert Xq8.dtype == torch.int8 and Xq8.is_contiguous() and Xq8.shape[1] == w.K
+    assert w_scratch.dtype == torch.int8 and w_scratch.is_contiguous() and w_scratch.numel() >= w.N * w.K
+    if Y is None:
+        Y = torch.empty((M, w.N), dtype=torch.bfloat16, device=Xq8.device)
+    ldy = Y.stride(0) if M > 1 else w.N
+    _check(lib().qvggt_w4a4_linear_c8_packed_weights(w.handle, _ptr(Xq8), _ptr(a_scale), M, _ptr(Y), ldy, _ptr(w_scratch), _ptr(acc_debug),
+                                                     _stream()), "qvggt_w4a4_linear_c8_packed_weights")
     return Y
 
 

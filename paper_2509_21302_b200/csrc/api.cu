@@ -250,6 +250,23 @@ int qvggt_w4a4_linear_c8(const qvggt_weights_t *w, const signed char *Xq8, const
     return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
 }
 
+int qvggt_w4a4_linear_c8_packed_weights(const qvggt_weights_t *w, const signed char *Xq8, const float *a_scale, int M, void *Y_bf16,
+                                        long long ldy, signed char *w_scratch, int *acc_debug, void *cuda_stream)
+{
+    if (!w) return QVGGT_ERR_NULL;
+    if (M < 0) return QVGGT_ERR_SHAPE;
+    if (!w->Wq) return QVGGT_ERR_UNSUPPORTED;
+    if (M == 0) return QVGGT_OK;
+    if (!Xq8 || !a_scale || !Y_bf16 || !w_scratch) return QVGGT_ERR_NULL;
+    if (ldy < w->N) return QVGGT_ERR_SHAPE;
+    if (ldy % 8 != 0 || !aligned16(Xq8) || !aligned16(Y_bf16) || !aligned16(w_scratch) || (acc_debug && !aligned16(acc_debug)) ||
+        (reinterpret_cast<uintptr_t>(a_scale) & 3u))
+        return QVGGT_ERR_ALIGN;
+    cudaError_t e = qvggt_launch_gemm_c8_packed_weights(w, Xq8, a_scale, M, Y_bf16, ldy, w_scratch, acc_debug, static_cast<cudaStream_t>(cuda_stream));
+    if (e == cudaErrorNotSupported) return QVGGT_ERR_UNSUPPORTED;
+    return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
+}
+
 int qvggt_debug_starved_linear_c8(const qvggt_weights_t *w, const signed char *Xq8, const float *a_scale, int M, void *Y_bf16,
                                   long long ldy, long long wait_limit_cycles, void *cuda_stream)
 {

@@ -232,8 +232,34 @@ gemm_c8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     }
 }
 
+// Packed weight codes [N, K/2] (byte i = code 2i in bits 0-3, code 2i+1 in bits 4-7, two's complement) -> one code per
+// byte [N, K], 16 packed bytes per thread.  Used when the handle keeps only the packed codes: the unpacked copy is a
+// per-launch scratch of a few megabytes that the GEMM behind it reads back from L2.
+__global__ void __launch_bounds__(256) unpack_w4_kernel(const uint4 *__restrict__ packed, uint4 *__restrict__ out, long long n16)
+{
+    ptx::grid_launch_dependents();
+    ptx::grid_dependency_wait();           // the scratch may still be read by the previous GEMM of the stream
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n16) return;
+    const uint4 p = __ldg(packed + i);
+    const uint32_t w[4] = {p.x, p.y, p.z, p.w};
+    uint32_t o[8];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t x = (w[e] >> (16 * h)) & 0xFFFFu;          // four nibbles
+            x = (x | (x << 8)) & 0x00FF00FFu;
+            x = (x | (x << 4)) & 0x0F0F0F0Fu;                    // one nibble per byte, natural order
+            o[2 * e + h] = x | ((x & 0x08080808u) * 0x1Eu);     // sign extension: bit 3 -> bits 4..7 of its byte
+        }
+    }
+    out[2 * i] = make_uint4(o[0], o[1], o[2], o[3]);
+    out[2 * i + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+}
+
 template <bool DUMP>
-cudaError_t launch(const qvggt_weights *w, const signed char *Xq8, const float *a_scale, int M, void *Y, long long ldy,
+cudaError_t launch(const qvggt_weights *w, const signed char *wq8, const signed char *Xq8, const float *a_scale, int M, void *Y, long long ldy,
                    int *acc_debug, cudaStream_t st, long long wait_limit, int skip_loads)
 {
     static QvggtPerDevice cache;
@@ -243,7 +269,7 @@ cudaError_t launch(const qvggt_weights *w, const signed char *Xq8, const float *
     const int K = w->K, N = w->N;
     CUtensorMap map_x, map_w, map_y;
     if (!qvggt_make_map(&map_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, Xq8, K, M, K, BK, BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !qvggt_make_map(&map_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, w->Wq8, K, N, K, BK, B_ROWS, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !qvggt_make_map(&map_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, wq8, K, N, K, BK, B_ROWS, CU_TENSOR_MAP_SWIZZLE_128B) ||
         !qvggt_make_map(&map_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Y, N, M, (uint64_t)ldy * 2, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B))
         return cudaErrorInvalidValue;
     const int total_tiles = ((M + 2 * BM - 1) / (2 * BM)) * ((N + BN - 1) / BN);
@@ -271,8 +297,29 @@ cudaError_t qvggt_launch_gemm_c8(const qvggt_weights *w, const signed char *Xq8,
 {
     if (M == 0) return cudaSuccess;
     if (!w->Wq8) return cudaErrorNotSupported;      // the handle was prepared without the 8-bit-container copy
-    return acc_debug ? launch<true>(w, Xq8, a_scale, M, Y, ldy, acc_debug, st, ptx::kWaitLimitCycles, 0)
-                     : launch<false>(w, Xq8, a_scale, M, Y, ldy, acc_debug, st, ptx::kWaitLimitCycles, 0);
+    return acc_debug ? launch<true>(w, w->Wq8, Xq8, a_scale, M, Y, ldy, acc_debug, st, ptx::kWaitLimitCycles, 0)
+                     : launch<false>(w, w->Wq8, Xq8, a_scale, M, Y, ldy, acc_debug, st, ptx::kWaitLimitCycles, 0);
+}
+
+cudaError_t qvggt_launch_gemm_c8_packed_weights(const qvggt_weights *w, const signed char *Xq8, const float *a_scale, int M, void *Y,
+                                                long long ldy, signed char *w_scratch, int *acc_debug, cudaStream_t st)
+{
+    if (M == 0) return cudaSuccess;
+    if (!w->Wq) return cudaErrorNotSupported;       // the handle holds no packed codes
+    const long long n16 = (long long)w->N * w->K / 32;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((n16 + 255) / 256));
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, unpack_w4_kernel, reinterpret_cast<const uint4 *>(w->Wq), reinterpret_cast<uint4 *>(w_scratch), n16);
+    if (e != cudaSuccess) return e;
+    return acc_debug ? launch<true>(w, w_scratch, Xq8, a_scale, M, Y, ldy, acc_debug, st, ptx::kWaitLimitCycles, 0)
+                     : launch<false>(w, w_scratch, Xq8, a_scale, M, Y, ldy, acc_debug, st, ptx::kWaitLimitCycles, 0);
 }
 
 cudaError_t qvggt_launch_gemm_c8_starved(const qvggt_weights *w, const signed char *Xq8, const float *a_scale, int M, void *Y,
@@ -280,5 +327,5 @@ cudaError_t qvggt_launch_gemm_c8_starved(const qvggt_weights *w, const signed ch
 {
     if (M == 0) return cudaSuccess;
     if (!w->Wq8) return cudaErrorNotSupported;
-    return launch<false>(w, Xq8, a_scale, M, Y, ldy, nullptr, st, wait_limit_cycles, 1);
+    return launch<false>(w, w->Wq8, Xq8, a_scale, M, Y, ldy, nullptr, st, wait_limit_cycles, 1);
 }

@@ -9,7 +9,10 @@
 //   - one CTA per tile of 128 tokens x 128 channels (tcgen05.mma.cta_group::1, M = 128, N = 128);
 //   - every K-block of 128 codes is one scale group: it accumulates into its own TMEM buffer (two
 //     buffers of 128 columns, ping-pong), which the epilogue warps drain while the next group runs;
-//   - an epilogue thread keeps the running sums of its row's 64 columns in registers.
+//   - the fp32 running sums live in a third region of tensor memory (128 columns): an epilogue thread reads 16 of
+//     its row's sums, adds the rescaled group sums and writes them back, so it never holds more than 32 values
+//     (64 sums in registers next to the accumulator chunk did not fit the 96 registers a thread of this 18-warp CTA
+//     may use: they spilled to local memory and the kernel ran 10 x slower).
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -51,7 +54,8 @@ struct C {
     static constexpr int OFF_FLAGS = OFF_ABORT + 4;
     static constexpr int SMEM_BYTES = OFF_FLAGS + 8 * (2 + CONV_WARPS);
     static constexpr int DYN_SMEM = SMEM_BYTES + 1024;
-    static constexpr int TMEM_COLS = ACC_BUFS * BN;                     // 256
+    static constexpr int SUM_COL = ACC_BUFS * BN;                       // first tensor-memory column of the running sums
+    static constexpr int TMEM_COLS = 512;                               // 2 accumulators + sums = 384, rounded up to a power of two
     static_assert(DYN_SMEM <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 };
 constexpr int PS = C::PS, US = C::US, PK_STAGE = C::PK_STAGE, UP_STAGE = C::UP_STAGE;
@@ -130,51 +134,62 @@ gemm_w4a4_grouped_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                 // buffer tb was last read two tiles ago; every epilogue warp has passed a group barrier since
                 gemmc::load_channel_params(s_ws + tb * BN, s_bs + tb * BN, w_scale, bias, nt0, N, threadIdx.x);
             }
-            float sum[64];
-#pragma unroll
-            for (int j = 0; j < 64; ++j) sum[j] = 0.0f;
 #pragma unroll 1
             for (int kb = 0; kb < KB; ++kb, ++it) {
                 const int b = it & 1;
+                const bool first = kb == 0, last = kb == KB - 1;
                 // a_scale / 256: exact, cancels the factor 256 carried by the raw accumulator
                 const float as = row_ok ? __fmul_rn(__ldg(a_scale + (long long)gm * KB + kb), 0.00390625f) : 0.0f;
                 alive = ptx::mbar_wait_group(bar_tfull + 8 * b, (it >> 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM,
                                              threadIdx.x == 0, 1, EPI_WARPS * 32, s_flags, toggle, 20) && alive;
                 ptx::tc_fence_after_sync();
-                if (alive) {
-#pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        uint32_t raw[32];
-                        ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + b * BN + chalf * 64 + c * 32, raw);
-                        ptx::tmem_ld_wait();
-                        if (c == 1) {
-                            ptx::tc_fence_before_sync();
-                            __syncwarp();
-                            if (lane == 0) ptx::mbar_arrive(bar_tempty + 8 * b);
-                        }
-                        // s = fl(s + fl(float(acc_g) * a_scale[m][g])): separate multiply and add
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            sum[32 * c + j] = __fadd_rn(sum[32 * c + j], __fmul_rn(static_cast<float>(static_cast<int>(raw[j])), as));
-                        if (acc_debug && row_ok) gemmc::dump_acc_x32<8>(acc_debug + ((long long)kb * M + gm) * N + n0 + c * 32, raw);
-                    }
-                }
-            }
-            if (alive) {
+                if (!alive) continue;
+                const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
                 const float *wsb = s_ws + tb * BN + chalf * 64;
                 const float *bsb = s_bs + tb * BN + chalf * 64;
+                uint32_t out[16];                     // two 16-column chunks make one 32-column staging tile
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    uint32_t out[16];
-#pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
-                        const float z0 = __fadd_rn(__fmul_rn(sum[32 * c + j], wsb[32 * c + j]), bsb[32 * c + j]);
-                        const float z1 = __fadd_rn(__fmul_rn(sum[32 * c + j + 1], wsb[32 * c + j + 1]), bsb[32 * c + j + 1]);
-                        out[j >> 1] = ptx::pack_bf16x2(z0, z1);
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t raw[16], sum[16];
+                    ptx::tmem_ld_32x16(tmem_base + lane_base + b * BN + chalf * 64 + c * 16, raw);
+                    if (!first) ptx::tmem_ld_32x16(tmem_base + lane_base + C::SUM_COL + chalf * 64 + c * 16, sum);
+                    ptx::tmem_ld_wait();
+                    if (c == 3) {
+                        // last read of this accumulator: hand it back to the MMA thread
+                        ptx::tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(bar_tempty + 8 * b);
                     }
-                    gemmc::stage_row_32(stg, out, lane);
-                    gemmc::store_staged_32x32(&map_y, stg_addr, n0 + c * 32, m0, m0 < M, lane);
+                    // s = fl(s + fl(float(acc_g) * a_scale[m][g])), g ascending: separate multiply and add
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const float p = __fmul_rn(static_cast<float>(static_cast<int>(raw[j])), as);
+                        sum[j] = __float_as_uint(__fadd_rn(first ? 0.0f : __uint_as_float(sum[j]), p));
+                    }
+                    if (acc_debug && row_ok) {
+                        uint4 *dbg = reinterpret_cast<uint4 *>(acc_debug + ((long long)kb * M + gm) * N + n0 + c * 16);
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4)
+                            dbg[q4] = make_uint4(static_cast<int>(raw[4 * q4]) >> 8, static_cast<int>(raw[4 * q4 + 1]) >> 8,
+                                                 static_cast<int>(raw[4 * q4 + 2]) >> 8, static_cast<int>(raw[4 * q4 + 3]) >> 8);
+                    }
+                    if (!last) {
+                        ptx::tmem_st_32x16(tmem_base + lane_base + C::SUM_COL + chalf * 64 + c * 16, sum);
+                    } else {
+                        // bf16( fl(fl(s * w_scale) + bias) )
+#pragma unroll
+                        for (int j = 0; j < 16; j += 2) {
+                            const float z0 = __fadd_rn(__fmul_rn(__uint_as_float(sum[j]), wsb[16 * c + j]), bsb[16 * c + j]);
+                            const float z1 = __fadd_rn(__fmul_rn(__uint_as_float(sum[j + 1]), wsb[16 * c + j + 1]), bsb[16 * c + j + 1]);
+                            out[8 * (c & 1) + (j >> 1)] = ptx::pack_bf16x2(z0, z1);
+                        }
+                        if (c & 1) {
+                            gemmc::stage_row_32(stg, out, lane);
+                            gemmc::store_staged_32x32(&map_y, stg_addr, n0 + (c >> 1) * 32, m0, m0 < M, lane);
+                        }
+                    }
                 }
+                if (!last) ptx::tmem_st_wait();       // the sums are back in tensor memory before the next group reads them
             }
         }
         if (lane == 0) ptx::tma_store_wait_all();

@@ -65,3 +65,7 @@ cudaError_t qvggt_launch_gemm_c8(const qvggt_weights *w, const signed char *Xq8,
 // out and the kernel leaves through its timeout path (exercised by the tests; nothing asynchronous is in flight).
 cudaError_t qvggt_launch_gemm_c8_starved(const qvggt_weights *w, const signed char *Xq8, const float *a_scale, int M, void *Y,
                                          long long ldy, long long wait_limit_cycles, cudaStream_t st);
+// The same GEMM for a handle that keeps only the packed weight codes: they are unpacked into w_scratch (int8 [N, K]) by a
+// small kernel in front of the GEMM.
+cudaError_t qvggt_launch_gemm_c8_packed_weights(const qvggt_weights *w, const signed char *Xq8, const float *a_scale, int M, void *Y,
+                                                long long ldy, signed char *w_scratch, int *acc_debug, cudaStream_t st);

@@ -246,3 +246,38 @@ def test_c8_only_handle_keeps_one_byte_per_weight():
     assert st == -4                                               # QVGGT_ERR_UNSUPPORTED: no packed weights in this handle
     assert h.device_status() == 0
     h.free()
+
+
+@pytest.mark.parametrize("K,N,M", [(1024, 384, 700), (4096, 128, 300), (1024, 1024, 1374)])
+def test_packed_weights_handle_on_the_one_code_per_byte_gemm(K, N, M):
+    """A handle prepared without flags keeps only the packed weight codes (0.5 bytes per weight); the one-code-per-byte GEMM
+    takes it through a caller-supplied scratch that holds the unpacked codes of one layer.  Same sums, same outputs."""
+    spec = workload.LinearSpec("pw", K, N, workload.DIST_NORMAL, 23, 0)
+    W, b, X = spec.weight(), spec.bias(), spec.x_rows(0, M)
+    c = oracle.smooth_factors(spec.x_calib(128), W)
+    ref = oracle.w4a4_linear(X, oracle.prepare_weights(W, c), b, 0)
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    h = q.prepare_weights(dev_bf16(W), dev_bf16(b), torch.from_numpy(c).cuda(), None)          # flags = 0
+    torch.cuda.synchronize()
+    taken = free0 - torch.cuda.mem_get_info()[0]
+    assert taken <= N * K // 2 + (4 << 20), "the handle should hold about half a byte per weight (plus allocation granules)"
+    assert h.view_c8() is None and h.view()["wq"].shape == (N, K // 2)
+    scratch = torch.full((N * K + 64,), 0x55, dtype=torch.int8, device="cuda")
+    Xq8, a = q.rotate_smooth_quantize_c8(h, dev_bf16(X))
+    assert np.array_equal(Xq8.cpu().numpy(), ref["xq"])
+    acc = torch.zeros((M, N), dtype=torch.int32, device="cuda")
+    Y = q.w4a4_linear_c8_packed_weights(h, Xq8, a, scratch, acc_debug=acc)
+    assert np.array_equal(scratch[:N * K].view(N, K).cpu().numpy(), ref_wq := oracle.prepare_weights(W, c)["wq"])   # the unpacked codes
+    assert np.array_equal(acc.cpu().numpy(), ref["acc"])
+    assert np.array_equal(host_bits(Y), ref["y"])
+    Y2 = q.w4a4_linear_c8_packed_weights(h, Xq8, a, scratch)                                      # production instantiation, scratch reused
+    assert torch.equal(Y2.view(torch.int16), Y.view(torch.int16))
+    assert torch.all(scratch[N * K:] == 0x55)
+    assert h.device_status() == 0
+    h.free()
+    only = q.prepare_weights(dev_bf16(W), None, torch.from_numpy(c).cuda(), None, c8="only")
+    st = q.lib().qvggt_w4a4_linear_c8_packed_weights(only.handle, Xq8.data_ptr(), a.data_ptr(), M, Y.data_ptr(), N, scratch.data_ptr(), None,
+                                                     torch.cuda.current_stream().cuda_stream)
+    assert st == -4
+    only.free()
