@@ -323,7 +323,7 @@ def gelu_rotate_smooth_quantize_c8(w: Weights, X: torch.Tensor, Xq8: torch.Tenso
     if a_scale is None:
         a_scale = torch.empty((M,), dtype=torch.float32, device=X.device)
     _check(lib().qvggt_gelu_rotate_smooth_quantize_c8(w.handle, _ptr(X), X.stride(0) if M > 1 else w.K, M, _ptr(Xq8), _ptr(a_scale),
-                                                      _stream()), "qvggt_gelu_rotate_smooth_quantize_c8", "qvggt_w4a4_linear_c8_packed_weights")
+                                                      _stream()), "qvggt_gelu_rotate_smooth_quantize_c8")
     return Xq8, a_scale
 
 
