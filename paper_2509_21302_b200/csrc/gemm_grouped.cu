@@ -134,53 +134,66 @@ gemm_w4a4_grouped_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                 // buffer tb was last read two tiles ago; every epilogue warp has passed a group barrier since
                 gemmc::load_channel_params(s_ws + tb * BN, s_bs + tb * BN, w_scale, bias, nt0, N, threadIdx.x);
             }
+            // the group's activation scale is fetched one K-block ahead: it comes from L2, several hundred cycles away
+            float as_next = row_ok ? __ldg(a_scale + (long long)gm * KB) : 0.0f;
 #pragma unroll 1
             for (int kb = 0; kb < KB; ++kb, ++it) {
                 const int b = it & 1;
                 const bool first = kb == 0, last = kb == KB - 1;
                 // a_scale / 256: exact, cancels the factor 256 carried by the raw accumulator
-                const float as = row_ok ? __fmul_rn(__ldg(a_scale + (long long)gm * KB + kb), 0.00390625f) : 0.0f;
+                const float as = __fmul_rn(as_next, 0.00390625f);
+                if (!last && row_ok) as_next = __ldg(a_scale + (long long)gm * KB + kb + 1);
+                // polled without back-off: this wait sits on the critical path of every K-block, and a sleep, however short
+                // it is asked to be, costs of the order of a microsecond
                 alive = ptx::mbar_wait_group(bar_tfull + 8 * b, (it >> 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM,
-                                             threadIdx.x == 0, 1, EPI_WARPS * 32, s_flags, toggle, 20) && alive;
+                                             threadIdx.x == 0, 1, EPI_WARPS * 32, s_flags, toggle, 0) && alive;
                 ptx::tc_fence_after_sync();
                 if (!alive) continue;
                 const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
                 const float *wsb = s_ws + tb * BN + chalf * 64;
                 const float *bsb = s_bs + tb * BN + chalf * 64;
                 uint32_t out[16];                     // two 16-column chunks make one 32-column staging tile
+                // the loads of chunk c + 1 are in flight while chunk c is rescaled (tcgen05.wait::ld waits for every load
+                // issued so far, so the next chunk's loads go out right behind the wait)
+                uint32_t raw[2][16], sum[2][16];
+                const uint32_t acc_addr = tmem_base + lane_base + b * BN + chalf * 64, sum_addr = tmem_base + lane_base + C::SUM_COL + chalf * 64;
+                ptx::tmem_ld_32x16(acc_addr, raw[0]);
+                if (!first) ptx::tmem_ld_32x16(sum_addr, sum[0]);
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    uint32_t raw[16], sum[16];
-                    ptx::tmem_ld_32x16(tmem_base + lane_base + b * BN + chalf * 64 + c * 16, raw);
-                    if (!first) ptx::tmem_ld_32x16(tmem_base + lane_base + C::SUM_COL + chalf * 64 + c * 16, sum);
                     ptx::tmem_ld_wait();
-                    if (c == 3) {
+                    if (c < 3) {
+                        ptx::tmem_ld_32x16(acc_addr + (c + 1) * 16, raw[(c + 1) & 1]);
+                        if (!first) ptx::tmem_ld_32x16(sum_addr + (c + 1) * 16, sum[(c + 1) & 1]);
+                    } else {
                         // last read of this accumulator: hand it back to the MMA thread
                         ptx::tc_fence_before_sync();
                         __syncwarp();
                         if (lane == 0) ptx::mbar_arrive(bar_tempty + 8 * b);
                     }
+                    uint32_t (&r)[16] = raw[c & 1];
+                    uint32_t (&sm)[16] = sum[c & 1];
                     // s = fl(s + fl(float(acc_g) * a_scale[m][g])), g ascending: separate multiply and add
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
-                        const float p = __fmul_rn(static_cast<float>(static_cast<int>(raw[j])), as);
-                        sum[j] = __float_as_uint(__fadd_rn(first ? 0.0f : __uint_as_float(sum[j]), p));
+                        const float p = __fmul_rn(static_cast<float>(static_cast<int>(r[j])), as);
+                        sm[j] = __float_as_uint(__fadd_rn(first ? 0.0f : __uint_as_float(sm[j]), p));
                     }
                     if (acc_debug && row_ok) {
                         uint4 *dbg = reinterpret_cast<uint4 *>(acc_debug + ((long long)kb * M + gm) * N + n0 + c * 16);
 #pragma unroll
                         for (int q4 = 0; q4 < 4; ++q4)
-                            dbg[q4] = make_uint4(static_cast<int>(raw[4 * q4]) >> 8, static_cast<int>(raw[4 * q4 + 1]) >> 8,
-                                                 static_cast<int>(raw[4 * q4 + 2]) >> 8, static_cast<int>(raw[4 * q4 + 3]) >> 8);
+                            dbg[q4] = make_uint4(static_cast<int>(r[4 * q4]) >> 8, static_cast<int>(r[4 * q4 + 1]) >> 8,
+                                                 static_cast<int>(r[4 * q4 + 2]) >> 8, static_cast<int>(r[4 * q4 + 3]) >> 8);
                     }
                     if (!last) {
-                        ptx::tmem_st_32x16(tmem_base + lane_base + C::SUM_COL + chalf * 64 + c * 16, sum);
+                        ptx::tmem_st_32x16(sum_addr + c * 16, sm);
                     } else {
                         // bf16( fl(fl(s * w_scale) + bias) )
 #pragma unroll
                         for (int j = 0; j < 16; j += 2) {
-                            const float z0 = __fadd_rn(__fmul_rn(__uint_as_float(sum[j]), wsb[16 * c + j]), bsb[16 * c + j]);
-                            const float z1 = __fadd_rn(__fmul_rn(__uint_as_float(sum[j + 1]), wsb[16 * c + j + 1]), bsb[16 * c + j + 1]);
+                            const float z0 = __fadd_rn(__fmul_rn(__uint_as_float(sm[j]), wsb[16 * c + j]), bsb[16 * c + j]);
+                            const float z1 = __fadd_rn(__fmul_rn(__uint_as_float(sm[j + 1]), wsb[16 * c + j + 1]), bsb[16 * c + j + 1]);
                             out[8 * (c & 1) + (j >> 1)] = ptx::pack_bf16x2(z0, z1);
                         }
                         if (c & 1) {
