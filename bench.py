@@ -696,7 +696,8 @@ def measure_scene(q, torch, peaks, reps=5):
         ops = layer_ops(M, s)
         variants = (("per_token_c8", lambda: q.rotate_smooth_quantize_c8(h, x, xq8, a), lambda: q.w4a4_linear_c8(h, xq8, a, y), 1),
                     ("per_token_packed", lambda: q.rotate_smooth_quantize(h, x, 0, xq4, a), lambda: q.w4a4_linear(h, xq4, a, 0, y), 1),
-                    ("group128_packed", lambda: q.rotate_smooth_quantize(h, x, 128, xq4, ag), lambda: q.w4a4_linear(h, xq4, ag, 128, y), s.K // 128))
+                    ("group128_packed", lambda: q.rotate_smooth_quantize(h, x, 128, xq4, ag), lambda: q.w4a4_linear(h, xq4, ag, 128, y), s.K // 128),
+                    ("group128_c8", lambda: q.rotate_smooth_quantize_c8_grouped(h, x, xq8, ag), lambda: q.w4a4_linear_c8_grouped(h, xq8, ag, y), s.K // 128))
         for name, rsq, gemm, groups in variants:
             for fn in (rsq, gemm):
                 for _ in range(2):

@@ -135,6 +135,17 @@ int qvggt_w4a4_linear_c8(const qvggt_weights_t *w, const signed char *Xq8, const
                          void *Y_bf16, long long ldy, int *acc_debug, void *cuda_stream);
 
 /*
+ * Group-wise activation scales (group = 128, see qvggt_rotate_smooth_quantize / qvggt_w4a4_linear) on codes held one per byte:
+ * the same codes, scales, integer partial sums and outputs as the packed entry points with group = 128, bit for bit, on the
+ * TMA-fed GEMM (about 4 x faster than the packed group-wise GEMM).  4-bit codes only; the handle needs QVGGT_PREP_C8[_ONLY].
+ *   Xq8      int8 [M, K];  a_scale fp32 [M, K/128];  acc_debug NULL or int32 [K/128, M, N]
+ */
+int qvggt_rotate_smooth_quantize_c8_grouped(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M,
+                                            signed char *Xq8, float *a_scale, void *cuda_stream);
+int qvggt_w4a4_linear_c8_grouped(const qvggt_weights_t *w, const signed char *Xq8, const float *a_scale, int M,
+                                 void *Y_bf16, long long ldy, int *acc_debug, void *cuda_stream);
+
+/*
  * The one-code-per-byte GEMM for a handle that keeps ONLY the packed weight codes (flags = 0 at preparation: 0.5 bytes
  * per weight, the paper's memory footprint, Tab. "efficiency").  A small kernel in front of the GEMM unpacks the
  * layer's codes into w_scratch, from where the GEMM's TMA loads read them back (a few megabytes: they stay in L2), so

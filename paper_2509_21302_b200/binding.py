@@ -24,7 +24,8 @@ EXPORTS = ("qvggt_prepare_weights", "qvggt_rotate_smooth_quantize", "qvggt_w4a4_
            "qvggt_weights_view_c8", "qvggt_rotate_smooth_quantize_static_c8",
            "qvggt_layernorm_rotate_smooth_quantize_c8", "qvggt_layernorm", "qvggt_debug_starved_linear_c8",
            "qvggt_rotate_smooth_quantize_tc", "qvggt_rotate_smooth_quantize_tc_c8", "qvggt_gelu",
-           "qvggt_gelu_rotate_smooth_quantize_c8", "qvggt_w4a4_linear_c8_packed_weights")
+           "qvggt_gelu_rotate_smooth_quantize_c8", "qvggt_w4a4_linear_c8_packed_weights",
+           "qvggt_rotate_smooth_quantize_c8_grouped", "qvggt_w4a4_linear_c8_grouped")
 PREP_C8 = 1   # QVGGT_PREP_C8: keep an int8 [N, K] copy of the weight codes for the *_c8 entry points
 PREP_W8A8 = 2  # QVGGT_PREP_W8A8: 8-bit codes (one per byte only)
 PREP_C8_ONLY = 4  # QVGGT_PREP_C8_ONLY: 4-bit codes one per byte only (no packed copy)
@@ -61,6 +62,8 @@ def lib() -> ctypes.CDLL:
         L.qvggt_rotate_smooth_quantize_tc.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp]
         L.qvggt_rotate_smooth_quantize_tc_c8.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp]
         L.qvggt_w4a4_linear_c8_packed_weights.argtypes = [vp, vp, vp, i32, vp, i64, vp, vp, vp]
+        L.qvggt_rotate_smooth_quantize_c8_grouped.argtypes = [vp, vp, i64, i32, vp, vp, vp]
+        L.qvggt_w4a4_linear_c8_grouped.argtypes = [vp, vp, vp, i32, vp, i64, vp, vp]
         L.qvggt_gelu.argtypes = [vp, i64, i32, i32, vp, vp]
         L.qvggt_gelu_rotate_smooth_quantize_c8.argtypes = [vp, vp, i64, i32, vp, vp, vp]
         L.qvggt_debug_starved_linear_c8.argtypes = [vp, vp, vp, i32, vp, i64, i64, vp]
@@ -300,6 +303,33 @@ def layernorm(X: torch.Tensor, gamma: torch.Tensor, beta: torch.Tensor, eps: flo
     assert Y.is_contiguous() and Y.element_size() == 2
     ldx = X.stride(0) if M > 1 else K
     _check(lib().qvggt_layernorm(_ptr(X), ldx, M, K, _ptr(gamma), _ptr(beta), eps, _ptr(Y), _stream()), "qvggt_layernorm")
+    return Y
+
+
+def rotate_smooth_quantize_c8_grouped(w: Weights, X: torch.Tensor, Xq8: torch.Tensor | None = None, a_scale: torch.Tensor | None = None):
+    """One scale per token per 128 rotated channels, codes one per byte -> (Xq8 [M,K] int8, a_scale fp32 [M, K/128])."""
+    assert X.dim() == 2 and X.element_size() == 2 and X.stride(1) == 1 and X.shape[1] == w.K
+    M = X.shape[0]
+    if Xq8 is None:
+        Xq8 = torch.empty((M, w.K), dtype=torch.int8, device=X.device)
+    if a_scale is None:
+        a_scale = torch.empty((M, w.K // 128), dtype=torch.float32, device=X.device)
+    _check(lib().qvggt_rotate_smooth_quantize_c8_grouped(w.handle, _ptr(X), X.stride(0) if M > 1 else w.K, M, _ptr(Xq8), _ptr(a_scale),
+                                                         _stream()), "qvggt_rotate_smooth_quantize_c8_grouped")
+    return Xq8, a_scale
+
+
+def w4a4_linear_c8_grouped(w: Weights, Xq8: torch.Tensor, a_scale: torch.Tensor, Y: torch.Tensor | None = None,
+                           acc_debug: torch.Tensor | None = None) -> torch.Tensor:
+    """-> Y [M,N] bf16 from one-code-per-byte codes with group-128 scales; acc_debug: optional int32 [K/128, M, N]."""
+    M = Xq8.shape[0]
+    assert Xq8.dtype == torch.int8 and Xq8.is_contiguous() and Xq8.shape[1] == w.K
+    assert a_scale.dtype == torch.float32 and a_scale.is_contiguous() and a_scale.shape == (M, w.K // 128)
+    if Y is None:
+        Y = torch.empty((M, w.N), dtype=torch.bfloat16, device=Xq8.device)
+    ldy = Y.stride(0) if M > 1 else w.N
+    _check(lib().qvggt_w4a4_linear_c8_grouped(w.handle, _ptr(Xq8), _ptr(a_scale), M, _ptr(Y), ldy, _ptr(acc_debug), _stream()),
+           "qvggt_w4a4_linear_c8_grouped")
     return Y
 
 

@@ -232,6 +232,241 @@ gemm_c8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// The same TMA-fed CTA-pair design for one activation scale per token per 128 rotated channels (an extension of the
+// paper's token-wise granularity; the weights keep one scale per output channel).  A K-block of 128 codes is one scale
+// group, so every K-block accumulates into its own tensor-memory buffer (two of 128 columns, ping-pong) and the
+// epilogue warps rescale it while the next one runs:
+//   s = fl(s + fl(float(acc_g) * a_scale[m][g])), g ascending;  Y = bf16(fl(fl(s * w_scale[n]) + bias[n])).
+// Tile 256 tokens x 128 channels per pair; an epilogue thread keeps the 64 running sums of its row in registers (10
+// warps per CTA leave 168 registers per thread).  Per K-block the pair does 376 cycles of MMA work (four N = 128
+// instructions) against 3 instructions per output element in the epilogue: the epilogue sets the pace.
+namespace grp {
+
+constexpr int GN = 128;                                // channels per tile
+constexpr int GEPI = 16;                               // epilogue warps: lane quarter w % 4, 32-column part w / 4 (four per scheduler: the
+                                                       // epilogue is latency-bound, cf. 1400 against 2400 cycles per K-block with eight)
+constexpr int G_MMA_WARP = GEPI, G_TMA_WARP = GEPI + 1;
+constexpr int GTHREADS = (GEPI + 2) * 32;
+constexpr int GB_ROWS = GN / 2;                        // weight rows staged by one CTA
+constexpr int GSTAGE = (BM + GB_ROWS) * BK;            // 24 KB
+constexpr int GSTAGES = 7;
+constexpr int OFF_STG = GSTAGES * GSTAGE;
+constexpr int OFF_CH = OFF_STG + GEPI * STG_BYTES;          // [2][GN] channel scales, [2][GN] bias, fp32
+constexpr int OFF_BAR = OFF_CH + 2 * 2 * GN * 4;                 // full[GSTAGES] empty[GSTAGES] tfull[2] tempty[2]
+constexpr int NBARS = 2 * GSTAGES + 2 * ACC_BUFS;
+constexpr int OFF_TMEM = OFF_BAR + NBARS * 8;
+constexpr int OFF_ABORT = OFF_TMEM + 4;
+constexpr int OFF_FLAGS = OFF_ABORT + 4;
+constexpr int DYN_SMEM = OFF_FLAGS + 8 + 1024;
+constexpr int TMEM_COLS = ACC_BUFS * GN;                          // 256
+static_assert(DYN_SMEM <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
+static_assert(GSTAGE % 1024 == 0, "operand tiles must stay 1024-byte aligned");
+
+template <bool DUMP>
+__global__ void __launch_bounds__(GTHREADS, 1)
+gemm_c8_grouped_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                       const __grid_constant__ CUtensorMap map_y, const float *__restrict__ a_scale,
+                       const float *__restrict__ w_scale, const uint16_t *__restrict__ bias, int *__restrict__ acc_debug,
+                       int M, int N, int K, int *status)
+{
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = ptx::smem_addr(smem);
+    const uint32_t bar_full = sbase + OFF_BAR;
+    const uint32_t bar_empty = bar_full + GSTAGES * 8;
+    const uint32_t bar_tfull = bar_empty + GSTAGES * 8;
+    const uint32_t bar_tempty = bar_tfull + ACC_BUFS * 8;
+    uint32_t *s_tmem = reinterpret_cast<uint32_t *>(smem + OFF_TMEM);
+    volatile int *s_abort = reinterpret_cast<volatile int *>(smem + OFF_ABORT);
+    volatile int *s_flags = reinterpret_cast<volatile int *>(smem + OFF_FLAGS);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_ctarank();
+    const int worker = blockIdx.x / 2, workers = gridDim.x / 2;
+    const int KB = K / BK;                                   // = number of scale groups
+    const int n_tiles = N / GN;
+    const int total_tiles = ((M + 2 * BM - 1) / (2 * BM)) * n_tiles;
+    const int my_tiles = (total_tiles > worker) ? (total_tiles - 1 - worker) / workers + 1 : 0;
+
+    if (threadIdx.x == 0) {
+        gemmc::init_barriers(bar_full, GSTAGES, 1);
+        gemmc::init_barriers(bar_empty, GSTAGES, 1);
+        gemmc::init_barriers(bar_tfull, ACC_BUFS, 1);
+        gemmc::init_barriers(bar_tempty, ACC_BUFS, GEPI * 2);
+        *s_abort = 0;
+        ptx::fence_mbar_init();
+    }
+    if (warp == G_MMA_WARP) { ptx::tmem_alloc_pair(ptx::smem_addr(s_tmem), TMEM_COLS); ptx::tmem_relinquish_pair(); }
+    if (warp == G_TMA_WARP && lane == 0) {
+        ptx::prefetch_tensormap(&map_x);
+        ptx::prefetch_tensormap(&map_w);
+        ptx::prefetch_tensormap(&map_y);
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::cluster_sync();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *s_tmem;
+    ptx::grid_launch_dependents();
+    ptx::grid_dependency_wait();
+
+    if (warp < GEPI) {
+        // ------------------------------------------------------------ epilogue
+        const int quarter = warp & 3, cpart = warp >> 2;   // TMEM lane quarter, 32-column part
+        unsigned char *stg = smem + OFF_STG + warp * STG_BYTES;
+        const uint32_t stg_addr = sbase + OFF_STG + warp * STG_BYTES;
+        float *s_ws = reinterpret_cast<float *>(smem + OFF_CH);    // [2][GN]
+        float *s_bs = s_ws + 2 * GN;                                // [2][GN]
+        const uint32_t leader_tempty = ptx::map_to_cta(bar_tempty, 0);
+        const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
+        bool alive = true;
+        uint32_t toggle = 0;
+        int it = 0;                                                 // K-blocks seen so far (all tiles)
+        for (int t = 0; t < my_tiles; ++t) {
+            const int tile = worker + t * workers;
+            const int m0 = (tile / n_tiles) * (2 * BM) + (int)rank * BM + quarter * 32;
+            const int nt0 = (tile % n_tiles) * GN;
+            const int n0 = nt0 + cpart * 32;
+            const int tb = t & 1;
+            const int gm = m0 + lane;
+            const bool row_ok = gm < M;
+            // buffer tb was last read two tiles ago; every epilogue warp has passed a group barrier since
+            if (threadIdx.x < GN) gemmc::load_channel_params(s_ws + tb * GN, s_bs + tb * GN, w_scale, bias, nt0, N, threadIdx.x);
+            float sum[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) sum[j] = 0.0f;
+            // the group's scale is fetched one K-block ahead (it comes from L2)
+            float as_next = row_ok ? __ldg(a_scale + (long long)gm * KB) : 0.0f;
+#pragma unroll 1
+            for (int kb = 0; kb < KB; ++kb, ++it) {
+                const int b = it & 1;
+                const float as = as_next;
+                if (kb + 1 < KB && row_ok) as_next = __ldg(a_scale + (long long)gm * KB + kb + 1);
+                alive = ptx::mbar_wait_group(bar_tfull + 8 * b, (it >> 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM,
+                                             threadIdx.x == 0, 1, GEPI * 32, s_flags, toggle, 0) && alive;
+                ptx::tc_fence_after_sync();
+                if (!alive) continue;
+                uint32_t raw[32];
+                ptx::tmem_ld_32x32(tmem_base + lane_base + b * GN + cpart * 32, raw);
+                ptx::tmem_ld_wait();
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive_cluster(leader_tempty + 8 * b);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) sum[j] = __fadd_rn(sum[j], __fmul_rn(static_cast<float>(static_cast<int>(raw[j])), as));
+                if (DUMP && acc_debug && row_ok) gemmc::dump_acc_x32<0>(acc_debug + ((long long)kb * M + gm) * N + n0, raw);
+            }
+            if (alive) {
+                const float *wsb = s_ws + tb * GN + cpart * 32;
+                const float *bsb = s_bs + tb * GN + cpart * 32;
+                uint32_t out[16];
+#pragma unroll
+                for (int j = 0; j < 32; j += 2) {
+                    const float z0 = __fadd_rn(__fmul_rn(sum[j], wsb[j]), bsb[j]);
+                    const float z1 = __fadd_rn(__fmul_rn(sum[j + 1], wsb[j + 1]), bsb[j + 1]);
+                    out[j >> 1] = ptx::pack_bf16x2(z0, z1);
+                }
+                gemmc::stage_row_32(stg, out, lane);
+                gemmc::store_staged_32x32(&map_y, stg_addr, n0, m0, m0 < M, lane);
+            }
+        }
+        if (lane == 0) ptx::tma_store_wait_read<0>();
+    } else if (warp == G_MMA_WARP) {
+        // ------------------------------------------------------------ MMA issuer: one accumulator per K-block
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = ptx::idesc_i8(2 * BM, GN);
+            bool alive = true;
+            Ring r;
+            const int total_kb = my_tiles * KB;
+            for (int it = 0; it < total_kb && alive; ++it) {
+                const int b = it & 1;
+                if (it >= ACC_BUFS) {
+                    alive = ptx::mbar_wait_cluster(bar_tempty + 8 * b, ((it >> 1) - 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_TMEM_FREE);
+                    if (!alive) break;
+                    ptx::tc_fence_after_sync();
+                }
+                alive = ptx::mbar_wait_cluster(bar_full + 8 * r.s, r.ph, s_abort, status, QVGGT_DEV_TIMEOUT_FULL);
+                if (!alive) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t a_addr = sbase + r.s * GSTAGE;
+                gemmc::mma_kblock_i8<true>(tmem_base + b * GN, a_addr, a_addr + BM * BK, idesc, true);
+                ptx::mma_commit_pair(bar_empty + 8 * r.s, 3);
+                ptx::mma_commit_pair(bar_tfull + 8 * b, 3);
+                r.advance(GSTAGES);
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------ TMA producer (one thread per CTA)
+        if (lane == 0) {
+            const uint32_t leader_full = ptx::map_to_cta(bar_full, 0);
+            bool alive = true;
+            Ring r;
+            int it = 0;
+            for (int t = 0; t < my_tiles && alive; ++t) {
+                const int tile = worker + t * workers;
+                const int m0 = (tile / n_tiles) * (2 * BM) + (int)rank * BM;
+                const int n0 = (tile % n_tiles) * GN + (int)rank * GB_ROWS;
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    if (it >= GSTAGES) {
+                        alive = ptx::mbar_wait(bar_empty + 8 * r.s, r.ph ^ 1, s_abort, status, QVGGT_DEV_TIMEOUT_EMPTY, 20);
+                        if (!alive) break;
+                    }
+                    const uint32_t dst = sbase + r.s * GSTAGE;
+                    if (rank == 0) ptx::mbar_arrive_expect_tx(bar_full + 8 * r.s, 2 * GSTAGE);
+                    ptx::tma_load_2d_pair(&map_x, leader_full + 8 * r.s, dst, kb * BK, m0);
+                    ptx::tma_load_2d_pair(&map_w, leader_full + 8 * r.s, dst + BM * BK, kb * BK, n0);
+                    r.advance(GSTAGES);
+                }
+            }
+        }
+        __syncwarp();
+    }
+
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::cluster_sync();
+    if (warp == G_MMA_WARP) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc_pair(tmem_base, TMEM_COLS);
+    }
+}
+
+template <bool DUMP>
+cudaError_t launch(const qvggt_weights *w, const signed char *Xq8, const float *a_scale, int M, void *Y, long long ldy,
+                   int *acc_debug, cudaStream_t st)
+{
+    static QvggtPerDevice cache;
+    int max_workers = 0;
+    cudaError_t e = qvggt_configure_kernel(gemm_c8_grouped_kernel<DUMP>, GTHREADS, DYN_SMEM, 2, cache, &max_workers);
+    if (e != cudaSuccess) return e;
+    const int K = w->K, N = w->N;
+    CUtensorMap map_x, map_w, map_y;
+    if (!qvggt_make_map(&map_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, Xq8, K, M, K, BK, BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !qvggt_make_map(&map_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, w->Wq8, K, N, K, BK, GB_ROWS, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !qvggt_make_map(&map_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Y, N, M, (uint64_t)ldy * 2, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+        return cudaErrorInvalidValue;
+    const int total_tiles = ((M + 2 * BM - 1) / (2 * BM)) * (N / GN);
+    const int workers = total_tiles < max_workers ? total_tiles : max_workers;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(workers * 2);
+    cfg.blockDim = dim3(GTHREADS);
+    cfg.dynamicSmemBytes = DYN_SMEM;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, gemm_c8_grouped_kernel<DUMP>, map_x, map_w, map_y, a_scale, (const float *)w->w_scale,
+                              (const uint16_t *)w->bias, acc_debug, M, N, K, w->status);
+}
+
+}  // namespace grp
+
 // Packed weight codes [N, K/2] (byte i = code 2i in bits 0-3, code 2i+1 in bits 4-7, two's complement) -> one code per
 // byte [N, K], 16 packed bytes per thread.  Used when the handle keeps only the packed codes: the unpacked copy is a
 // per-launch scratch of a few megabytes that the GEMM behind it reads back from L2.
@@ -328,4 +563,12 @@ cudaError_t qvggt_launch_gemm_c8_starved(const qvggt_weights *w, const signed ch
     if (M == 0) return cudaSuccess;
     if (!w->Wq8) return cudaErrorNotSupported;
     return launch<false>(w, w->Wq8, Xq8, a_scale, M, Y, ldy, nullptr, st, wait_limit_cycles, 1);
+}
+
+cudaError_t qvggt_launch_gemm_c8_grouped(const qvggt_weights *w, const signed char *Xq8, const float *a_scale, int M, void *Y,
+                                         long long ldy, int *acc_debug, cudaStream_t st)
+{
+    if (M == 0) return cudaSuccess;
+    if (!w->Wq8 || w->bits != 4) return cudaErrorNotSupported;
+    return acc_debug ? grp::launch<true>(w, Xq8, a_scale, M, Y, ldy, acc_debug, st) : grp::launch<false>(w, Xq8, a_scale, M, Y, ldy, acc_debug, st);
 }

@@ -454,25 +454,37 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
             for (int g = 0; g < NG; ++g) am[g] = fmaxf(red[g], red[NG + g]);
         }
         if constexpr (C8) {
-            static_assert(!C8 || GROUP == 0, "byte output is built for per-token scales");
             static_assert(QMAX == 7 || QMAX == 127, "4-bit or 8-bit codes");
             float inv;
             if (STATIC) {
                 inv = __fdiv_rn(1.0f, delta);
                 am[0] = __fmul_rn(delta, static_cast<float>(QMAX));     // the scale written below is am / QMAX = delta
             } else {
-                am[0] = fmaxf(am[0], 1e-8f);
+#pragma unroll
+                for (int g = 0; g < NG; ++g) am[g] = fmaxf(am[g], 1e-8f);
                 inv = __fdiv_rn(static_cast<float>(QMAX), am[0]);
             }
-            const uint64_t inv2 = ptx::f32x2_pack(inv, inv), magic2 = ptx::f32x2_pack(12582912.0f, 12582912.0f);
+            uint64_t inv2 = ptx::f32x2_pack(inv, inv), inv2b = inv2;
+            const uint64_t magic2 = ptx::f32x2_pack(12582912.0f, 12582912.0f);
             // byte exchange between the 4 lanes that share (t / 4): a 4 x 4 byte transpose in two steps
             const uint32_t sel0 = (lane & 1) ? 0x3715u : 0x6240u, sel1 = (lane & 2) ? 0x3276u : 0x5410u;
 #pragma unroll
             for (int kk = 0; kk < T / 4; ++kk) {
+                if constexpr (GROUP == 128) {
+                    // registers 4 kk .. 4 kk + 3 lie in one scale group (T = 32: GREGS = 4) or in two (T = 64: GREGS = 2)
+                    const int g0 = (4 * kk) / GREGS, g1 = (4 * kk + 2) / GREGS;   // compile-time after unrolling
+                    const float i0 = __fdiv_rn(static_cast<float>(QMAX), am[(4 * kk) / GREGS]);
+                    inv2 = ptx::f32x2_pack(i0, i0);
+                    inv2b = inv2;
+                    if (g1 != g0) {
+                        const float i1 = __fdiv_rn(static_cast<float>(QMAX), am[(4 * kk + 2) / GREGS]);
+                        inv2b = ptx::f32x2_pack(i1, i1);
+                    }
+                }
                 // exact product + 1.5*2^23, rounded once (half-to-even): the low mantissa byte is the int8 code
                 float f0, f1, f2, f3;
                 ptx::f32x2_unpack(ptx::f32x2_fma(ptx::f32x2_pack(v[4 * kk], v[4 * kk + 1]), inv2, magic2), f0, f1);
-                ptx::f32x2_unpack(ptx::f32x2_fma(ptx::f32x2_pack(v[4 * kk + 2], v[4 * kk + 3]), inv2, magic2), f2, f3);
+                ptx::f32x2_unpack(ptx::f32x2_fma(ptx::f32x2_pack(v[4 * kk + 2], v[4 * kk + 3]), inv2b, magic2), f2, f3);
                 if (STATIC) {
                     // The clamp of Eq. "quantization", taken on the sum with the magic number: inside +-2^22 that sum is
                     // 1.5 * 2^23 + q exactly; beyond, the fused operation still returns the correctly rounded (huge) sum,
@@ -633,11 +645,15 @@ cudaError_t launch_sq(const uint16_t *x, long long ldx, int M, const float *mul,
 }  // namespace
 
 cudaError_t qvggt_launch_rsq_c8(const void *X, long long ldx, int M, int K, const float *mul, int bits, signed char *Xq8,
-                                float *scales, cudaStream_t st)
+                                float *scales, cudaStream_t st, int group)
 {
     if (M == 0) return cudaSuccess;
     const uint16_t *x = static_cast<const uint16_t *>(X);
     unsigned char *out = reinterpret_cast<unsigned char *>(Xq8);
+    if (group == 128) {
+        if (bits != 4) return cudaErrorNotSupported;
+        return K == 1024 ? launch_sq<5, 128, true>(x, ldx, M, mul, out, scales, st) : launch_sq<6, 128, true>(x, ldx, M, mul, out, scales, st);
+    }
     if (bits == 8)
         return K == 1024 ? launch_sq<5, 0, true, 127>(x, ldx, M, mul, out, scales, st) : launch_sq<6, 0, true, 127>(x, ldx, M, mul, out, scales, st);
     return K == 1024 ? launch_sq<5, 0, true>(x, ldx, M, mul, out, scales, st) : launch_sq<6, 0, true>(x, ldx, M, mul, out, scales, st);

@@ -281,3 +281,27 @@ def test_packed_weights_handle_on_the_one_code_per_byte_gemm(K, N, M):
                                                      torch.cuda.current_stream().cuda_stream)
     assert st == -4
     only.free()
+
+
+@pytest.mark.parametrize("K,N,M", [(1024, 128, 1), (1024, 384, 257), (4096, 256, 300), (4096, 128, 1374)])
+def test_c8_grouped_matches_the_oracle_and_the_packed_grouped_path(K, N, M):
+    """Group-128 activation scales on codes held one per byte: codes, scales, per-group integer sums bit-exact against the
+    oracle, outputs bit-equal, and identical to the packed group-wise entry points."""
+    spec = workload.LinearSpec("g8", K, N, workload.DIST_NORMAL, 29, 0)
+    W, b, X = spec.weight(), spec.bias(), spec.x_rows(0, M)
+    c = oracle.smooth_factors(spec.x_calib(128), W)
+    prep = oracle.prepare_weights(W, c)
+    ref = oracle.w4a4_linear(X, prep, b, 128)
+    h = q.prepare_weights(dev_bf16(W), dev_bf16(b), torch.from_numpy(c).cuda(), None, c8=True)
+    Xq8, a = q.rotate_smooth_quantize_c8_grouped(h, dev_bf16(X))
+    assert np.array_equal(Xq8.cpu().numpy(), ref["xq"]) and np.array_equal(a.cpu().numpy(), ref["a_scale"])
+    acc = torch.full((K // 128, M, N), -7, dtype=torch.int32, device="cuda")
+    Y = q.w4a4_linear_c8_grouped(h, Xq8, a, acc_debug=acc)
+    assert np.array_equal(acc.cpu().numpy(), ref["acc"])
+    assert np.array_equal(host_bits(Y), ref["y"])
+    Y2 = q.w4a4_linear_c8_grouped(h, Xq8, a)
+    assert torch.equal(Y2.view(torch.int16), Y.view(torch.int16))
+    Xq, a4 = q.rotate_smooth_quantize(h, dev_bf16(X), 128)
+    assert torch.equal(a4, a) and torch.equal(q.w4a4_linear(h, Xq, a4, 128).view(torch.int16), Y.view(torch.int16))
+    assert h.device_status() == 0
+    h.free()

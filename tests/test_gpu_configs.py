@@ -54,8 +54,7 @@ def run_layer(spec, M, rows="all", group=0, fmt="packed", X=None, check_gemm=Tru
         X = spec.x_rows(0, M)
     Xd = dev_bf16(X)
     if fmt == "c8":
-        assert group == 0
-        Xq, a_scale = q.rotate_smooth_quantize_c8(h, Xd)
+        Xq, a_scale = q.rotate_smooth_quantize_c8_grouped(h, Xd) if group else q.rotate_smooth_quantize_c8(h, Xd)
     else:
         Xq, a_scale = q.rotate_smooth_quantize(h, Xd, group)
     del Xd
@@ -74,8 +73,11 @@ def run_layer(spec, M, rows="all", group=0, fmt="packed", X=None, check_gemm=Tru
     assert torch.equal(pick(a_scale), torch.from_numpy(scales).cuda()), f"{spec.name}: scales differ from the oracle"
     del want_codes
     if check_gemm:
-        lin = (lambda acc: q.w4a4_linear_c8(h, Xq, a_scale, acc_debug=acc)) if fmt == "c8" else \
-              (lambda acc: q.w4a4_linear(h, Xq, a_scale, group, acc_debug=acc))
+        if fmt == "c8":
+            lin = (lambda acc: q.w4a4_linear_c8_grouped(h, Xq, a_scale, acc_debug=acc)) if group else \
+                  (lambda acc: q.w4a4_linear_c8(h, Xq, a_scale, acc_debug=acc))
+        else:
+            lin = lambda acc: q.w4a4_linear(h, Xq, a_scale, group, acc_debug=acc)
         Y = lin(None)
         acc = oracle.gemm_i32(codes, prep["wq"], group)
         want = oracle.epilogue(acc, scales, prep["w_scale"], b)
@@ -113,9 +115,11 @@ def test_config2_block_linears_8_frames_every_row(which, fmt):
     assert run_layer(spec, 8 * F, fmt=fmt, check_acc=which in (0, 3)) == 8 * F
 
 
-def test_config2_group128_every_row_with_integer_sums():
-    spec = workload.block_specs(0, 0)[1]
-    assert run_layer(spec, 8 * F, group=128, check_acc=True) == 8 * F
+@pytest.mark.parametrize("fmt", ["packed", "c8"])
+@pytest.mark.parametrize("which", [1, 3])
+def test_config2_group128_every_row_with_integer_sums(which, fmt):
+    spec = workload.block_specs(0, 0)[which]
+    assert run_layer(spec, 8 * F, group=128, fmt=fmt, check_acc=(which == 1)) == 8 * F
 
 
 # ------------------------------------------------------------------------------ config 3: quantize kernel sweep, every row
@@ -149,6 +153,8 @@ def test_config4_stack_blocks_32_frames(block, fmt):
     (3, 0, "packed", "all", False),    # fc2 whole through the packed-operand kernel
     (2, 128, "packed", "edges", False),
     (3, 128, "packed", "edges", False),
+    (2, 128, "c8", "all", False),      # group-wise scales on the TMA-fed GEMM, every row
+    (3, 128, "c8", "edges", False),
 ])
 def test_config5_large_scene(which, group, fmt, rows, acc):
     spec = workload.block_specs(4, 0)[which]
