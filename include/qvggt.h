@@ -129,6 +129,9 @@ int qvggt_w4a4_linear(const qvggt_weights_t *w, const unsigned char *Xq, const f
 #define QVGGT_PREP_C8 1
 #define QVGGT_PREP_W8A8 2
 #define QVGGT_PREP_C8_ONLY 4 /* 4-bit codes one per byte only, no packed copy (1 byte per weight; the packed entry points refuse the handle) */
+#define QVGGT_PREP_W_TENSORWISE 8 /* weights with ONE step size for the whole tensor (the tensor-wise arm of Tab. "granularity") instead of one
+                                     per output channel: Delta = max|W~| / qmax, w_scale[n] = Delta for every n; needs QVGGT_PREP_C8_ONLY or
+                                     QVGGT_PREP_W8A8 (otherwise QVGGT_ERR_UNSUPPORTED) */
 int qvggt_rotate_smooth_quantize_c8(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M,
                                     signed char *Xq8, float *a_scale, void *cuda_stream);
 int qvggt_w4a4_linear_c8(const qvggt_weights_t *w, const signed char *Xq8, const float *a_scale, int M,

@@ -263,13 +263,19 @@ def bf16_to_f32(bits: np.ndarray) -> np.ndarray:
     return (np.asarray(bits).astype(np.uint32) << 16).view(np.float32)
 
 
-def prepare_weights(W: np.ndarray, c: np.ndarray, v: np.ndarray | None = None, bits: int = 4):
-    """Offline weight path: fold H and diag(c) into W, quantize per output channel (N = bits).
+def prepare_weights(W: np.ndarray, c: np.ndarray, v: np.ndarray | None = None, bits: int = 4, tensorwise: bool = False):
+    """Offline weight path: fold H and diag(c) into W, quantize per output channel (N = bits), or -- tensorwise, the other arm of
+    Tab. "granularity" -- with one step size for the whole tensor: Delta = max|W~| / qmax = the largest per-row step size, then
+    Eq. "quantization" with that Delta for every row (its clamp cannot act: Delta covers the largest element).
 
     -> dict(wq codes int8 [N, K], wq_packed uint8 [N, K/2] (bits = 4 only), w_scale fp32 [N], amul fp32 [K], wmul fp32 [K])
     """
     amul, wmul = multipliers(c, v)
     wq, w_scale = rotate_smooth_quantize(W, wmul, 0, bits)
+    if tensorwise:
+        delta = np.float32(w_scale.max())
+        wq = rotate_smooth_quantize_static(W, wmul, float(delta), bits)
+        w_scale = np.full(W.shape[0], delta, np.float32)
     return dict(wq=wq, wq_packed=pack_int4(wq) if bits == 4 else None, w_scale=w_scale, amul=amul, wmul=wmul, bits=bits)
 
 

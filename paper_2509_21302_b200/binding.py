@@ -29,6 +29,7 @@ EXPORTS = ("qvggt_prepare_weights", "qvggt_rotate_smooth_quantize", "qvggt_w4a4_
 PREP_C8 = 1   # QVGGT_PREP_C8: keep an int8 [N, K] copy of the weight codes for the *_c8 entry points
 PREP_W8A8 = 2  # QVGGT_PREP_W8A8: 8-bit codes (one per byte only)
 PREP_C8_ONLY = 4  # QVGGT_PREP_C8_ONLY: 4-bit codes one per byte only (no packed copy)
+PREP_W_TENSORWISE = 8  # QVGGT_PREP_W_TENSORWISE: one weight step size for the whole tensor
 
 
 class QvggtError(RuntimeError):
@@ -175,10 +176,11 @@ def _from_device_ptr(ptr: int, nbytes: int, dtype: torch.dtype, shape) -> torch.
 
 
 def prepare_weights(W: torch.Tensor, bias: torch.Tensor | None, smooth_c: torch.Tensor,
-                    sign_v: torch.Tensor | None = None, c8: bool | str = False, bits: int = 4) -> Weights:
+                    sign_v: torch.Tensor | None = None, c8: bool | str = False, bits: int = 4, w_tensorwise: bool = False) -> Weights:
     """W [N,K] bf16, bias [N] bf16 or None, smooth_c [K] fp32, sign_v [K] int8 (+1/-1) or None.
     c8: True = also keep the codes one per byte, as the *_c8 entry points need them; "only" = keep only that copy.
-    bits: 4 (W4A4) or 8 (W8A8: one code per byte only; use the *_c8 entry points)."""
+    bits: 4 (W4A4) or 8 (W8A8: one code per byte only; use the *_c8 entry points).
+    w_tensorwise: one weight step size for the whole tensor instead of one per output channel (needs c8="only" or bits=8)."""
     assert bits in (4, 8) and c8 in (False, True, "only")
     assert W.dim() == 2 and W.element_size() == 2 and W.is_contiguous()
     N, K = W.shape
@@ -189,7 +191,8 @@ def prepare_weights(W: torch.Tensor, bias: torch.Tensor | None, smooth_c: torch.
         assert sign_v.dtype == torch.int8 and sign_v.numel() == K and sign_v.is_contiguous()
     h = ctypes.c_void_p()
     _check(lib().qvggt_prepare_weights(_ptr(W), _ptr(bias), _ptr(smooth_c), _ptr(sign_v), N, K,
-                                       PREP_W8A8 if bits == 8 else (PREP_C8_ONLY if c8 == "only" else (PREP_C8 if c8 else 0)), _stream(),
+                                       (PREP_W8A8 if bits == 8 else (PREP_C8_ONLY if c8 == "only" else (PREP_C8 if c8 else 0))) | (PREP_W_TENSORWISE if w_tensorwise else 0),
+                                       _stream(),
                                        ctypes.byref(h)), "qvggt_prepare_weights")
     return Weights(h.value, N, K)
 

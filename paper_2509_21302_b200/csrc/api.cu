@@ -36,7 +36,10 @@ extern "C" {
 int qvggt_prepare_weights(const void *W_bf16, const void *bias_bf16, const float *smooth_c, const signed char *sign_v,
                           int N, int K, int flags, void *cuda_stream, qvggt_weights_t **out)
 {
-    if (flags & ~(QVGGT_PREP_C8 | QVGGT_PREP_W8A8 | QVGGT_PREP_C8_ONLY)) return QVGGT_ERR_UNSUPPORTED;
+    if (flags & ~(QVGGT_PREP_C8 | QVGGT_PREP_W8A8 | QVGGT_PREP_C8_ONLY | QVGGT_PREP_W_TENSORWISE)) return QVGGT_ERR_UNSUPPORTED;
+    const bool tensorwise = (flags & QVGGT_PREP_W_TENSORWISE) != 0;
+    // the tensor-wise weight quantizer is built on the one-code-per-byte kernels: it needs a handle without packed copy
+    if (tensorwise && !(flags & (QVGGT_PREP_W8A8 | QVGGT_PREP_C8_ONLY))) return QVGGT_ERR_UNSUPPORTED;
     const bool w8 = (flags & QVGGT_PREP_W8A8) != 0;       // 8-bit codes exist one per byte only
     const bool c8 = w8 || (flags & (QVGGT_PREP_C8 | QVGGT_PREP_C8_ONLY)) != 0;
     const bool packed = !w8 && !(flags & QVGGT_PREP_C8_ONLY);
@@ -55,12 +58,12 @@ int qvggt_prepare_weights(const void *W_bf16, const void *bias_bf16, const float
     w->bits = w8 ? 8 : 4;
     w->Wq = nullptr; w->Wq8 = nullptr; w->w_scale = nullptr; w->amul = nullptr; w->bias = nullptr; w->status = nullptr;
     cudaGetDevice(&w->device);
-    float *wmul = nullptr;
+    float *wmul = nullptr;                                   // [K] multipliers, followed by one float for the tensor-wise step size
     bool ok = (!packed || cudaMalloc(&w->Wq, (size_t)N * K / 2) == cudaSuccess) &&
               cudaMalloc(&w->w_scale, sizeof(float) * N) == cudaSuccess &&
               cudaMalloc(&w->amul, sizeof(float) * K) == cudaSuccess &&
               cudaMalloc(&w->status, sizeof(int)) == cudaSuccess &&
-              cudaMallocAsync(&wmul, sizeof(float) * K, st) == cudaSuccess &&
+              cudaMallocAsync(&wmul, sizeof(float) * (K + 4), st) == cudaSuccess &&
               (!bias_bf16 || cudaMalloc(&w->bias, sizeof(uint16_t) * N) == cudaSuccess) &&
               (!c8 || cudaMalloc(&w->Wq8, (size_t)N * K) == cudaSuccess);
     if (!ok) {
@@ -75,6 +78,12 @@ int qvggt_prepare_weights(const void *W_bf16, const void *bias_bf16, const float
     if (e == cudaSuccess) e = qvggt_launch_multipliers(smooth_c, sign_v, K, w->amul, wmul, st);
     if (e == cudaSuccess && w->Wq) e = qvggt_launch_rsq(W_bf16, K, N, K, wmul, 0, w->Wq, w->w_scale, st);
     if (e == cudaSuccess && w->Wq8) e = qvggt_launch_rsq_c8(W_bf16, K, N, K, wmul, w->bits, w->Wq8, w->w_scale, st);
+    if (e == cudaSuccess && tensorwise) {
+        // one step size for the whole tensor (Tab. "granularity"): the largest of the per-row step sizes just computed,
+        // i.e. max|W~| / qmax (the division is monotone), then the static quantizer, which also writes that step as every row's scale
+        e = qvggt_launch_max_reduce(w->w_scale, N, wmul + K, st);
+        if (e == cudaSuccess) e = qvggt_launch_rsq_static_c8(W_bf16, K, N, K, wmul, w->bits, wmul + K, w->Wq8, w->w_scale, st);
+    }
     // wmul is scratch: stream-ordered release so that the call stays asynchronous
     if (cudaFreeAsync(wmul, st) != cudaSuccess) cudaGetLastError();
     if (e != cudaSuccess) {

@@ -41,6 +41,7 @@ cudaError_t qvggt_launch_ln_rsq_c8(const void *X, long long ldx, int M, int K, c
                                    const float *beta, float eps, signed char *Xq8, float *scales, void *ln_out, cudaStream_t st);
 cudaError_t qvggt_launch_gelu_rsq_c8(const void *X, long long ldx, int M, int K, const float *mul, int bits, signed char *Xq8,
                                      float *scales, void *gelu_out, cudaStream_t st);
+cudaError_t qvggt_launch_max_reduce(const float *in, int n, float *out, cudaStream_t st);
 cudaError_t qvggt_launch_colmax(const void *X, int M, int K, float *colmax, cudaStream_t st);
 cudaError_t qvggt_launch_smooth_finalize(const float *ax, const float *aw, int K, float alpha, float lo, float hi,
                                          float *c, cudaStream_t st);

@@ -580,6 +580,24 @@ __global__ void multipliers_kernel(const float *__restrict__ c, const signed cha
     if (wmul) wmul[k] = __fmul_rn(sgn, c[k]);
 }
 
+// out[0] = max_i in[i] (one block; the values are non-negative scales)
+__global__ void __launch_bounds__(1024) max_reduce_kernel(const float *__restrict__ in, int n, float *__restrict__ out)
+{
+    __shared__ float part[32];
+    float m = 0.0f;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) m = fmaxf(m, in[i]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        m = part[threadIdx.x];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+        if (threadIdx.x == 0) out[0] = m;
+    }
+}
+
 __global__ void smooth_finalize_kernel(const float *__restrict__ ax, const float *__restrict__ aw, int K, float alpha,
                                        float lo, float hi, float *__restrict__ c)
 {
@@ -714,6 +732,12 @@ cudaError_t qvggt_launch_rsq(const void *X, long long ldx, int M, int K, const f
     if (K == 1024)
         return group == 128 ? launch_sq<5, 128, false>(x, ldx, M, mul, Xq, scales, st) : launch_sq<5, 0, false>(x, ldx, M, mul, Xq, scales, st);
     return group == 128 ? launch_sq<6, 128, false>(x, ldx, M, mul, Xq, scales, st) : launch_sq<6, 0, false>(x, ldx, M, mul, Xq, scales, st);
+}
+
+cudaError_t qvggt_launch_max_reduce(const float *in, int n, float *out, cudaStream_t st)
+{
+    max_reduce_kernel<<<1, 1024, 0, st>>>(in, n, out);
+    return cudaGetLastError();
 }
 
 cudaError_t qvggt_launch_colmax(const void *X, int M, int K, float *colmax, cudaStream_t st)

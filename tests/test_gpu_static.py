@@ -72,3 +72,32 @@ def test_static_quantizer_full_size_sampled_rows():
     codes = oracle.rotate_smooth_quantize_static(np.ascontiguousarray(spec.x_rows(0, M)[rows]), prep["amul"], float(delta.item()), 4)
     assert np.array_equal(Xq8[torch.from_numpy(rows).cuda()].cpu().numpy(), codes)
     assert torch.all(a_scale == delta)
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+@pytest.mark.parametrize("K,N", [(1024, 384), (4096, 128)])
+def test_tensorwise_weight_quantizer_matches_the_oracle_through_the_layer(K, N, bits):
+    """QVGGT_PREP_W_TENSORWISE (the weight side of Tab. "granularity"): one step size for the whole weight tensor.  Codes and the
+    step bit-exact against the oracle, and the layer built on them reproduces the oracle's sums and outputs."""
+    import workload
+    M = 300
+    spec = workload.LinearSpec("tw", K, N, workload.DIST_NORMAL, 51, 0)
+    W, b, X = spec.weight(), spec.bias(), spec.x_rows(0, M)
+    c = oracle.smooth_factors(spec.x_calib(128), W)
+    prep = oracle.prepare_weights(W, c, None, bits, tensorwise=True)
+    h = q.prepare_weights(dev_bf16(W), dev_bf16(b), torch.from_numpy(c).cuda(), None, c8=("only" if bits == 4 else True), bits=bits, w_tensorwise=True)
+    assert np.array_equal(h.view_c8().cpu().numpy(), prep["wq"])
+    assert np.array_equal(h.view()["w_scale"].cpu().numpy(), prep["w_scale"])
+    ref = oracle.w4a4_linear(X, prep, b, 0)
+    Xq8, a = q.rotate_smooth_quantize_c8(h, dev_bf16(X))
+    acc = torch.zeros((M, N), dtype=torch.int32, device="cuda")
+    Y = q.w4a4_linear_c8(h, Xq8, a, acc_debug=acc)
+    assert np.array_equal(acc.cpu().numpy(), ref["acc"]) and np.array_equal(host_bits(Y), ref["y"])
+    assert h.device_status() == 0
+    h.free()
+    # the flag needs a handle without packed copy
+    import ctypes
+    out = ctypes.c_void_p()
+    Wd, cd = dev_bf16(W), torch.from_numpy(c).cuda()
+    st = q.lib().qvggt_prepare_weights(Wd.data_ptr(), None, cd.data_ptr(), None, N, K, 8, torch.cuda.current_stream().cuda_stream, ctypes.byref(out))
+    assert st == -4 and out.value is None

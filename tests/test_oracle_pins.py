@@ -579,3 +579,26 @@ def test_gelu_bf16_is_the_nearest_bf16_of_the_fp64_value():
     wide = np.zeros((4, 256), np.uint16)
     wide[:, :128] = xb[:4]
     assert np.array_equal(oracle.gelu(wide[:, :128]), out[:4])
+
+
+# ------------------------------------------------------------------ tensor-wise weight quantizer (Tab. "granularity")
+@pytest.mark.parametrize("bits", [4, 8])
+def test_tensorwise_weight_quantizer_bound_extreme_and_reduction_to_channelwise(bits):
+    K, N = 1024, 24
+    qmax = 2 ** (bits - 1) - 1
+    W = workload.normal_bf16(9, 1, N, K, 0.02)
+    c = workload.loguniform_f32(9, 2, K, 0.2, 5.0)
+    tw = oracle.prepare_weights(W, c, None, bits, tensorwise=True)
+    cw = oracle.prepare_weights(W, c, None, bits)
+    delta = tw["w_scale"][0]
+    assert np.all(tw["w_scale"] == delta) and delta == cw["w_scale"].max()          # one step for the tensor: the largest row's
+    y = oracle.rotate_f64(W, tw["wmul"].astype(np.float64))
+    assert abs(delta * qmax - np.abs(y).max()) <= 2.0 ** -20 * np.abs(y).max()       # Delta = max|W~| / qmax
+    assert np.all(np.abs(y - np.float64(delta) * tw["wq"]) <= delta / 2 * (1 + 2.0 ** -12))   # Eq. "quantization": |y - Delta q| <= Delta / 2
+    assert np.abs(tw["wq"]).max() == qmax and tw["wq"].min() >= -qmax                # the largest element reaches +-qmax, nothing clips
+    row = int(np.argmax(cw["w_scale"]))
+    assert np.array_equal(tw["wq"][row], cw["wq"][row])                              # on the row that sets Delta the two quantizers coincide
+    # rows that are sign flips and copies of one row have equal maxima: tensor-wise == channel-wise everywhere
+    W2 = np.stack([W[0], W[0] ^ np.uint16(0x8000), W[0]])
+    a, b = oracle.prepare_weights(W2, c, None, bits, tensorwise=True), oracle.prepare_weights(W2, c, None, bits)
+    assert np.array_equal(a["wq"], b["wq"]) and np.array_equal(a["w_scale"], b["w_scale"])
