@@ -235,7 +235,7 @@ void orc_rotate_smooth_quantize_static(const uint16_t *X, int64_t ldx, int64_t M
  * fp32 once; the multiplier, the absolute maximum and Eq. "quantization" follow unchanged.  This is the reference of
  * the tolerance contract for rotations that do not reproduce the fp32 butterfly order (a tensor-core Hadamard):
  * such a rotation cannot match orc_rotate_smooth_quantize_bits bit for bit, because that one rounds after each of
- * its log2 K stages in one particular order; it is judged by its distance from the exact rotation instead.
+ * its log2 K stages in one particular order; it is measured by its distance from the exact rotation instead.
  *   y_out   fp32 [M, K] or NULL: the rotated, smoothed row fl(fl32(u) * mul) the codes were taken from
  *   abs_sum fp64 [M] or NULL: sum_k |x_k|, the quantity the rounding bound of any fp32 rotation scales with
  * Per-row scales only (group = 0).

@@ -30,7 +30,7 @@ def unpack_codes(packed: np.ndarray) -> np.ndarray:
 
 
 def assert_bf16_within_one_ulp(got_bits: np.ndarray, want_bits: np.ndarray, what: str = "Y") -> float:
-    """Spec tolerance for bf16 outputs: equal or adjacent bf16 values, or |diff| <= 2^-7 |want|.
+    """Tolerance for bf16 outputs: equal or adjacent bf16 values, or |diff| <= 2^-7 |want|.
 
     Returns the fraction of elements that are not bit-equal (expected 0: the kernel uses the same
     separate multiply, multiply, add as the oracle)."""
