@@ -354,8 +354,16 @@ gemm_c8_grouped_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
                 ptx::tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive_cluster(leader_tempty + 8 * b);
+                // two elements per multiply (one issue slot for two IEEE multiplications); the additions stay scalar: a packed
+                // multiply feeding a packed add was seen contracted into one fused operation, one rounding instead of two
+                const uint64_t as2 = ptx::f32x2_pack(as, as);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) sum[j] = __fadd_rn(sum[j], __fmul_rn(static_cast<float>(static_cast<int>(raw[j])), as));
+                for (int j = 0; j < 32; j += 2) {
+                    float p0, p1;
+                    ptx::f32x2_unpack(ptx::f32x2_mul(ptx::f32x2_pack(static_cast<float>(static_cast<int>(raw[j])), static_cast<float>(static_cast<int>(raw[j + 1]))), as2), p0, p1);
+                    sum[j] = __fadd_rn(sum[j], p0);
+                    sum[j + 1] = __fadd_rn(sum[j + 1], p1);
+                }
                 if (DUMP && acc_debug && row_ok) gemmc::dump_acc_x32<0>(acc_debug + ((long long)kb * M + gm) * N + n0, raw);
             }
             if (alive) {
