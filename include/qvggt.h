@@ -115,7 +115,8 @@ int qvggt_w4a4_linear(const qvggt_weights_t *w, const unsigned char *Xq, const f
  * the GEMM spends nothing on unpacking.  Codes, scales, integer sums and outputs are those of the
  * packed entry points, bit for bit; only the layout of Xq differs.  The handle must have been
  * prepared with QVGGT_PREP_C8 in `flags` (which adds an int8 [N, K] copy of Wq to the handle: 1 byte
- * per weight on top of the packed 0.5), otherwise QVGGT_ERR_UNSUPPORTED.  Per-token scales only.
+ * per weight on top of the packed 0.5) or with QVGGT_PREP_C8_ONLY (that copy alone), otherwise
+ * QVGGT_ERR_UNSUPPORTED.  Per-token scales here; the *_c8_grouped pair below takes group-wise scales.
  *   Xq8      int8 [M, K], one code per byte in [-7, 7], natural element order, 16-byte aligned
  *   a_scale  fp32 [M]
  *   Y_bf16, ldy, acc_debug (int32 [M, N]) as for qvggt_w4a4_linear with group 0
@@ -140,7 +141,7 @@ int qvggt_w4a4_linear_c8(const qvggt_weights_t *w, const signed char *Xq8, const
 /*
  * Group-wise activation scales (group = 128, see qvggt_rotate_smooth_quantize / qvggt_w4a4_linear) on codes held one per byte:
  * the same codes, scales, integer partial sums and outputs as the packed entry points with group = 128, bit for bit, on the
- * TMA-fed GEMM (about 4 x faster than the packed group-wise GEMM).  4-bit codes only; the handle needs QVGGT_PREP_C8[_ONLY].
+ * TMA-fed GEMM (about twice as fast as the packed group-wise GEMM).  4-bit codes only; the handle needs QVGGT_PREP_C8[_ONLY].
  *   Xq8      int8 [M, K];  a_scale fp32 [M, K/128];  acc_debug NULL or int32 [K/128, M, N]
  */
 int qvggt_rotate_smooth_quantize_c8_grouped(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M,
