@@ -70,14 +70,19 @@ class Path:
         self.bits = 8 if fmt == "w8a8" else 4
         self.name = fmt + ("_tc" if tc else "")
         if fmt == "c8_w4":
-            # activations one code per byte, weights packed in the handle (0.5 B/weight), unpacked per launch into one scratch
+            # activations one code per byte, weights packed in the handle (0.5 B/weight) and expanded per layer into one
+            # scratch: by the quantize launch itself (exact mode), or by a small kernel in front of the GEMM
             scratch = torch.empty(4096 * 1024, dtype=torch.int8, device="cuda")
             self.prepare = lambda W, b, c: q.prepare_weights(W, b, c, None)
-            self.rsq = (lambda h, x, xq, a: q.rotate_smooth_quantize_tc(h, x, True, xq, a)) if tc else \
-                       (lambda h, x, xq, a: q.rotate_smooth_quantize_c8(h, x, xq, a))
-            self.gemm = lambda h, xq, a, y: q.w4a4_linear_c8_packed_weights(h, xq, a, scratch, y)
+            if tc:
+                self.rsq = lambda h, x, xq, a: q.rotate_smooth_quantize_tc(h, x, True, xq, a)
+                self.gemm = lambda h, xq, a, y: q.w4a4_linear_c8_packed_weights(h, xq, a, scratch, y)
+                self.gemm_kernel = "unpack_w4_kernel + gemm_c8_kernel"
+            else:
+                self.rsq = lambda h, x, xq, a: q.rotate_smooth_quantize_c8_expand(h, x, scratch, xq, a)
+                self.gemm = lambda h, xq, a, y: q.w4a4_linear_c8_expanded(h, xq, a, scratch, y)
+                self.gemm_kernel = "gemm_c8_kernel (weights expanded by the quantize launch)"
             self.new_xq = lambda M, K: torch.empty((M, K), dtype=torch.int8, device="cuda")
-            self.gemm_kernel = "unpack_w4_kernel + gemm_c8_kernel"
         elif fmt in ("c8", "w8a8"):
             self.prepare = lambda W, b, c: q.prepare_weights(W, b, c, None, c8=(True if fmt == "w8a8" else "only"), bits=self.bits)
             self.rsq = (lambda h, x, xq, a: q.rotate_smooth_quantize_tc(h, x, True, xq, a)) if tc else \
@@ -93,6 +98,7 @@ class Path:
             self.new_xq = lambda M, K: torch.empty((M, K // 2), dtype=torch.uint8, device="cuda")
             self.gemm_kernel = "gemm_w4a4_kernel"
         self.rsq_kernel = "rsq_tc_kernel" if tc else "rsq_sq_kernel"
+        self.launches_per_layer = 3 if (fmt == "c8_w4" and tc) else 2
 
 
 def rank_row0(rank: int, rows_per_rank: int) -> int:
@@ -497,11 +503,11 @@ def run_ours(args, rank, world, local_rank):
                             "repeats); the per-kernel durations behind roofline / per_layer come from a further pass of the same steps "
                             "with an event after every launch",
                    "code_format": {"c8": "int4 codes one per byte between the kernels (c8)", "packed": "int4 codes packed two per byte",
-                                   "c8_w4": "activation codes one per byte, weights packed two per byte in the handle (unpacked per launch into an L2-resident scratch)",
+                                   "c8_w4": "activation codes one per byte, weights packed two per byte in the handle (expanded per layer into an L2-resident scratch by the quantize launch)",
                                    "w8a8": "W8A8: int8 codes (Eq. quantization with N = 8), one per byte"}[path.fmt],
                    "quantize_kernel": "tensor-core Hadamard mode (tolerance contract)" if path.tc else "exact fp32 butterflies (bit-exact contract)"},
         "clocks": clocks,
-        "gpu_launches": int(2 * len(specs) * args.steps * len(ms_rep)),
+        "gpu_launches": int(path.launches_per_layer * len(specs) * args.steps * len(ms_rep)),
         "e2e": {"value": world * ops_step / (e2e * 1e-3) / 1e12, "unit": "TOPS", "ms_per_step": e2e,
                 "h2d_bytes_per_step": int(sum(M * s.K * 2 for s in specs)),
                 "d2h_bytes_per_step": int(sum(M * s.N * 2 for s in specs))},
@@ -758,7 +764,7 @@ def measure_stack(q, torch, path, reps=3):
     ops = blocks * sum(layer_ops(M, s) for s in kinds)
     res = {"workload": "48-block linear stack, 32 frames M=43968, activations regenerated per layer (192 tensors, ~30 GB in HBM)",
            "code_format": path.name, "ms": round(ms, 3), "tops": round(ops / (ms * 1e-3) / 1e12, 1), "tokens_per_s": round(M / (ms * 1e-3)),
-           "gpu_launches": 2 * len(layers) * reps, "reps": reps, "setup_s": round(setup_s, 1)}
+           "gpu_launches": path.launches_per_layer * len(layers) * reps, "reps": reps, "setup_s": round(setup_s, 1)}
     for _, h, _x in layers:
         h.free()
     del layers, xq, y

@@ -164,6 +164,25 @@ int qvggt_w4a4_linear_c8_packed_weights(const qvggt_weights_t *w, const signed c
                                         void *cuda_stream);
 
 /*
+ * The same pair of steps for a packed-codes-only handle with the expansion folded into the quantize launch, so that a
+ * layer costs two launches as with a QVGGT_PREP_C8 handle (Tab. "efficiency": the memory footprint of 4-bit weights
+ * without giving up the latency).  qvggt_rotate_smooth_quantize_c8_expand is qvggt_rotate_smooth_quantize_c8 (same
+ * codes and scales bit for bit, per-token scales, 4-bit handles) whose thread blocks, while their first rows are in
+ * flight from memory, also expand the handle's packed weight codes into w_scratch between them;
+ * qvggt_w4a4_linear_c8_expanded is qvggt_w4a4_linear_c8 reading the weight codes from w_scratch.  The caller keeps the
+ * pair together: w_scratch must hold THIS handle's codes, written by an _expand call (or by
+ * qvggt_w4a4_linear_c8_packed_weights) ordered before the GEMM on the same stream, with no other write to it in between.
+ * M = 0: _expand still fills w_scratch; _expanded does nothing.
+ *   w_scratch  int8 [N, K] device scratch supplied by the caller, 16-byte aligned
+ * QVGGT_ERR_UNSUPPORTED: the handle holds no packed codes (QVGGT_PREP_C8_ONLY) or is not 4-bit.
+ */
+int qvggt_rotate_smooth_quantize_c8_expand(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M,
+                                           signed char *Xq8, float *a_scale, signed char *w_scratch, void *cuda_stream);
+int qvggt_w4a4_linear_c8_expanded(const qvggt_weights_t *w, const signed char *Xq8, const float *a_scale, int M,
+                                  void *Y_bf16, long long ldy, const signed char *w_scratch, int *acc_debug,
+                                  void *cuda_stream);
+
+/*
  * The activation path with the bulk of the rotation on the tensor core (Sec. 3.2, Pre-Global-Rotation: the Kronecker
  * recursion H_{2^n} = H_2 (x) H_{2^(n-1)} lets the transform factor over any split of the index bits).  Index bits
  * 3..9 are transformed by one product with the +-1 matrix H_128 (bf16 operands: every product exact, fp32

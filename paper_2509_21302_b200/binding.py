@@ -25,7 +25,8 @@ EXPORTS = ("qvggt_prepare_weights", "qvggt_rotate_smooth_quantize", "qvggt_w4a4_
            "qvggt_layernorm_rotate_smooth_quantize_c8", "qvggt_layernorm", "qvggt_debug_starved_linear_c8",
            "qvggt_rotate_smooth_quantize_tc", "qvggt_rotate_smooth_quantize_tc_c8", "qvggt_gelu",
            "qvggt_gelu_rotate_smooth_quantize_c8", "qvggt_w4a4_linear_c8_packed_weights",
-           "qvggt_rotate_smooth_quantize_c8_grouped", "qvggt_w4a4_linear_c8_grouped")
+           "qvggt_rotate_smooth_quantize_c8_grouped", "qvggt_w4a4_linear_c8_grouped",
+           "qvggt_rotate_smooth_quantize_c8_expand", "qvggt_w4a4_linear_c8_expanded")
 PREP_C8 = 1   # QVGGT_PREP_C8: keep an int8 [N, K] copy of the weight codes for the *_c8 entry points
 PREP_W8A8 = 2  # QVGGT_PREP_W8A8: 8-bit codes (one per byte only)
 PREP_C8_ONLY = 4  # QVGGT_PREP_C8_ONLY: 4-bit codes one per byte only (no packed copy)
@@ -64,6 +65,8 @@ def lib() -> ctypes.CDLL:
         L.qvggt_rotate_smooth_quantize_tc_c8.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp]
         L.qvggt_w4a4_linear_c8_packed_weights.argtypes = [vp, vp, vp, i32, vp, i64, vp, vp, vp]
         L.qvggt_rotate_smooth_quantize_c8_grouped.argtypes = [vp, vp, i64, i32, vp, vp, vp]
+        L.qvggt_rotate_smooth_quantize_c8_expand.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp]
+        L.qvggt_w4a4_linear_c8_expanded.argtypes = [vp, vp, vp, i32, vp, i64, vp, vp, vp]
         L.qvggt_w4a4_linear_c8_grouped.argtypes = [vp, vp, vp, i32, vp, i64, vp, vp]
         L.qvggt_gelu.argtypes = [vp, i64, i32, i32, vp, vp]
         L.qvggt_gelu_rotate_smooth_quantize_c8.argtypes = [vp, vp, i64, i32, vp, vp, vp]
@@ -388,6 +391,37 @@ def w4a4_linear_c8_packed_weights(w: Weights, Xq8: torch.Tensor, a_scale: torch.
     ldy = Y.stride(0) if M > 1 else w.N
     _check(lib().qvggt_w4a4_linear_c8_packed_weights(w.handle, _ptr(Xq8), _ptr(a_scale), M, _ptr(Y), ldy, _ptr(w_scratch), _ptr(acc_debug),
                                                      _stream()), "qvggt_w4a4_linear_c8_packed_weights")
+    return Y
+
+
+def rotate_smooth_quantize_c8_expand(w: Weights, X: torch.Tensor, w_scratch: torch.Tensor, Xq8: torch.Tensor | None = None,
+                                     a_scale: torch.Tensor | None = None):
+    """rotate_smooth_quantize_c8 whose launch also expands the handle's packed weight codes into w_scratch (int8, at
+    least N*K elements) -> (Xq8 [M,K] int8, a_scale [M])."""
+    assert X.dim() == 2 and X.element_size() == 2 and X.stride(1) == 1 and X.shape[1] == w.K
+    assert w_scratch.dtype == torch.int8 and w_scratch.is_contiguous() and w_scratch.numel() >= w.N * w.K
+    M = X.shape[0]
+    if Xq8 is None:
+        Xq8 = torch.empty((M, w.K), dtype=torch.int8, device=X.device)
+    if a_scale is None:
+        a_scale = torch.empty((M,), dtype=torch.float32, device=X.device)
+    _check(lib().qvggt_rotate_smooth_quantize_c8_expand(w.handle, _ptr(X), X.stride(0) if M > 1 else w.K, M, _ptr(Xq8), _ptr(a_scale),
+                                                        _ptr(w_scratch), _stream()), "qvggt_rotate_smooth_quantize_c8_expand")
+    return Xq8, a_scale
+
+
+def w4a4_linear_c8_expanded(w: Weights, Xq8: torch.Tensor, a_scale: torch.Tensor, w_scratch: torch.Tensor,
+                            Y: torch.Tensor | None = None, acc_debug: torch.Tensor | None = None) -> torch.Tensor:
+    """The one-code-per-byte GEMM reading this handle's weight codes from w_scratch, where rotate_smooth_quantize_c8_expand
+    put them."""
+    M = Xq8.shape[0]
+    assert Xq8.dtype == torch.int8 and Xq8.is_contiguous() and Xq8.shape[1] == w.K
+    assert w_scratch.dtype == torch.int8 and w_scratch.is_contiguous() and w_scratch.numel() >= w.N * w.K
+    if Y is None:
+        Y = torch.empty((M, w.N), dtype=torch.bfloat16, device=Xq8.device)
+    ldy = Y.stride(0) if M > 1 else w.N
+    _check(lib().qvggt_w4a4_linear_c8_expanded(w.handle, _ptr(Xq8), _ptr(a_scale), M, _ptr(Y), ldy, _ptr(w_scratch), _ptr(acc_debug),
+                                               _stream()), "qvggt_w4a4_linear_c8_expanded")
     return Y
 
 

@@ -139,6 +139,27 @@ int qvggt_rotate_smooth_quantize_c8(const qvggt_weights_t *w, const void *X_bf16
     return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
 }
 
+int qvggt_rotate_smooth_quantize_c8_expand(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M, signed char *Xq8,
+                                           float *a_scale, signed char *w_scratch, void *cuda_stream)
+{
+    if (!w) return QVGGT_ERR_NULL;
+    if (M < 0) return QVGGT_ERR_SHAPE;
+    if (!w->Wq || w->bits != 4) return QVGGT_ERR_UNSUPPORTED;
+    if (!w_scratch) return QVGGT_ERR_NULL;
+    if (!aligned16(w_scratch)) return QVGGT_ERR_ALIGN;
+    if (M == 0) {
+        // no rows to quantize: the scratch is still filled, by the stand-alone expansion
+        cudaError_t e0 = qvggt_launch_unpack_w4(w, w_scratch, static_cast<cudaStream_t>(cuda_stream));
+        return e0 == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
+    }
+    if (!X_bf16 || !Xq8 || !a_scale) return QVGGT_ERR_NULL;
+    if (ldx < w->K) return QVGGT_ERR_SHAPE;
+    if (ldx % 8 != 0 || !aligned16(X_bf16) || !aligned16(Xq8) || (reinterpret_cast<uintptr_t>(a_scale) & 3u)) return QVGGT_ERR_ALIGN;
+    cudaError_t e = qvggt_launch_rsq_c8(X_bf16, ldx, M, w->K, w->amul, w->bits, Xq8, a_scale, static_cast<cudaStream_t>(cuda_stream), 0,
+                                        w->Wq, w_scratch, (long long)w->N * w->K);
+    return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
+}
+
 int qvggt_rotate_smooth_quantize_c8_grouped(const qvggt_weights_t *w, const void *X_bf16, long long ldx, int M, signed char *Xq8,
                                             float *a_scale, void *cuda_stream)
 {
@@ -304,6 +325,22 @@ int qvggt_w4a4_linear_c8_packed_weights(const qvggt_weights_t *w, const signed c
         return QVGGT_ERR_ALIGN;
     cudaError_t e = qvggt_launch_gemm_c8_packed_weights(w, Xq8, a_scale, M, Y_bf16, ldy, w_scratch, acc_debug, static_cast<cudaStream_t>(cuda_stream));
     if (e == cudaErrorNotSupported) return QVGGT_ERR_UNSUPPORTED;
+    return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
+}
+
+int qvggt_w4a4_linear_c8_expanded(const qvggt_weights_t *w, const signed char *Xq8, const float *a_scale, int M, void *Y_bf16,
+                                  long long ldy, const signed char *w_scratch, int *acc_debug, void *cuda_stream)
+{
+    if (!w) return QVGGT_ERR_NULL;
+    if (M < 0) return QVGGT_ERR_SHAPE;
+    if (w->bits != 4) return QVGGT_ERR_UNSUPPORTED;
+    if (M == 0) return QVGGT_OK;
+    if (!Xq8 || !a_scale || !Y_bf16 || !w_scratch) return QVGGT_ERR_NULL;
+    if (ldy < w->N) return QVGGT_ERR_SHAPE;
+    if (ldy % 8 != 0 || !aligned16(Xq8) || !aligned16(Y_bf16) || !aligned16(w_scratch) || (acc_debug && !aligned16(acc_debug)) ||
+        (reinterpret_cast<uintptr_t>(a_scale) & 3u))
+        return QVGGT_ERR_ALIGN;
+    cudaError_t e = qvggt_launch_gemm_c8_expanded(w, Xq8, a_scale, M, Y_bf16, ldy, w_scratch, acc_debug, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? QVGGT_OK : QVGGT_ERR_CUDA;
 }
 

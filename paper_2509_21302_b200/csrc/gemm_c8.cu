@@ -26,6 +26,7 @@
 #include "qvggt_internal.cuh"
 #include "sm100_ptx.cuh"
 #include "tensor_map.cuh"
+#include "unpack_w4.cuh"
 
 namespace {
 
@@ -485,21 +486,7 @@ __global__ void __launch_bounds__(256) unpack_w4_kernel(const uint4 *__restrict_
     ptx::grid_dependency_wait();           // the scratch may still be read by the previous GEMM of the stream
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n16) return;
-    const uint4 p = __ldg(packed + i);
-    const uint32_t w[4] = {p.x, p.y, p.z, p.w};
-    uint32_t o[8];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            uint32_t x = (w[e] >> (16 * h)) & 0xFFFFu;          // four nibbles
-            x = (x | (x << 8)) & 0x00FF00FFu;
-            x = (x | (x << 4)) & 0x0F0F0F0Fu;                    // one nibble per byte, natural order
-            o[2 * e + h] = x | ((x & 0x08080808u) * 0x1Eu);     // sign extension: bit 3 -> bits 4..7 of its byte
-        }
-    }
-    out[2 * i] = make_uint4(o[0], o[1], o[2], o[3]);
-    out[2 * i + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+    qvggt_unpack_w4_item(packed, out, i);
 }
 
 template <bool DUMP>
@@ -545,10 +532,8 @@ cudaError_t qvggt_launch_gemm_c8(const qvggt_weights *w, const signed char *Xq8,
                      : launch<false>(w, w->Wq8, Xq8, a_scale, M, Y, ldy, acc_debug, st, ptx::kWaitLimitCycles, 0);
 }
 
-cudaError_t qvggt_launch_gemm_c8_packed_weights(const qvggt_weights *w, const signed char *Xq8, const float *a_scale, int M, void *Y,
-                                                long long ldy, signed char *w_scratch, int *acc_debug, cudaStream_t st)
+cudaError_t qvggt_launch_unpack_w4(const qvggt_weights *w, signed char *w_scratch, cudaStream_t st)
 {
-    if (M == 0) return cudaSuccess;
     if (!w->Wq) return cudaErrorNotSupported;       // the handle holds no packed codes
     const long long n16 = (long long)w->N * w->K / 32;
     cudaLaunchAttribute attr;
@@ -560,10 +545,25 @@ cudaError_t qvggt_launch_gemm_c8_packed_weights(const qvggt_weights *w, const si
     cfg.stream = st;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, unpack_w4_kernel, reinterpret_cast<const uint4 *>(w->Wq), reinterpret_cast<uint4 *>(w_scratch), n16);
+    return cudaLaunchKernelEx(&cfg, unpack_w4_kernel, reinterpret_cast<const uint4 *>(w->Wq), reinterpret_cast<uint4 *>(w_scratch), n16);
+}
+
+cudaError_t qvggt_launch_gemm_c8_packed_weights(const qvggt_weights *w, const signed char *Xq8, const float *a_scale, int M, void *Y,
+                                                long long ldy, signed char *w_scratch, int *acc_debug, cudaStream_t st)
+{
+    if (M == 0) return cudaSuccess;
+    cudaError_t e = qvggt_launch_unpack_w4(w, w_scratch, st);
     if (e != cudaSuccess) return e;
     return acc_debug ? launch<true>(w, w_scratch, Xq8, a_scale, M, Y, ldy, acc_debug, st, ptx::kWaitLimitCycles, 0)
                      : launch<false>(w, w_scratch, Xq8, a_scale, M, Y, ldy, acc_debug, st, ptx::kWaitLimitCycles, 0);
+}
+
+cudaError_t qvggt_launch_gemm_c8_expanded(const qvggt_weights *w, const signed char *Xq8, const float *a_scale, int M, void *Y,
+                                          long long ldy, const signed char *w_expanded, int *acc_debug, cudaStream_t st)
+{
+    if (M == 0) return cudaSuccess;
+    return acc_debug ? launch<true>(w, w_expanded, Xq8, a_scale, M, Y, ldy, acc_debug, st, ptx::kWaitLimitCycles, 0)
+                     : launch<false>(w, w_expanded, Xq8, a_scale, M, Y, ldy, acc_debug, st, ptx::kWaitLimitCycles, 0);
 }
 
 cudaError_t qvggt_launch_gemm_c8_starved(const qvggt_weights *w, const signed char *Xq8, const float *a_scale, int M, void *Y,

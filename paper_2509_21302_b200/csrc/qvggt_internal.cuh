@@ -34,7 +34,8 @@ cudaError_t qvggt_launch_multipliers(const float *c, const signed char *v, int K
 cudaError_t qvggt_launch_rsq(const void *X, long long ldx, int M, int K, const float *mul, int group,
                              unsigned char *Xq, float *scales, cudaStream_t st);
 cudaError_t qvggt_launch_rsq_c8(const void *X, long long ldx, int M, int K, const float *mul, int bits, signed char *Xq8,
-                                float *scales, cudaStream_t st, int group = 0);
+                                float *scales, cudaStream_t st, int group = 0, const void *w_packed = nullptr,
+                                void *w_expanded = nullptr, long long w_codes = 0);
 cudaError_t qvggt_launch_rsq_static_c8(const void *X, long long ldx, int M, int K, const float *mul, int bits, const float *delta,
                                        signed char *Xq8, float *scales, cudaStream_t st);
 cudaError_t qvggt_launch_ln_rsq_c8(const void *X, long long ldx, int M, int K, const float *mul, int bits, const float *gamma,
@@ -70,6 +71,11 @@ cudaError_t qvggt_launch_gemm_c8_starved(const qvggt_weights *w, const signed ch
 // small kernel in front of the GEMM.
 cudaError_t qvggt_launch_gemm_c8_packed_weights(const qvggt_weights *w, const signed char *Xq8, const float *a_scale, int M, void *Y,
                                                 long long ldy, signed char *w_scratch, int *acc_debug, cudaStream_t st);
+// The expansion alone.
+cudaError_t qvggt_launch_unpack_w4(const qvggt_weights *w, signed char *w_scratch, cudaStream_t st);
+// The same GEMM on weight codes that an earlier launch of the stream already expanded into w_expanded (int8 [N, K]).
+cudaError_t qvggt_launch_gemm_c8_expanded(const qvggt_weights *w, const signed char *Xq8, const float *a_scale, int M, void *Y,
+                                          long long ldy, const signed char *w_expanded, int *acc_debug, cudaStream_t st);
 // One activation scale per token per 128 rotated channels on one-code-per-byte operands (a_scale [M, K/128]).
 cudaError_t qvggt_launch_gemm_c8_grouped(const qvggt_weights *w, const signed char *Xq8, const float *a_scale, int M, void *Y,
                                          long long ldy, int *acc_debug, cudaStream_t st);

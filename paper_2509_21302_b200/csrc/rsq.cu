@@ -11,6 +11,7 @@
 #include "qvggt_internal.cuh"
 #include "sm100_ptx.cuh"
 #include "tensor_map.cuh"
+#include "unpack_w4.cuh"
 
 namespace {
 
@@ -248,7 +249,7 @@ template <int LOGT, int GROUP, bool C8 = false, int QMAX = 7, bool STATIC = fals
 __global__ void __launch_bounds__(SqGeom<LOGT>::CTA_THREADS, sq_ctas_per_sm(LOGT, LN))
 rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float *__restrict__ mul,
               unsigned char *__restrict__ Xq, float *__restrict__ scales, const float *__restrict__ static_delta,
-              const LnArgs ln)
+              const LnArgs ln, const QvggtExpand ex)
 {
     static_assert(!STATIC || (C8 && GROUP == 0), "the static step size is built for one code per byte");
     static_assert(LN == 0 || (C8 && GROUP == 0 && !STATIC), "the fused LayerNorm is built for the dynamic one-code-per-byte path");
@@ -294,6 +295,12 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
         for (int j = 0; j < CH; ++j) cp_async16(stage + cp_dst[j], src + 16 * (t + T * j));
     }
     cp_async_commit();
+    // Handles that keep the weights at half a byte per code: while the first row's copies are in flight, every block
+    // expands its share of the layer's packed weight codes into the scratch that the GEMM behind this launch reads.
+    if constexpr (C8 && GROUP == 0 && !STATIC && QMAX == 7) {
+        for (long long i = (long long)blockIdx.x * G::CTA_THREADS + threadIdx.x; i < ex.n16; i += (long long)gridDim.x * G::CTA_THREADS)
+            qvggt_unpack_w4_item(ex.packed, ex.out, i);
+    }
     const float delta = STATIC ? __ldg(static_delta) : 0.0f;
     // LayerNorm parameters: one copy per CTA in shared memory behind the row slots, as 16-byte pieces ordered
     // [piece][thread], so that thread t reads its T contiguous gammas with conflict-free 16-byte loads (read straight
@@ -635,7 +642,8 @@ namespace {
 // kernel of the stream drains (they wait in grid_dependency_wait() before touching global memory).
 template <int LOGT, int GROUP, bool C8, int QMAX = 7, bool STATIC = false, int LN = 0>
 cudaError_t launch_sq(const uint16_t *x, long long ldx, int M, const float *mul, unsigned char *out, float *scales,
-                      cudaStream_t st, const float *static_delta = nullptr, LnArgs ln = LnArgs{nullptr, nullptr, 0.0f, nullptr})
+                      cudaStream_t st, const float *static_delta = nullptr, LnArgs ln = LnArgs{nullptr, nullptr, 0.0f, nullptr},
+                      QvggtExpand ex = QvggtExpand{nullptr, nullptr, 0})
 {
     using G = SqGeom<LOGT>;
     constexpr int SMEM = G::SMEM + ((LN == 1 || LN == 2) ? 2 * G::K * 4 : 0);   // + the CTA's copy of gamma and beta
@@ -651,23 +659,39 @@ cudaError_t launch_sq(const uint16_t *x, long long ldx, int M, const float *mul,
     attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr.val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(rsq_grid(M, G::ROWS, sq_ctas_per_sm(LOGT, LN)));
+    int grid = rsq_grid(M, G::ROWS, sq_ctas_per_sm(LOGT, LN));
+    if (ex.n16 > 0) {
+        // enough blocks for the expansion even when there are few rows (blocks without rows only expand)
+        const long long want = (ex.n16 + G::CTA_THREADS - 1) / G::CTA_THREADS;
+        const int cap = rsq_grid(1 << 30, G::ROWS, sq_ctas_per_sm(LOGT, LN));
+        const int need = (int)(want < cap ? want : cap);
+        if (grid < need) grid = need;
+    }
+    cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(G::CTA_THREADS);
     cfg.dynamicSmemBytes = SMEM;
     cfg.stream = st;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, rsq_sq_kernel<LOGT, GROUP, C8, QMAX, STATIC, LN>, x, ldx, M, mul, out, scales, static_delta, ln);
+    return cudaLaunchKernelEx(&cfg, rsq_sq_kernel<LOGT, GROUP, C8, QMAX, STATIC, LN>, x, ldx, M, mul, out, scales, static_delta, ln, ex);
 }
 
 }  // namespace
 
 cudaError_t qvggt_launch_rsq_c8(const void *X, long long ldx, int M, int K, const float *mul, int bits, signed char *Xq8,
-                                float *scales, cudaStream_t st, int group)
+                                float *scales, cudaStream_t st, int group, const void *w_packed, void *w_expanded, long long w_codes)
 {
     if (M == 0) return cudaSuccess;
     const uint16_t *x = static_cast<const uint16_t *>(X);
     unsigned char *out = reinterpret_cast<unsigned char *>(Xq8);
+    if (w_packed) {
+        // the same launch also expands w_codes packed weight codes (4-bit, token-wise activations only)
+        if (group != 0 || bits != 4) return cudaErrorNotSupported;
+        const QvggtExpand ex{static_cast<const uint4 *>(w_packed), static_cast<uint4 *>(w_expanded), w_codes / 32};
+        const LnArgs none{nullptr, nullptr, 0.0f, nullptr};
+        return K == 1024 ? launch_sq<5, 0, true>(x, ldx, M, mul, out, scales, st, nullptr, none, ex)
+                         : launch_sq<6, 0, true>(x, ldx, M, mul, out, scales, st, nullptr, none, ex);
+    }
     if (group == 128) {
         if (bits != 4) return cudaErrorNotSupported;
         return K == 1024 ? launch_sq<5, 128, true>(x, ldx, M, mul, out, scales, st) : launch_sq<6, 128, true>(x, ldx, M, mul, out, scales, st);

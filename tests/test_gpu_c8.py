@@ -283,6 +283,47 @@ def test_packed_weights_handle_on_the_one_code_per_byte_gemm(K, N, M):
     only.free()
 
 
+@pytest.mark.parametrize("K,N,M", [(1024, 128, 1), (1024, 384, 700), (4096, 128, 300), (1024, 4096, 10992), (4096, 1024, 5000), (1024, 1024, 0)])
+def test_weight_expansion_folded_into_the_quantize_launch(K, N, M):
+    """The quantize launch that also expands the handle's packed weight codes: codes and scales as without the expansion
+    (the rows are dealt to fewer blocks, the arithmetic per row is the same), the scratch holds the oracle's weight codes
+    and nothing beyond them, and the GEMM reading it gives the oracle's sums and outputs."""
+    spec = workload.LinearSpec("ex", K, N, workload.DIST_NORMAL, 31, 0)
+    W, b = spec.weight(), spec.bias()
+    c = oracle.smooth_factors(spec.x_calib(128), W)
+    prep = oracle.prepare_weights(W, c)
+    h = q.prepare_weights(dev_bf16(W), dev_bf16(b), torch.from_numpy(c).cuda(), None)          # packed codes only
+    scratch = torch.full((N * K + 64,), 0x55, dtype=torch.int8, device="cuda")
+    X = spec.x_rows(0, M) if M else np.zeros((0, K), dtype=np.uint16)
+    Xd = dev_bf16(X) if M else torch.empty((0, K), dtype=torch.bfloat16, device="cuda")
+    Xq8, a = q.rotate_smooth_quantize_c8_expand(h, Xd, scratch)
+    assert np.array_equal(scratch[:N * K].view(N, K).cpu().numpy(), prep["wq"])
+    assert torch.all(scratch[N * K:] == 0x55)
+    if M:
+        rows = np.arange(M) if M <= 1500 else np.unique(np.concatenate([np.arange(0, M, 97), np.arange(M - 300, M), np.arange(300)]))
+        codes, scales = oracle.rotate_smooth_quantize(np.ascontiguousarray(X[rows]), prep["amul"], 0)
+        ridx = torch.from_numpy(rows).cuda()
+        assert np.array_equal(Xq8[ridx].cpu().numpy(), codes) and np.array_equal(a[ridx].cpu().numpy(), scales)
+        Xq_plain, a_plain = q.rotate_smooth_quantize_c8(h, Xd)                                  # every row against the plain launch
+        assert torch.equal(Xq8, Xq_plain) and torch.equal(a, a_plain)
+        acc = torch.zeros((M, N), dtype=torch.int32, device="cuda")
+        Y = q.w4a4_linear_c8_expanded(h, Xq8, a, scratch, acc_debug=acc)
+        acc_ref = oracle.gemm_i32(codes, prep["wq"], 0)
+        assert np.array_equal(acc[ridx].cpu().numpy(), acc_ref)
+        assert np.array_equal(host_bits(Y[ridx]), oracle.epilogue(acc_ref, scales, prep["w_scale"], b))
+        Y2 = q.w4a4_linear_c8_expanded(h, Xq8, a, scratch)
+        assert torch.equal(Y2.view(torch.int16), Y.view(torch.int16))
+    else:
+        assert q.w4a4_linear_c8_expanded(h, Xq8, a, scratch).shape == (0, N)
+    assert h.device_status() == 0
+    h.free()
+    only = q.prepare_weights(dev_bf16(W), None, torch.from_numpy(c).cuda(), None, c8="only")
+    st = q.lib().qvggt_rotate_smooth_quantize_c8_expand(only.handle, Xd.data_ptr(), K, M, Xq8.data_ptr(), a.data_ptr(), scratch.data_ptr(),
+                                                        torch.cuda.current_stream().cuda_stream)
+    assert st == -4                                               # QVGGT_ERR_UNSUPPORTED: no packed codes to expand
+    only.free()
+
+
 @pytest.mark.parametrize("K,N,M", [(1024, 128, 1), (1024, 384, 257), (4096, 256, 300), (4096, 128, 1374)])
 def test_c8_grouped_matches_the_oracle_and_the_packed_grouped_path(K, N, M):
     """Group-128 activation scales on codes held one per byte: codes, scales, per-group integer sums bit-exact against the
