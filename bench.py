@@ -174,7 +174,8 @@ class ClockSampler:
             except Exception:
                 pass
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": smax, "reasons": sorted(reasons),
-                "samples": len(sm), "power_w_max": max(power) if power else None}
+                "samples": len(sm), "power_w_max": max(power) if power else None,
+                "power_w_median": float(np.median(power)) if power else None}
 
 
 def dev_bf16(torch, bits):
