@@ -439,26 +439,45 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
             const uint64_t y = ptx::f32x2_mul(ptx::f32x2_pack(v[k], v[k + 1]), ptx::f32x2_pack(m[k], m[k + 1]));
             ptx::f32x2_unpack(y, v[k], v[k + 1]);
         }
-        // absolute maxima: one per row, or one per 128 consecutive elements (GREGS registers of every thread)
-        float am[NG];
+        // absolute maxima: one per row, or one per 128 consecutive elements (GREGS registers of every thread).  Non-negative
+        // floats order like their bit patterns, so the warp-wide maximum is one integer reduction (redux.sync) per value.
+        float am[NG];          // GROUP == 0: the row's maximum; GROUP == 128: overwritten below by qmax / maximum of every group
 #pragma unroll
         for (int g = 0; g < (STATIC ? 0 : NG); ++g) {
             float a = fmaxf(fabsf(v[g * GREGS]), fabsf(v[g * GREGS + 1]));
 #pragma unroll
             for (int k = 2; k < GREGS; k += 2)     // max(|a|, |x|, |y|) in one instruction
                 asm("max.abs.f32 %0, %1, %2, %3;" : "=f"(a) : "f"(a), "f"(v[g * GREGS + k]), "f"(v[g * GREGS + k + 1]));
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, o));
-            am[g] = a;
+            am[g] = __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(a)));
         }
-        if (T == 64 && !STATIC) {
-            if (lane == 0) {
+        if constexpr (GROUP == 128) {
+            // One lane per group finishes it: floor, the two divisions (scale = max / qmax is stored from here, 128 bytes
+            // per row in one piece; qmax / max goes back to every thread), instead of NG divisions in every thread.
+            float mine;                                        // the maximum of group `lane mod NG`
+            if constexpr (T == 64) {
+                static_assert(NG == 32, "one group per lane");
+                if (lane == 0) {
 #pragma unroll
-                for (int g = 0; g < NG; ++g) red[(t >> 5) * NG + g] = am[g];
+                    for (int g = 0; g < NG; g += 4)
+                        *reinterpret_cast<float4 *>(red + (t >> 5) * NG + g) = make_float4(am[g], am[g + 1], am[g + 2], am[g + 3]);
+                }
+                group_sync<T>(slot);
+                mine = fmaxf(red[lane], red[NG + lane]);       // both warps of the row compute all 32 (no second exchange)
+            } else {
+                static_assert(NG == 8, "eight groups per row");
+                mine = am[0];
+#pragma unroll
+                for (int g = 1; g < NG; ++g) mine = ((lane & (NG - 1)) == g) ? am[g] : mine;
             }
-            group_sync<T>(slot);
+            mine = fmaxf(mine, 1e-8f);
+            const float inv_mine = __fdiv_rn(static_cast<float>(QMAX), mine);
+            if (t < NG) scales[row * NG + t] = __fdiv_rn(mine, static_cast<float>(QMAX));
 #pragma unroll
-            for (int g = 0; g < NG; ++g) am[g] = fmaxf(red[g], red[NG + g]);
+            for (int g = 0; g < NG; ++g) am[g] = __shfl_sync(0xFFFFFFFFu, inv_mine, g);
+        } else if (T == 64 && !STATIC) {
+            if (lane == 0) red[t >> 5] = am[0];
+            group_sync<T>(slot);
+            am[0] = fmaxf(red[0], red[1]);
         }
         if constexpr (C8) {
             static_assert(QMAX == 7 || QMAX == 127, "4-bit or 8-bit codes");
@@ -467,9 +486,8 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
                 inv = __fdiv_rn(1.0f, delta);
                 am[0] = __fmul_rn(delta, static_cast<float>(QMAX));     // the scale written below is am / QMAX = delta
             } else {
-#pragma unroll
-                for (int g = 0; g < NG; ++g) am[g] = fmaxf(am[g], 1e-8f);
-                inv = __fdiv_rn(static_cast<float>(QMAX), am[0]);
+                if constexpr (GROUP == 0) am[0] = fmaxf(am[0], 1e-8f);
+                inv = (GROUP == 0) ? __fdiv_rn(static_cast<float>(QMAX), am[0]) : 0.0f;
             }
             uint64_t inv2 = ptx::f32x2_pack(inv, inv), inv2b = inv2;
             const uint64_t magic2 = ptx::f32x2_pack(12582912.0f, 12582912.0f);
@@ -480,13 +498,8 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
                 if constexpr (GROUP == 128) {
                     // registers 4 kk .. 4 kk + 3 lie in one scale group (T = 32: GREGS = 4) or in two (T = 64: GREGS = 2)
                     const int g0 = (4 * kk) / GREGS, g1 = (4 * kk + 2) / GREGS;   // compile-time after unrolling
-                    const float i0 = __fdiv_rn(static_cast<float>(QMAX), am[(4 * kk) / GREGS]);
-                    inv2 = ptx::f32x2_pack(i0, i0);
-                    inv2b = inv2;
-                    if (g1 != g0) {
-                        const float i1 = __fdiv_rn(static_cast<float>(QMAX), am[(4 * kk + 2) / GREGS]);
-                        inv2b = ptx::f32x2_pack(i1, i1);
-                    }
+                    inv2 = ptx::f32x2_pack(am[g0], am[g0]);                        // am[] holds qmax / maximum here
+                    inv2b = ptx::f32x2_pack(am[g1], am[g1]);
                 }
                 // exact product + 1.5*2^23, rounded once (half-to-even): the low mantissa byte is the int8 code
                 float f0, f1, f2, f3;
@@ -513,8 +526,8 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
         uint32_t word[T / 8];
 #pragma unroll
         for (int g = 0; g < NG; ++g) {
-            am[g] = fmaxf(am[g], 1e-8f);
-            const float inv = __fdiv_rn(static_cast<float>(QMAX), am[g]);
+            if constexpr (GROUP == 0) am[g] = fmaxf(am[g], 1e-8f);
+            const float inv = (GROUP == 0) ? __fdiv_rn(static_cast<float>(QMAX), am[g]) : am[g];   // GROUP == 128: already qmax / maximum
             const uint64_t inv2 = ptx::f32x2_pack(inv, inv), magic2 = ptx::f32x2_pack(12582912.0f, 12582912.0f);
 #pragma unroll
             for (int k = g * GREGS; k < (g + 1) * GREGS; k += 2) {
@@ -539,10 +552,7 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
             *reinterpret_cast<uint32_t *>(Xq + row * (K / 2) + 4 * ((T / 8) * (8 * kk + (t & 7)) + (t >> 3))) = x;
         }
         }
-        if (t == 0) {
-#pragma unroll
-            for (int g = 0; g < NG; ++g) scales[row * NG + g] = STATIC ? delta : __fdiv_rn(am[g], static_cast<float>(QMAX));
-        }
+        if (GROUP == 0 && t == 0) scales[row] = STATIC ? delta : __fdiv_rn(am[0], static_cast<float>(QMAX));
     }
 }
 
