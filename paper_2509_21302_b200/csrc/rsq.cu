@@ -479,15 +479,22 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
             group_sync<T>(slot);
             am[0] = fmaxf(red[0], red[1]);
         }
+        if constexpr (GROUP == 0 && !STATIC) {
+            // One division sequence yields both quotients: thread 1 of the row divides the other way round and stores the
+            // scale max / qmax; every other lane gets qmax / max, which thread 1 then takes from lane 0.
+            const float amax = fmaxf(am[0], 1e-8f);
+            const bool scale_lane = (t == 1);
+            const float r = __fdiv_rn(scale_lane ? amax : static_cast<float>(QMAX), scale_lane ? static_cast<float>(QMAX) : amax);
+            if (scale_lane) scales[row] = r;
+            am[0] = __shfl_sync(0xFFFFFFFFu, r, 0);            // am[0] = qmax / maximum from here on
+        }
         if constexpr (C8) {
             static_assert(QMAX == 7 || QMAX == 127, "4-bit or 8-bit codes");
             float inv;
             if (STATIC) {
                 inv = __fdiv_rn(1.0f, delta);
-                am[0] = __fmul_rn(delta, static_cast<float>(QMAX));     // the scale written below is am / QMAX = delta
             } else {
-                if constexpr (GROUP == 0) am[0] = fmaxf(am[0], 1e-8f);
-                inv = (GROUP == 0) ? __fdiv_rn(static_cast<float>(QMAX), am[0]) : 0.0f;
+                inv = am[0];                                    // qmax / maximum (GROUP == 128: replaced per group below)
             }
             uint64_t inv2 = ptx::f32x2_pack(inv, inv), inv2b = inv2;
             const uint64_t magic2 = ptx::f32x2_pack(12582912.0f, 12582912.0f);
@@ -526,8 +533,7 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
         uint32_t word[T / 8];
 #pragma unroll
         for (int g = 0; g < NG; ++g) {
-            if constexpr (GROUP == 0) am[g] = fmaxf(am[g], 1e-8f);
-            const float inv = (GROUP == 0) ? __fdiv_rn(static_cast<float>(QMAX), am[g]) : am[g];   // GROUP == 128: already qmax / maximum
+            const float inv = am[g];                            // qmax / maximum of the row or of the group
             const uint64_t inv2 = ptx::f32x2_pack(inv, inv), magic2 = ptx::f32x2_pack(12582912.0f, 12582912.0f);
 #pragma unroll
             for (int k = g * GREGS; k < (g + 1) * GREGS; k += 2) {
@@ -552,7 +558,7 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
             *reinterpret_cast<uint32_t *>(Xq + row * (K / 2) + 4 * ((T / 8) * (8 * kk + (t & 7)) + (t >> 3))) = x;
         }
         }
-        if (GROUP == 0 && t == 0) scales[row] = STATIC ? delta : __fdiv_rn(am[0], static_cast<float>(QMAX));
+        if (STATIC && t == 0) scales[row] = delta;
     }
 }
 
