@@ -243,12 +243,16 @@ rsq_tc_kernel(const __grid_constant__ CUtensorMap map_x, int M, const float *__r
             float *ex = exch + b * 128;
             if (lane < TOK_G) ex[lane * 4 + quarter] = __uint_as_float(mine);
             asm volatile("bar.sync %0, %1;" ::"r"(1 + cg), "r"(128) : "memory");
+            // lanes 0 .. TOK_G-1 compute qmax / max of their token, lanes TOK_G .. 2 TOK_G-1 the scale max / qmax of the same tokens:
+            // one division sequence for both quotients
             float inv_mine = 0.0f;
-            if (lane < TOK_G) {
-                const float4 q4 = *reinterpret_cast<const float4 *>(ex + lane * 4);
+            if (lane < 2 * TOK_G) {
+                const int tok = lane & (TOK_G - 1);
+                const bool scale_lane = lane >= TOK_G;
+                const float4 q4 = *reinterpret_cast<const float4 *>(ex + tok * 4);
                 const float amax = fmaxf(fmaxf(fmaxf(q4.x, q4.y), fmaxf(q4.z, q4.w)), 1e-8f);
-                inv_mine = __fdiv_rn(static_cast<float>(QMAX), amax);
-                if (alive && quarter == 0 && row0 + lane < M) scales[row0 + lane] = __fdiv_rn(amax, static_cast<float>(QMAX));
+                inv_mine = __fdiv_rn(scale_lane ? amax : static_cast<float>(QMAX), scale_lane ? static_cast<float>(QMAX) : amax);
+                if (scale_lane && alive && quarter == 0 && row0 + tok < M) scales[row0 + tok] = inv_mine;
             }
             const uint64_t magic2 = ptx::f32x2_pack(12582912.0f, 12582912.0f);
 #pragma unroll
