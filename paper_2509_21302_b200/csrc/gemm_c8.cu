@@ -281,7 +281,6 @@ gemm_c8_grouped_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     const uint32_t bar_tempty = bar_tfull + GACC * 8;
     uint32_t *s_tmem = reinterpret_cast<uint32_t *>(smem + OFF_TMEM);
     volatile int *s_abort = reinterpret_cast<volatile int *>(smem + OFF_ABORT);
-    volatile int *s_flags = reinterpret_cast<volatile int *>(smem + OFF_FLAGS);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();
@@ -323,7 +322,6 @@ gemm_c8_grouped_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         const uint32_t leader_tempty = ptx::map_to_cta(bar_tempty, 0);
         const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
         bool alive = true;
-        uint32_t toggle = 0;
         int it = 0;                                                 // K-blocks seen so far (all tiles)
         for (int t = 0; t < my_tiles; ++t) {
             const int tile = worker + t * workers;
@@ -345,8 +343,11 @@ gemm_c8_grouped_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
                 const int b = it % GACC;
                 const float as = as_next;
                 if (kb + 1 < KB && row_ok) as_next = __ldg(a_scale + (long long)gm * KB + kb + 1);
-                alive = ptx::mbar_wait_group(bar_tfull + 8 * b, (it / GACC) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM,
-                                             threadIdx.x == 32, 1, GEPI * 32, s_flags, toggle, 0) && alive;   // the poller sits on another scheduler than the MMA thread
+                {   // every warp polls for itself (lane 0; the warp follows): no warp waits for a slower one between K-blocks
+                    int ok = 1;
+                    if (lane == 0) ok = (alive && ptx::mbar_wait(bar_tfull + 8 * b, (it / GACC) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM, 20)) ? 1 : 0;
+                    alive = __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
+                }
                 ptx::tc_fence_after_sync();
                 if (!alive) continue;
                 uint32_t raw[32];
@@ -367,6 +368,8 @@ gemm_c8_grouped_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
                 }
                 if (DUMP && acc_debug && row_ok) gemmc::dump_acc_x32<0>(acc_debug + ((long long)kb * M + gm) * N + n0, raw);
             }
+            // once per tile the epilogue warps meet: publishes s_ws / s_bs of this tile and orders their reuse two tiles on
+            asm volatile("bar.sync %0, %1;" ::"r"(1), "r"(GEPI * 32) : "memory");
             if (alive) {
                 const float *wsb = s_ws + tb * GN + cpart * 32;
                 const float *bsb = s_bs + tb * GN + cpart * 32;

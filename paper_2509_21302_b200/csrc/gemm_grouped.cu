@@ -120,7 +120,6 @@ gemm_w4a4_grouped_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
         float *s_ws = reinterpret_cast<float *>(smem + OFF_CH);    // [2][BN]
         float *s_bs = s_ws + 2 * BN;                                // [2][BN]
         bool alive = true;
-        uint32_t toggle = 0;
         int it = 0;                                                 // K-blocks seen so far (all tiles)
         for (int t = 0; t < my_tiles; ++t) {
             const int tile = worker + t * workers;
@@ -131,9 +130,11 @@ gemm_w4a4_grouped_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
             const int gm = m0 + lane;
             const bool row_ok = gm < M;
             if (threadIdx.x < BN) {
-                // buffer tb was last read two tiles ago; every epilogue warp has passed a group barrier since
+                // buffer tb was last read two tiles ago; every epilogue warp has passed the barrier of the tile in between since
                 gemmc::load_channel_params(s_ws + tb * BN, s_bs + tb * BN, w_scale, bias, nt0, N, threadIdx.x);
             }
+            // once per tile the epilogue warps meet: publishes s_ws / s_bs of this tile and orders their reuse two tiles on
+            asm volatile("bar.sync %0, %1;" ::"r"(1), "r"(EPI_WARPS * 32) : "memory");
             // the group's activation scale is fetched one K-block ahead: it comes from L2, several hundred cycles away
             float as_next = row_ok ? __ldg(a_scale + (long long)gm * KB) : 0.0f;
 #pragma unroll 1
@@ -143,10 +144,11 @@ gemm_w4a4_grouped_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                 // a_scale / 256: exact, cancels the factor 256 carried by the raw accumulator
                 const float as = __fmul_rn(as_next, 0.00390625f);
                 if (!last && row_ok) as_next = __ldg(a_scale + (long long)gm * KB + kb + 1);
-                // polled without back-off: this wait sits on the critical path of every K-block, and a sleep, however short
-                // it is asked to be, costs of the order of a microsecond
-                alive = ptx::mbar_wait_group(bar_tfull + 8 * b, (it >> 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM,
-                                             threadIdx.x == 0, 1, EPI_WARPS * 32, s_flags, toggle, 0) && alive;
+                {   // every warp polls for itself (lane 0; the warp follows): no warp waits for a slower one between K-blocks
+                    int ok = 1;
+                    if (lane == 0) ok = (alive && ptx::mbar_wait(bar_tfull + 8 * b, (it >> 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM, 20)) ? 1 : 0;
+                    alive = __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
+                }
                 ptx::tc_fence_after_sync();
                 if (!alive) continue;
                 const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
