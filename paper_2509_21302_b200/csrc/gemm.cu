@@ -140,7 +140,6 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         float *s_bs = s_ws + ACC_BUFS * BN;                                   // [2][BN] bias as fp32
         const uint32_t leader_tempty = ptx::map_to_cta(bar_tempty, 0);
         bool alive = true;
-        uint32_t toggle = 0;
         for (int t = 0; t < my_tiles; ++t) {
             const int tile = worker + t * workers;
             const int m0 = (tile / n_tiles) * (BM * CG) + (int)rank * BM + quarter * 32;
@@ -156,9 +155,13 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             // a_scale / 256: exact (power of two), cancels the factor 256 carried by the raw accumulator
             const float as = row_ok ? __fmul_rn(__ldg(a_scale + gm), 0.00390625f) : 0.0f;
             const uint64_t as2 = ptx::f32x2_pack(as, as);
-            // one thread polls for all epilogue warps (named barrier 1); the barrier also publishes s_ws / s_bs
-            alive = ptx::mbar_wait_group(bar_tfull + 8 * b, (t >> 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM,
-                                         threadIdx.x == 0, 1, EPI_WARPS * 32, s_flags, toggle, 64) && alive;
+            // the epilogue warps meet (named barrier 1: publishes s_ws / s_bs), then every warp polls the accumulator barrier itself
+            asm volatile("bar.sync %0, %1;" ::"r"(1), "r"(EPI_WARPS * 32) : "memory");
+            {
+                int ok = 1;
+                if (lane == 0) ok = (alive && ptx::mbar_wait(bar_tfull + 8 * b, (t >> 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM, 32)) ? 1 : 0;
+                alive = __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
+            }
             ptx::tc_fence_after_sync();
             if (alive) {
                 const float *wsb = s_ws + b * BN + chalf * 128;

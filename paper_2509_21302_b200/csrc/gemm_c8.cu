@@ -76,7 +76,6 @@ gemm_c8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     const uint32_t bar_tempty = bar_tfull + ACC_BUFS * 8;
     uint32_t *s_tmem = reinterpret_cast<uint32_t *>(smem + OFF_TMEM);
     volatile int *s_abort = reinterpret_cast<volatile int *>(smem + OFF_ABORT);
-    volatile int *s_flags = reinterpret_cast<volatile int *>(smem + OFF_FLAGS);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();                       // 0 = leader of the pair
@@ -119,7 +118,6 @@ gemm_c8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         float *s_bs = s_ws + ACC_BUFS * BN;                                  // [2][BN] bias as fp32
         const uint32_t leader_tempty = ptx::map_to_cta(bar_tempty, 0);
         bool alive = true;
-        uint32_t toggle = 0;
         constexpr int CW = BN / 2, NCH = CW / 32;              // columns and 32-column chunks of one warp's part
         for (int t = 0; t < my_tiles; ++t) {
             const int tile = worker + t * workers;
@@ -135,9 +133,13 @@ gemm_c8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             gemmc::load_channel_params(s_ws + b * BN, s_bs + b * BN, w_scale, bias, nt0, N, threadIdx.x);
             const float as = row_ok ? __ldg(a_scale + gm) : 0.0f;
             const uint64_t as2 = ptx::f32x2_pack(as, as);
-            // one thread polls for all epilogue warps (named barrier 1); the barrier also publishes s_ws / s_bs
-            alive = ptx::mbar_wait_group(bar_tfull + 8 * b, (t >> 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM,
-                                         threadIdx.x == 0, 1, EPI_WARPS * 32, s_flags, toggle, 64, wait_limit) && alive;
+            // the epilogue warps meet (named barrier 1: publishes s_ws / s_bs), then every warp polls the accumulator barrier itself
+            asm volatile("bar.sync %0, %1;" ::"r"(1), "r"(EPI_WARPS * 32) : "memory");
+            {
+                int ok = 1;
+                if (lane == 0) ok = (alive && ptx::mbar_wait(bar_tfull + 8 * b, (t >> 1) & 1, s_abort, status, QVGGT_DEV_TIMEOUT_ACCUM, 32, wait_limit)) ? 1 : 0;
+                alive = __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
+            }
             ptx::tc_fence_after_sync();
             if (alive) {
                 const float *wsb = s_ws + b * BN + cpart * CW;
