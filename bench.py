@@ -577,12 +577,22 @@ def measure_single(q, torch, peaks):
             p.gemm(h, xq, a, y)
 
         us = back_to_back_us(torch, step, reps=200)
+        # the same two launches captured once into a CUDA graph and replayed: what a launch-bound serving loop would do
+        graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            step()
+            torch.cuda.synchronize()
+            with torch.cuda.graph(graph, stream=side):
+                step()
+        torch.cuda.synchronize()
+        us_graph = back_to_back_us(torch, lambda i: graph.replay(), reps=200)
         flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
         cold = timed_us(torch, step, 20, flush)
         assert h.device_status() == 0
         ops = layer_ops(F, s)
-        out[fmt] = {"us_back_to_back": round(us, 2), "us_cold_l2": round(cold, 2), "tops_back_to_back": round(ops / us / 1e6, 1),
-                    "tokens_per_s": round(F / (us * 1e-6))}
+        out[fmt] = {"us_back_to_back": round(us, 2), "us_graph_replay": round(us_graph, 2), "us_cold_l2": round(cold, 2),
+                    "tops_back_to_back": round(ops / us / 1e6, 1), "tokens_per_s": round(F / (us * 1e-6))}
+        del graph
         h.free()
         del flush
     return out
