@@ -366,6 +366,9 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
                 uint4 *dst = reinterpret_cast<uint4 *>(ln.out + row * K + T * t);
 #pragma unroll
                 for (int k = 0; k < T / 8; ++k) dst[k] = make_uint4(packed[4 * k], packed[4 * k + 1], packed[4 * k + 2], packed[4 * k + 3]);
+                // every thread of the row has read its share of this stage before any of them starts the copy that will
+                // overwrite it (the next iteration's prefetch goes into this buffer; the other paths meet further down)
+                group_sync<T>(slot);
                 continue;
             }
             stages_in_registers<T, true>(v);    // strides 1 .. T/2
@@ -419,7 +422,7 @@ rsq_sq_kernel(const uint16_t *__restrict__ X, long long ldx, int M, const float 
                 uint4 *dst = reinterpret_cast<uint4 *>(ln.out + row * K + T * t);
 #pragma unroll
                 for (int k = 0; k < T / 8; ++k) dst[k] = make_uint4(packed[4 * k], packed[4 * k + 1], packed[4 * k + 2], packed[4 * k + 3]);
-                continue;
+                continue;                       // (the row sums above already made the row's threads meet after their reads of the stage)
             }
             stages_in_registers<T, true>(v);    // strides 1 .. T/2
         } else {

@@ -111,6 +111,29 @@ def test_fused_gelu_through_fc2_matches_the_oracle_layer_on_the_activated_input(
     h.free()
 
 
+@pytest.mark.parametrize("which,frames", [(3, 8), (1, 8), (3, 32)])
+def test_fused_gelu_full_size_every_row(which, frames):
+    """The fc2 input of the block (K = 4096; K = 1024 as well) at 8 and 32 frames through the GELU kernel and the fused
+    GELU -> rotate -> smooth -> quantize kernel: every row of the activation within one bf16 ulp of the oracle's GELU,
+    and every row of codes and scales equal to the oracle's quantizer on the GPU's own bf16 GELU output.  (Many rows per
+    thread block: the blocks walk through their rows with a two-deep staging ring.)"""
+    spec = workload.block_specs(0, 0)[which]
+    M = frames * workload.TOKENS_PER_FRAME
+    W = spec.weight()
+    pre = workload.LinearSpec("pre", spec.K, 128, workload.DIST_NORMAL, 47, 0).x_rows(0, M)
+    c = oracle.smooth_factors(oracle.gelu(pre[:256]), W)
+    prep = oracle.prepare_weights(W, c)
+    h = q.prepare_weights(dev_bf16(W), None, torch.from_numpy(c).cuda(), None, c8="only")
+    Xd = dev_bf16(pre)
+    act = host_bits(q.gelu(Xd))
+    assert_gelu_within_one_ulp(act, oracle.gelu(pre))
+    Xq, a = q.gelu_rotate_smooth_quantize_c8(h, Xd)
+    codes, scales = oracle.rotate_smooth_quantize(act, prep["amul"], 0)
+    assert np.array_equal(Xq.cpu().numpy(), codes) and np.array_equal(a.cpu().numpy(), scales)
+    assert h.device_status() == 0
+    h.free()
+
+
 def test_gelu_entry_points_validate_their_arguments():
     L = q.lib()
     X = torch.zeros((8, 1024), dtype=torch.bfloat16, device="cuda")
