@@ -204,10 +204,12 @@ def test_w4a4_linear_extreme_codes():
 
 
 # ------------------------------------------------------------------------------ calibration helper
-@pytest.mark.parametrize("K", [1024, 4096])
-def test_calibrate_smooth_matches_oracle(K):
-    spec = workload.LinearSpec("c", K, 256, workload.DIST_NORMAL, 6, 0)
-    Xc, W = spec.x_calib(300), spec.weight()
+@pytest.mark.parametrize("K,N,rows", [(1024, 256, 300), (4096, 256, 300), (1024, 3072, 10992), (4096, 1024, 10992), (1024, 128, 1)])
+def test_calibrate_smooth_matches_oracle(K, N, rows):
+    """Column maxima of the rotated calibration rows and weight rows and Eq. "smooth_factor" on them: a few hundred rows, one
+    row, and the block's own sizes (every thread block then walks through many rows)."""
+    spec = workload.LinearSpec("c", K, N, workload.DIST_NORMAL, 6, 0)
+    Xc, W = spec.x_calib(rows), spec.weight()
     want = oracle.smooth_factors(Xc, W)
     got = q.calibrate_smooth(dev_bf16(Xc), dev_bf16(W)).cpu().numpy()
     assert np.allclose(got, want, rtol=2e-5, atol=0)
