@@ -283,7 +283,8 @@ def test_packed_weights_handle_on_the_one_code_per_byte_gemm(K, N, M):
     only.free()
 
 
-@pytest.mark.parametrize("K,N,M", [(1024, 128, 1), (1024, 384, 700), (4096, 128, 300), (1024, 4096, 10992), (4096, 1024, 5000), (1024, 1024, 0)])
+@pytest.mark.parametrize("K,N,M", [(1024, 128, 1), (1024, 384, 700), (4096, 128, 300), (1024, 4096, 10992), (4096, 1024, 5000), (1024, 1024, 0),
+                                   (1024, 4096, 3), (4096, 3072, 1), (4096, 1024, 43968)])
 def test_weight_expansion_folded_into_the_quantize_launch(K, N, M):
     """The quantize launch that also expands the handle's packed weight codes: codes and scales as without the expansion
     (the rows are dealt to fewer blocks, the arithmetic per row is the same), the scratch holds the oracle's weight codes
