@@ -70,3 +70,40 @@ def test_repeated_launches_agree_bit_for_bit(q, seed):
         h.free()
         del Xd
         torch.cuda.empty_cache()
+
+
+def test_two_streams_share_a_handle(q):
+    """The same handle used from two CUDA streams at once (different inputs and outputs, launches interleaved from the
+    host): the results are those of the same calls made one after the other.  The handle is read-only during launches
+    (its status word apart), tensor maps travel with each launch, and the host-side caches are per device and atomic."""
+    spec = workload.block_specs(0, 0)[2]                         # fc1: K = 1024, N = 4096
+    W, b = spec.weight(), spec.bias()
+    c = oracle.smooth_factors(spec.x_calib(256), W)
+    h = q.prepare_weights(dev_bf16(W), dev_bf16(b), torch.from_numpy(c).cuda(), None, c8=True)
+    M = [5000, 3 * workload.TOKENS_PER_FRAME]
+    X = [dev_bf16(spec.x_rows(0, M[0])), dev_bf16(spec.x_rows(20000, M[1]))]
+    want = []
+    for x in X:                                                  # one after the other on the current stream
+        xq, a = q.rotate_smooth_quantize_c8(h, x)
+        xq4, a4 = q.rotate_smooth_quantize(h, x, 0)
+        want.append((q.w4a4_linear_c8(h, xq, a), q.w4a4_linear(h, xq4, a4, 0), xq, a))
+    torch.cuda.synchronize()
+    assert torch.equal(want[0][0].view(torch.int16), want[0][1].view(torch.int16))
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    got = [[], []]
+    for rep in range(8):
+        for i in (0, 1):
+            with torch.cuda.stream(streams[i]):
+                xq, a = q.rotate_smooth_quantize_c8(h, X[i])
+                y8 = q.w4a4_linear_c8(h, xq, a)
+                xq4, a4 = q.rotate_smooth_quantize(h, X[i], 0)
+                y4 = q.w4a4_linear(h, xq4, a4, 0)
+                got[i].append((y8, y4, xq, a))
+    torch.cuda.synchronize()
+    for i in (0, 1):
+        for y8, y4, xq, a in got[i]:
+            assert torch.equal(xq, want[i][2]) and torch.equal(a, want[i][3])
+            assert torch.equal(y8.view(torch.int16), want[i][0].view(torch.int16))
+            assert torch.equal(y4.view(torch.int16), want[i][0].view(torch.int16))
+    assert h.device_status() == 0
+    h.free()
