@@ -39,6 +39,9 @@
  *   - One process may drive several devices: a handle is bound to the device that was current when it was
  *     prepared, every other call uses the current device, and the library's caches (kernel attributes,
  *     occupancy, SM count) are kept per device.
+ *   - A handle is read-only during launches (its status word apart), so one handle may be used from several
+ *     streams and host threads at once as long as the calls' output buffers and scratch are distinct; preparing and
+ *     freeing a handle must not overlap calls that use it.
  */
 #ifndef QVGGT_H
 #define QVGGT_H
