@@ -217,6 +217,23 @@ def test_c8_entry_points_validate_their_arguments():
     out = ctypes.c_void_p()
     assert L.qvggt_prepare_weights(xp, None, gp, None, N, K, 16, st, ctypes.byref(out)) == UNSUP  # unknown flag
     assert out.value is None
+    # the pair that folds the weight expansion into the quantize launch
+    scratch = torch.zeros(N * K + 32, dtype=torch.int8, device="cuda")
+    sp = scratch.data_ptr()
+    assert L.qvggt_rotate_smooth_quantize_c8_expand(None, xp, K, M, qp, ap, sp, st) == NULL
+    assert L.qvggt_rotate_smooth_quantize_c8_expand(hp, xp, K, M, qp, ap, None, st) == NULL      # no scratch
+    assert L.qvggt_rotate_smooth_quantize_c8_expand(hp, xp, K, M, qp, ap, sp + 8, st) == ALIGN
+    assert L.qvggt_rotate_smooth_quantize_c8_expand(hp, xp, K - 8, M, qp, ap, sp, st) == SHAPE
+    assert L.qvggt_rotate_smooth_quantize_c8_expand(hp, None, K, M, qp, ap, sp, st) == NULL
+    assert L.qvggt_rotate_smooth_quantize_c8_expand(hp, xp, K, -1, qp, ap, sp, st) == SHAPE
+    assert L.qvggt_w4a4_linear_c8_expanded(hp, qp, ap, M, yp, N, None, None, st) == NULL         # no scratch
+    assert L.qvggt_w4a4_linear_c8_expanded(hp, qp, ap, M, yp, N, sp + 8, None, st) == ALIGN
+    assert L.qvggt_w4a4_linear_c8_expanded(hp, qp, ap, M, yp, N - 8, sp, None, st) == SHAPE
+    assert L.qvggt_w4a4_linear_c8_expanded(hp, qp, ap, 0, None, N, None, None, st) == 0          # M = 0 is a no-op
+    h8 = q.prepare_weights(dev_bf16(workload.normal_bf16(1, 1, N, K, 0.02)), None, torch.ones(K, device="cuda"), None, bits=8)
+    assert L.qvggt_rotate_smooth_quantize_c8_expand(h8.handle, xp, K, M, qp, ap, sp, st) == UNSUP    # 8-bit handles hold no packed codes
+    assert L.qvggt_w4a4_linear_c8_expanded(h8.handle, qp, ap, M, yp, N, sp, None, st) == UNSUP
+    h8.free()
     torch.cuda.synchronize()
     assert h.device_status() == 0
 
